@@ -1,0 +1,31 @@
+"""CPU oracle for the chunk-pipelined reduce / broadcast over an object store.
+
+TEST INFRASTRUCTURE ONLY.  Nothing here is part of the product: only ``tests/``, the
+smoke check and the benchmark's CPU-baseline leg may import it.  It is written from the
+paper (Hoplite, arXiv 2002.05814, Section 3) in plain Python + numpy, shares no code
+with the CUDA library and never imports it.
+
+What each module restates:
+
+* ``reduce_tree``    -- Section 3.4.2: d-ary reduce tree, arrival-order placement by the
+                        generalised in-order traversal, k-of-m selection; Section 3.5.2:
+                        removal of a failed node, replacement by the next ready source,
+                        clearing of the ancestors' partial results.
+* ``broadcast_tree`` -- Section 3.4.1: receiver-driven broadcast through the object
+                        directory (one location per query, complete copies preferred,
+                        sender removed while sending); Section 3.5.1: failover of a
+                        receiver whose sender failed, without cyclic dependencies.
+* ``values``         -- the plain definitions the method must reach: the reduce of the
+                        selected objects (in tree association order for fp32 bit patterns,
+                        and left to right in fp64 as the brute-force check) and
+                        byte-identical broadcast copies.
+* ``store``          -- Sections 3.1-3.3: object directory entries (size, locations with a
+                        partial/complete bit, refined to a chunk prefix), Put / Get /
+                        Reduce / Delete (Table 1) driven by a timeline of events.
+
+Parity status of the parts the paper does not fix (also listed in the design doc):
+the tree after a failure that leaves fewer live sources than requested ("shrink"), and
+the broadcast sender choice for more than one send slot per location, are build-defined
+readings -- **parity unpinned** beyond the invariants and brute-force value checks in
+``tests/test_oracle_*.py``.
+"""

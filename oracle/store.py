@@ -1,0 +1,231 @@
+"""Object store + directory driven by a timeline of events (Table 1 and Sections 3.1-3.5).
+
+Test infrastructure (see the package docstring).  One instance stands for the whole cluster:
+every object is one directory entry ``{size, owner, published prefix}`` (Section 3.2 keeps a
+partial/complete bit per location; the prefix in chunks refines it, Section 3.3), a Reduce is a
+:class:`ReduceSchedule` fed with arrivals and failures, a broadcast (many Gets of one id,
+Section 3.4.1) is a :class:`BroadcastSchedule`.  Calls must come in timeline order (equal
+times: failures, then publications, then requests).
+
+"Arrival" of an object is its first publication, which Section 3.2 places at the moment Put is
+called, before the copy has finished.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from .broadcast_tree import BroadcastSchedule
+from .reduce_tree import ReduceSchedule
+from .values import OP_SUM, tree_reduce
+
+OK = 0
+ERR_INVALID, ERR_NOT_FOUND, ERR_EXISTS, ERR_TIMEOUT, ERR_INSUFFICIENT, ERR_FAILED_WORKER = -1, -2, -3, -4, -5, -6
+
+DT_F32, DT_BF16 = 0, 1
+_ELEM = {DT_F32: 4, DT_BF16: 2}
+
+
+class StoreError(Exception):
+    def __init__(self, code: int, msg: str = ""):
+        super().__init__(f"{code}: {msg}")
+        self.code = code
+
+
+class _Entry:
+    def __init__(self, oid, worker, nbytes, dtype, chunk_bytes):
+        self.oid, self.worker, self.nbytes, self.dtype = oid, worker, nbytes, dtype
+        self.C = (nbytes + chunk_bytes - 1) // chunk_bytes
+        self.data = None
+        self.ready_bytes = 0
+        self.alive = True
+        self.t_arrival = -1
+        self.chunk_bytes = chunk_bytes
+
+    @property
+    def ready_chunks(self) -> int:
+        return self.C if self.ready_bytes >= self.nbytes else self.ready_bytes // self.chunk_bytes
+
+    @property
+    def complete(self) -> bool:
+        return self.ready_bytes >= self.nbytes
+
+
+class OracleStore:
+    def __init__(self, chunk_bytes: int, reduce_degree: int, bcast_degree: int, virt_chunk_ns: int = 0):
+        self.chunk_bytes = chunk_bytes
+        self.d_reduce = reduce_degree
+        self.d_bcast = bcast_degree
+        # default virtual chunk time: chunk_bytes at 64 GiB/s, in whole nanoseconds
+        self.tau = virt_chunk_ns if virt_chunk_ns > 0 else max(1, chunk_bytes * 1_000_000_000 // (64 << 30))
+        self.now = 0
+        self.objects: dict[int, _Entry] = {}
+        self.reduces: dict[int, dict] = {}       # target id -> {sched, op, srcs}
+        self.bcasts: dict[int, dict] = {}        # source id -> {sched, dsts}
+        self.dst_of: dict[int, int] = {}         # receiver id -> source id
+
+    # ------------------------------------------------------------------ clock
+    def advance(self, t_ns: int) -> None:
+        if t_ns < self.now:
+            raise StoreError(ERR_INVALID, "time goes forward")
+        self.now = t_ns
+        for b in self.bcasts.values():
+            b["sched"].advance(t_ns)
+
+    # ------------------------------------------------------------------ Table 1
+    def create(self, oid: int, worker: int, nbytes: int, dtype: int) -> None:
+        if oid in self.objects:
+            raise StoreError(ERR_EXISTS)
+        if nbytes <= 0 or nbytes % _ELEM[dtype]:
+            raise StoreError(ERR_INVALID)
+        self.objects[oid] = _Entry(oid, worker, nbytes, dtype, self.chunk_bytes)
+
+    def put(self, oid: int, data: np.ndarray, nbytes: int) -> None:
+        e = self._entry(oid)
+        if not e.alive:
+            raise StoreError(ERR_FAILED_WORKER)
+        if oid in self.reduces or oid in self.dst_of:
+            raise StoreError(ERR_INVALID, "produced by a collective")
+        if nbytes < e.ready_bytes or nbytes > e.nbytes or data.nbytes != e.nbytes:
+            raise StoreError(ERR_INVALID)
+        first = e.data is None
+        e.data = data
+        e.ready_bytes = nbytes
+        if first:
+            e.t_arrival = self.now
+            for r in self.reduces.values():
+                if oid in r["srcs"]:
+                    r["sched"].on_arrival(oid)
+        if oid in self.bcasts:
+            self.bcasts[oid]["sched"].source_progress(self.now, e.ready_chunks)
+
+    def reduce(self, target: int, srcs: list[int], k: int, op: int = OP_SUM, dtype: int = DT_F32) -> None:
+        if target in self.objects:
+            raise StoreError(ERR_EXISTS)
+        n = len(srcs)
+        if not (1 <= k <= n) or len(set(srcs)) != n:
+            raise StoreError(ERR_INVALID)
+        ents = [self._entry(s) for s in srcs]
+        if any(e.dtype != dtype or e.nbytes != ents[0].nbytes for e in ents):
+            raise StoreError(ERR_INVALID)
+        live = [e for e in ents if e.alive]
+        if len(live) < 1:
+            raise StoreError(ERR_INSUFFICIENT)
+        elems = ents[0].nbytes // _ELEM[dtype]
+        self.create(target, -1, elems * 4, DT_F32)
+        sched = ReduceSchedule(srcs, k, self.d_reduce)
+        for e in ents:                       # sources lost before the call never take part
+            if not e.alive:
+                sched.on_fail(e.oid, 0, self._delivered)
+        arrived = sorted((e for e in live if e.data is not None), key=lambda e: (e.t_arrival, srcs.index(e.oid)))
+        for e in arrived:
+            sched.on_arrival(e.oid)
+        self.reduces[target] = {"sched": sched, "op": op, "srcs": list(srcs)}
+
+    def broadcast(self, src: int, dsts: list[int]) -> None:
+        e = self._entry(src)
+        if src in self.bcasts:
+            raise StoreError(ERR_EXISTS)
+        for dd in dsts:
+            de = self._entry(dd)
+            if de.nbytes != e.nbytes or de.dtype != e.dtype or dd in self.dst_of or de.data is not None:
+                raise StoreError(ERR_INVALID)
+        sched = BroadcastSchedule(src, e.C, self.d_bcast, self.tau)
+        sched.advance(self.now)
+        if not e.alive:
+            raise StoreError(ERR_FAILED_WORKER)
+        if e.data is not None:
+            # chunks published before the broadcast existed count as available from t_arrival on
+            sched.source_progress(self.now, e.ready_chunks)
+        self.bcasts[src] = {"sched": sched, "dsts": list(dsts)}
+        for dd in dsts:
+            self.dst_of[dd] = src
+
+    def join(self, dst: int) -> None:
+        if dst not in self.dst_of:
+            raise StoreError(ERR_NOT_FOUND)
+        if not self.objects[dst].alive:
+            raise StoreError(ERR_FAILED_WORKER)
+        self.bcasts[self.dst_of[dst]]["sched"].join(self.now, dst)
+
+    def fail(self, worker: int) -> None:
+        lost = [e for e in self.objects.values() if e.worker == worker and e.alive]
+        for e in lost:
+            e.alive = False
+        for r in self.reduces.values():
+            for e in lost:
+                if e.oid in r["srcs"]:
+                    r["sched"].on_fail(e.oid, e.ready_chunks, self._delivered)
+        for src, b in self.bcasts.items():
+            mine = [e.oid for e in lost if e.oid == src or self.dst_of.get(e.oid) == src]
+            if mine:
+                b["sched"].fail(self.now, mine)
+
+    def delete(self, oid: int) -> None:
+        self._entry(oid)
+        if oid in self.dst_of or any(oid in r["srcs"] for r in self.reduces.values()):
+            raise StoreError(ERR_INVALID, "still referenced")
+        self.objects.pop(oid)
+        if oid in self.reduces:
+            self.reduces.pop(oid)
+        if oid in self.bcasts:
+            b = self.bcasts.pop(oid)
+            for dd in b["dsts"]:
+                self.dst_of.pop(dd, None)
+
+    def get(self, oid: int) -> np.ndarray:
+        """The complete object (read-only), or StoreError(ERR_TIMEOUT) if it cannot complete yet."""
+        e = self._entry(oid)
+        if oid in self.reduces:
+            r = self.reduces[oid]
+            sched: ReduceSchedule = r["sched"]
+            if sched.k == 0:
+                raise StoreError(ERR_INSUFFICIENT)
+            if not sched.full() or any(not self.objects[m].complete for m in sched.members()):
+                raise StoreError(ERR_TIMEOUT)
+            if e.data is None:
+                objs = {m: self.objects[m].data for m in sched.members()}
+                e.data = tree_reduce(sched.obj_at, sched.d, objs, r["op"])
+                e.ready_bytes = e.nbytes
+            return e.data
+        if oid in self.dst_of:
+            if not e.alive:
+                raise StoreError(ERR_FAILED_WORKER)
+            src = self.dst_of[oid]
+            sched: BroadcastSchedule = self.bcasts[src]["sched"]
+            loc = sched.by_obj.get(oid)
+            if loc is None:
+                raise StoreError(ERR_TIMEOUT, "never joined")
+            # blocking on the copy = letting virtual time run until it has landed
+            while not loc.complete and sched._heap:
+                sched.advance(sched._heap[0][0])
+            if not loc.complete:
+                raise StoreError(ERR_TIMEOUT)
+            self.now = max(self.now, sched.now)
+            for b in self.bcasts.values():
+                b["sched"].advance(self.now)
+            if e.data is None:
+                e.data = self.objects[src].data.copy() if src in self.objects else None
+                e.ready_bytes = e.nbytes
+            return e.data
+        if not e.alive:
+            raise StoreError(ERR_FAILED_WORKER)
+        if not e.complete:
+            raise StoreError(ERR_TIMEOUT)
+        return e.data
+
+    # ------------------------------------------------------------------ schedule dump
+    def dump(self, op_id: int) -> list[int]:
+        if op_id in self.reduces:
+            return self.reduces[op_id]["sched"].words(op_id)
+        if op_id in self.bcasts:
+            return self.bcasts[op_id]["sched"].words()
+        raise StoreError(ERR_NOT_FOUND)
+
+    # ------------------------------------------------------------------ helpers
+    def _entry(self, oid: int) -> _Entry:
+        if oid not in self.objects:
+            raise StoreError(ERR_NOT_FOUND)
+        return self.objects[oid]
+
+    def _delivered(self, oid: int) -> int:
+        return self.objects[oid].ready_chunks
