@@ -1,0 +1,184 @@
+/*
+ * hpl -- chunk-pipelined reduce and broadcast over an object store, on one B200 (sm_100a).
+ *
+ * The calls follow the core interface of Hoplite (arXiv 2002.05814, Table 1: Get, Put, Delete,
+ * Reduce) and its Section 3: objects are immutable buffers named by an id and owned by a task
+ * worker; an object directory records, per object, its size and where copies are, each copy
+ * with its progress (Section 3.2; the progress bit is refined here to a prefix counted in
+ * chunks, Section 3.3); Reduce arranges whichever k of n source objects become ready first
+ * into a degree-d tree filled in arrival order (Section 3.4.2); broadcast (many Gets of one
+ * id, Section 3.4.1) forms a receiver-driven tree; a failed worker is taken out and the
+ * schedules are re-formed (Section 3.5).  "Workers" are buffers in this GPU's memory and time
+ * is a clock the caller sets (hpl_advance), so a schedule is a pure function of the timeline.
+ *
+ * Conventions
+ *   - Every function returns HPL_OK (0) or a negative HPL_ERR_* code; nothing throws, nothing
+ *     aborts.  hpl_strerror() names a code.
+ *   - "device" pointers are addresses in the memory of the CUDA device that was current at
+ *     hpl_init(); "host" pointers are ordinary process memory.
+ *   - A context is not thread safe: one thread at a time.
+ *   - Calls are events on the timeline and must come in non-decreasing time; events at the
+ *     same time are to be issued failures first, then creations/puts, then reduce / broadcast /
+ *     join requests (each group by ascending id).
+ *   - All device work is enqueued on the stream given to hpl_init().  No call blocks on the
+ *     device except hpl_get, hpl_get_host, hpl_sync and hpl_shutdown; every wait of a kernel on
+ *     a progress counter is bounded by poll_budget_ns, after which the kernel gives up, records
+ *     HPL_ERR_TIMEOUT and returns (the context stays usable).
+ */
+#ifndef HPL_H_
+#define HPL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HPL_OK                 0
+#define HPL_ERR_INVALID       -1  /* bad argument: null, size 0, misaligned, unsupported dtype/op, time going back */
+#define HPL_ERR_NOT_FOUND     -2  /* unknown object id */
+#define HPL_ERR_EXISTS        -3  /* id already in use (objects are immutable, Section 2) */
+#define HPL_ERR_TIMEOUT       -4  /* the object cannot be complete yet, or a bounded device wait expired */
+#define HPL_ERR_INSUFFICIENT  -5  /* a Reduce is left with no live source */
+#define HPL_ERR_FAILED_WORKER -6  /* the object's only copy was owned by a failed worker */
+#define HPL_ERR_CUDA          -7  /* a CUDA call failed, or the context has no device (schedule-only) */
+#define HPL_ERR_NOMEM         -8  /* the arena is exhausted */
+
+#define HPL_F32  0   /* 32-bit IEEE float */
+#define HPL_BF16 1   /* bfloat16; reduced in fp32, result fp32 */
+
+#define HPL_SUM 0
+#define HPL_MIN 1    /* (b < a) ? b : a ; NaN inputs are outside the contract */
+#define HPL_MAX 2    /* (a < b) ? b : a */
+
+typedef struct hpl_ctx hpl_ctx;
+
+typedef struct hpl_config {
+    uint64_t chunk_bytes;     /* pipelining block (Section 3.3; 4 MB in the paper).  Multiple of 16.  An object
+                                 smaller than this is one chunk. */
+    int32_t  reduce_degree;   /* d of the reduce tree, >= 1 (Section 3.4.2, Eq. 1) */
+    int32_t  bcast_degree;    /* concurrent sends per location, >= 1 (1 = the rule of Section 3.4.1) */
+    uint64_t virt_chunk_ns;   /* virtual time for one chunk to cross one broadcast edge; 0 = chunk_bytes at 64 GiB/s */
+    uint64_t poll_budget_ns;  /* bound on any device-side wait; 0 = 2 s */
+    int32_t  eager;           /* 1: every event also plans and launches what has become runnable (as hpl_progress) */
+    int32_t  plan_ahead;      /* 1: chunks of a published object that are not ready yet are planned too; the
+                                 kernels poll the directory's progress counters for them (bounded) */
+    int32_t  fuse;            /* 1: a subtree whose inputs are all ready is reduced in registers in one pass
+                                 (same association, same bits); 0: every tree node writes its partial result */
+    int32_t  reserved;
+    void*    arena;           /* device memory the library may use for the directory, partial results, reduce
+                                 targets and copies of host objects; owned by the caller, must outlive the
+                                 context.  NULL = schedule-only context (no device work; hpl_get fails). */
+    uint64_t arena_bytes;
+} hpl_config;
+
+/* Creates a context.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Nothing is
+ * allocated on the device: everything lives in cfg->arena.  Pinned host staging of a few KiB is allocated. */
+int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out);
+
+/* Waits for enqueued work, releases host resources.  The arena and all object buffers stay the caller's. */
+int hpl_shutdown(hpl_ctx* ctx);
+
+/* Sets the clock for the events that follow (nanoseconds, non-decreasing).  Transfers of the virtual
+ * broadcast model that land up to t_ns are applied first. */
+int hpl_advance(hpl_ctx* ctx, uint64_t t_ns);
+
+/* Declares a future: object `object_id`, owned by task worker `worker` (>= 0), `total_bytes` long
+ * (a multiple of the element size).  Section 3.1: an ObjectID may be passed around before its value exists. */
+int hpl_create(hpl_ctx* ctx, int64_t object_id, int32_t worker, uint64_t total_bytes, int32_t dtype);
+
+/* Put (Table 1) with a DEVICE buffer, zero-copy.  `buf` points to the whole object (16-byte aligned); `bytes`
+ * is the length of the prefix that is valid now.  The first call publishes the location as partial -- this is
+ * the object's arrival (Section 3.2: the directory is told when Put is called, before the copy is done);
+ * later calls extend the prefix (same `buf`, larger `bytes`); bytes == total marks it complete.  The store
+ * borrows `buf`: the caller must not modify published bytes, nor free it before hpl_delete.  The bytes must
+ * have been written by work enqueued earlier on the context's stream (or be visible before the call). */
+int hpl_put(hpl_ctx* ctx, int64_t object_id, const void* buf, uint64_t bytes);
+
+/* Put (Table 1) with a HOST buffer: the store copies the prefix into its own device memory chunk by chunk,
+ * asynchronously, publishing each chunk as it lands (Section 3.3: the copy into the store is pipelined with
+ * the transfers that consume it).  `buf` must stay valid until hpl_sync/hpl_get returns; pinned memory makes
+ * the copy overlap. */
+int hpl_put_host(hpl_ctx* ctx, int64_t object_id, const void* buf, uint64_t bytes);
+
+/* Reduce (Table 1, Section 3.4.2).  Non-blocking.  Creates `target_id` (fp32, library-owned, in the arena)
+ * from `k_first_ready` of the `n` objects `src_ids` -- those that arrive first; ties by index in src_ids --
+ * combined with `op` in the association order of the degree-d tree.  All sources have dtype `dtype` and one
+ * size.  Sources may be futures. */
+int hpl_reduce(hpl_ctx* ctx, int64_t target_id, const int64_t* src_ids, int32_t n, int32_t k_first_ready,
+               int32_t op, int32_t dtype);
+
+/* Registers `n` receiver copies `dst_ids` of object `src_id` (Section 3.4.1: a group of tasks that Get the
+ * same object).  Each receiver was hpl_create'd with the source's size and dtype and is given its buffer by
+ * hpl_join. */
+int hpl_broadcast(hpl_ctx* ctx, int64_t src_id, const int64_t* dst_ids, int32_t n);
+
+/* Receiver `dst_id` asks for the object now (its Get): the directory gives it one sender and lists it as a
+ * partial copy.  `dst_buf`: device buffer of the object's size (16-byte aligned), caller-owned. */
+int hpl_join(hpl_ctx* ctx, int64_t dst_id, void* dst_buf);
+
+/* Get (Table 1), read-only form (Section 3.3, immutable get): waits until the object is complete, returns a
+ * device pointer into the store (valid until hpl_delete) and its size.  HPL_ERR_TIMEOUT if it cannot be
+ * complete yet (state stays valid; retry after more events).  For a broadcast receiver the wait lets virtual
+ * time run until its copy has landed. */
+int hpl_get(hpl_ctx* ctx, int64_t object_id, const void** dev_ptr, uint64_t* bytes);
+
+/* Get into HOST memory: as hpl_get, then copies the object to `dst` (capacity `cap` bytes) and waits. */
+int hpl_get_host(hpl_ctx* ctx, int64_t object_id, void* dst, uint64_t cap);
+
+/* Takes a task worker out (Section 3.5): every object and receiver copy it owns leaves all trees at once;
+ * its buffers are never read by work enqueued after the call.  Reduce: the next ready source takes the
+ * position, ancestors' partial results are cleared; with no spare left the tree shrinks.  Broadcast: the
+ * receivers it was sending to ask again and resume from what they hold. */
+int hpl_fail(hpl_ctx* ctx, int32_t worker);
+
+/* Delete (Table 1): drops the directory entry (and the collective it names, if it is a reduce target or a
+ * broadcast source).  Library-owned memory returns to the arena; caller buffers may then be freed. */
+int hpl_delete(hpl_ctx* ctx, int64_t object_id);
+
+/* Plans and launches everything that is runnable now (non-blocking). */
+int hpl_progress(hpl_ctx* ctx);
+
+/* Waits for all launched work.  HPL_ERR_TIMEOUT if a device wait expired (the expired work is re-planned by
+ * the next hpl_progress). */
+int hpl_sync(hpl_ctx* ctx);
+
+/* Serialises the schedule of the collective named by its reduce target id or broadcast source id into
+ * `words` (capacity `cap` 64-bit words); `*len` receives the number of words needed (HPL_ERR_INVALID if
+ * cap is too small; *len is still set).
+ *   Reduce:    0x48504C52, target, n, k requested, k now, d, #placements, {object, position}*, object at each
+ *              position (-1 open), parent of each position, #spares, spares*, #edits, then per edit:
+ *              epoch, kind (1 replaced by a spare, 2 position left open, 3 tree shrank), position, object
+ *              that left, object now there, position it moved from, chunks the departed object had
+ *              delivered, chunks the moved object had delivered, #cleared, cleared positions*.
+ *   Broadcast: 0x48504C42, source, d, chunks, virtual chunk time, clock, #joined, then per receiver in join
+ *              order: id, first sender, current sender (-1 none), first chunk fetched from it, join time,
+ *              chunks held, alive, completion time (-1 not yet); #edits, then per edit: epoch, kind
+ *              (1 new sender, 2 waits for a slot, 3 receiver left), receiver, old sender, new sender,
+ *              chunks held, time. */
+int hpl_schedule_dump(hpl_ctx* ctx, int64_t op_id, int64_t* words, uint64_t cap, uint64_t* len);
+
+typedef struct hpl_stats_t {
+    uint64_t kernel_launches;      /* kernels of this library launched so far */
+    uint64_t reduce_tasks;         /* subtree tasks planned */
+    uint64_t fanout_tasks;
+    uint64_t tiles;                /* tiles planned (one CTA iteration each) */
+    uint64_t bytes_read_planned;   /* bytes the planned tasks read */
+    uint64_t bytes_written_planned;
+    uint64_t device_timeouts;      /* bounded waits that expired */
+    uint64_t arena_used;           /* bytes of the arena in use */
+    uint64_t h2d_bytes;            /* copied by hpl_put_host */
+    uint64_t d2h_bytes;            /* copied by hpl_get_host */
+    uint64_t last_kernel_grid;     /* CTAs of the most recent launch */
+    uint64_t reserved[5];
+} hpl_stats_t;
+
+int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);
+
+const char* hpl_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HPL_H_ */

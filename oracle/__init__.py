@@ -23,7 +23,7 @@ What each module restates:
                         partial/complete bit, refined to a chunk prefix), Put / Get /
                         Reduce / Delete (Table 1) driven by a timeline of events.
 
-Parity status of the parts the paper does not fix (also listed in the design doc):
+Parity status of the parts the paper does not fix:
 the tree after a failure that leaves fewer live sources than requested ("shrink"), and
 the broadcast sender choice for more than one send slot per location, are build-defined
 readings -- **parity unpinned** beyond the invariants and brute-force value checks in

@@ -212,7 +212,7 @@ class BroadcastSchedule:
                 self.edits.append([self.epoch, EDIT_REPARENT, o.obj, old.obj, s.obj, o.have, t])
         self._serve_waiting(t)
 
-    # ---- serialisation (layout in the design doc)
+    # ---- serialisation (the word layout the library's schedule dump also produces)
     def words(self) -> list[int]:
         w = [0x48504C42, self.src_id, self.d, self.C, self.tau, self.now, len(self.locs) - 1]
         for r in self.locs[1:]:

@@ -185,7 +185,7 @@ class ReduceSchedule:
         self.edits.append(ReduceEdit(self.epoch, EDIT_SHRINK, dest, old_obj, new_obj, moved_from,
                                      hi_failed, hi_moved, cleared))
 
-    # -- serialisation (the layout both implementations must produce)
+    # -- serialisation (the word layout the library's schedule dump also produces)
     def words(self, target_id: int) -> list[int]:
         w = [0x48504C52, target_id, len(self.src), self.k0, self.k, self.d, len(self.placements)]
         for o, p in self.placements:

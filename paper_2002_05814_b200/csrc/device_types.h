@@ -1,0 +1,105 @@
+// Structures shared by the host planner and the kernels: the device-resident object directory
+// and the wave descriptors that are passed to the kernels as launch parameters.
+#pragma once
+#include <cstdint>
+
+namespace hpl {
+
+// One row of the object directory in device memory (arXiv 2002.05814, Section 3.2: per object its
+// size and, per location, the progress; here one row per copy, progress as a chunk prefix).
+struct DirRow {
+    unsigned long long ptr;     // device address of this copy (0 while unknown)
+    unsigned long long bytes;   // object size
+    unsigned int n_chunks;
+    unsigned int ready_chunks;  // chunks published so far; written by the host (copy engine), polled by kernels
+    unsigned int dtype;
+    unsigned int owner;
+};
+static_assert(sizeof(DirRow) == 32, "directory row layout");
+
+// Error record the kernels write when a bounded wait runs out.
+struct DeviceStatus {
+    unsigned int error;      // 0, or 1 = a wait on a progress counter expired
+    unsigned int row;        // directory row that was waited for
+    unsigned int chunk;      // chunk index that was waited for
+    unsigned int abort;      // set together with error: other CTAs stop waiting
+    unsigned long long waits;  // polls that did not succeed at the first look
+    unsigned long long pad;
+};
+
+constexpr int kTileElems = 4096;        // elements of the reduce output per tile (one CTA iteration)
+constexpr int kReduceThreads = 256;
+constexpr int kMaxAcc = 8;              // accumulators (tree depth that can be fused in registers)
+constexpr int kFanoutTileBytes = 16384;
+constexpr int kFanoutThreads = 256;
+
+enum : uint8_t { OPC_LOAD = 0, OPC_ADD_LOAD = 1, OPC_ADD_ACC = 2 };
+enum : uint8_t { SRC_F32 = 0, SRC_BF16 = 1 };
+
+// One step of a fused subtree evaluation.  LOAD: acc[a] = operand; ADD_LOAD: acc[a] = acc[a] (+) operand;
+// ADD_ACC: acc[a] = acc[a] (+) acc[b].  The result of a task is acc[0].
+struct ReduceStep {
+    uint8_t code;
+    uint8_t a;
+    uint8_t b;
+    uint8_t kind;       // SRC_F32 / SRC_BF16 for loads
+    uint32_t row;       // directory row of the operand
+};
+
+struct ReduceTask {
+    unsigned long long out_ptr;   // fp32 result (partial or target)
+    unsigned long long elems;     // elements in the whole object
+    uint32_t chunk_elems;
+    uint32_t c_begin, c_end;      // chunk range [c_begin, c_end)
+    uint32_t tiles_per_chunk;
+    uint32_t tile_begin;          // index of this task's first tile within the wave
+    uint32_t step_begin, n_steps;
+    uint32_t red_op;
+    uint32_t poll;                // 1: operands' progress counters must be polled before each chunk
+    uint32_t pad;
+};
+
+constexpr int kMaxTasksPerWave = 24;
+constexpr int kMaxStepsPerWave = 640;
+
+struct ReduceWave {
+    const DirRow* dir;
+    DeviceStatus* status;
+    unsigned long long budget_ns;
+    uint32_t n_tasks;
+    uint32_t total_tiles;
+    ReduceTask tasks[kMaxTasksPerWave];
+    ReduceStep steps[kMaxStepsPerWave];
+};
+
+struct FanoutTask {
+    uint32_t src_row;
+    uint32_t c_begin, c_end;
+    uint32_t tiles_per_chunk;
+    uint32_t tile_begin;
+    uint32_t dst_begin, n_dst;
+    uint32_t poll;
+    unsigned long long bytes;        // object size
+    unsigned long long chunk_bytes;
+};
+
+constexpr int kMaxFanoutTasks = 24;
+constexpr int kMaxFanoutDst = 1024;
+
+struct FanoutWave {
+    const DirRow* dir;
+    DeviceStatus* status;
+    unsigned long long budget_ns;
+    uint32_t n_tasks;
+    uint32_t total_tiles;
+    FanoutTask tasks[kMaxFanoutTasks];
+    uint32_t dst_rows[kMaxFanoutDst];
+};
+
+// Launchers (kernels.cu).  Return a cudaError_t as int.
+int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, int grid, void* stream);
+int launch_fanout_wave(const FanoutWave& w, int grid, void* stream);
+int reduce_ctas_per_sm(int n_acc, bool bf16);
+int fanout_ctas_per_sm();
+
+}  // namespace hpl

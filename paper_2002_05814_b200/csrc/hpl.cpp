@@ -1,0 +1,1258 @@
+// Host side of the library: object directory, event handling, planners that turn the current
+// schedules into waves of kernel tasks, and the C ABI (include/hpl.h).
+//
+// Division of labour (arXiv 2002.05814, Section 3): the schedule builders (sched_reduce.*,
+// sched_bcast.*) decide WHO combines / forwards WHAT, as a function of the event timeline only.
+// The planners below decide HOW the pending part of those schedules is executed on the GPU right
+// now: which subtrees of a reduce tree are complete for which chunks (those are fused into one
+// pass in registers), which partial results must be materialised, which receivers can be served
+// from which copy.  Execution order is free as long as the association order of the tree is
+// kept, so the bits do not depend on it.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/hpl.h"
+#include "device_types.h"
+#include "sched_bcast.h"
+#include "sched_reduce.h"
+
+using namespace hpl;
+
+namespace {
+
+constexpr uint32_t kMaxRows = 4096;
+constexpr uint32_t kMaxChunks = 1u << 20;
+constexpr uint64_t kAlign = 256;
+
+// ------------------------------------------------------------------------------------------ small utilities
+struct IntervalSet {  // disjoint, sorted [a, b) chunk ranges
+    std::vector<std::pair<uint32_t, uint32_t>> iv;
+    void clear() { iv.clear(); }
+    bool contains(uint32_t a, uint32_t b) const {
+        for (auto& x : iv)
+            if (x.first <= a && b <= x.second) return true;
+        return false;
+    }
+    void add(uint32_t a, uint32_t b) {
+        if (a >= b) return;
+        std::vector<std::pair<uint32_t, uint32_t>> out;
+        for (auto& x : iv) {
+            if (x.second < a || b < x.first)
+                out.push_back(x);
+            else {
+                a = std::min(a, x.first);
+                b = std::max(b, x.second);
+            }
+        }
+        out.emplace_back(a, b);
+        std::sort(out.begin(), out.end());
+        iv.swap(out);
+    }
+    void remove(uint32_t a, uint32_t b) {
+        std::vector<std::pair<uint32_t, uint32_t>> out;
+        for (auto& x : iv) {
+            if (x.second <= a || b <= x.first) {
+                out.push_back(x);
+                continue;
+            }
+            if (x.first < a) out.emplace_back(x.first, a);
+            if (b < x.second) out.emplace_back(b, x.second);
+        }
+        iv.swap(out);
+    }
+    void breakpoints(std::vector<uint32_t>& bp) const {
+        for (auto& x : iv) {
+            bp.push_back(x.first);
+            bp.push_back(x.second);
+        }
+    }
+};
+
+struct Arena {
+    uint8_t* base = nullptr;
+    uint64_t size = 0, used = 0;
+    std::map<uint64_t, uint64_t> free_;  // offset -> length
+    void init(void* p, uint64_t n) {
+        base = (uint8_t*)p;
+        size = n;
+        used = 0;
+        free_.clear();
+        uint64_t off = (kAlign - ((uintptr_t)p % kAlign)) % kAlign;
+        if (n > off) free_[off] = n - off;
+    }
+    void* alloc(uint64_t n) {
+        n = (n + kAlign - 1) / kAlign * kAlign;
+        for (auto it = free_.begin(); it != free_.end(); ++it) {
+            if (it->second >= n) {
+                const uint64_t off = it->first, len = it->second;
+                free_.erase(it);
+                if (len > n) free_[off + n] = len - n;
+                used += n;
+                sizes_[off] = n;
+                return base + off;
+            }
+        }
+        return nullptr;
+    }
+    void release(void* p) {
+        uint64_t off = (uint8_t*)p - base;
+        auto s = sizes_.find(off);
+        if (s == sizes_.end()) return;
+        uint64_t n = s->second;
+        sizes_.erase(s);
+        used -= n;
+        auto next = free_.lower_bound(off);
+        if (next != free_.end() && off + n == next->first) {
+            n += next->second;
+            next = free_.erase(next);
+        }
+        if (next != free_.begin()) {
+            auto prev = std::prev(next);
+            if (prev->first + prev->second == off) {
+                prev->second += n;
+                return;
+            }
+        }
+        free_[off] = n;
+    }
+    std::map<uint64_t, uint64_t> sizes_;
+};
+
+enum ObjKind { OBJ_PLAIN = 0, OBJ_TARGET = 1, OBJ_RECEIVER = 2, OBJ_PARTIAL = 3 };
+
+struct Object {
+    int64_t id = 0;
+    int32_t worker = -1;
+    uint64_t bytes = 0;
+    int32_t dtype = HPL_F32;
+    uint32_t C = 0;
+    ObjKind kind = OBJ_PLAIN;
+    int64_t op_key = 0;        // receiver: its source id
+    void* ptr = nullptr;
+    bool lib_owned = false;
+    bool from_host = false;
+    uint64_t ready_bytes = 0;  // published prefix
+    uint32_t landed = 0;       // chunks whose counter update is ordered before later launches on the main stream
+    bool alive = true;
+    bool arrived = false;
+    int64_t t_arrival = -1;
+    uint64_t seq = 0;          // creation order
+    int row = -1;
+};
+
+struct Journal {  // what was planned since the last successful sync (undone if a device wait expires)
+    struct R { int64_t target; int pos; uint32_t a, b; };
+    struct B { int64_t src; int loc; int64_t old_have; };
+    std::vector<R> r;
+    std::vector<B> b;
+    void clear() { r.clear(); b.clear(); }
+};
+
+struct PlannedReduceTask {
+    int pos;
+    int level;
+    uint32_t a, b;
+    int n_acc;
+    bool poll;
+    std::vector<ReduceStep> steps;
+};
+
+struct ReduceOp {
+    int64_t target;
+    std::unique_ptr<ReduceTreeSchedule> sched;
+    int red_op, in_dtype;
+    uint64_t elems;
+    uint32_t C, chunk_elems;
+    uint64_t seq;
+    std::vector<IntervalSet> computed;      // per position: chunks of its result that are materialised and valid
+    std::vector<int64_t> partial_key;       // per position: internal object id of its partial buffer (0 none)
+};
+
+struct BcastOp {
+    int64_t src;
+    std::unique_ptr<BroadcastTreeSchedule> sched;
+    std::vector<int64_t> dsts;
+    std::vector<int64_t> phys_have;  // per location index: chunks physically planned (index 0 unused)
+    uint64_t seq;
+};
+
+}  // namespace
+
+struct hpl_ctx {
+    hpl_config cfg{};
+    cudaStream_t stream = nullptr, copy_stream = nullptr;
+    cudaEvent_t copy_ev = nullptr;
+    bool device = false;
+    bool copy_pending = false;
+    int n_sm = 0;
+    uint64_t now = 0, tau = 1, seq = 0;
+    int64_t next_internal = -1;  // ids of partial buffers: negative, never visible outside
+    Arena arena;
+    DirRow* d_dir = nullptr;
+    DirRow* h_dir = nullptr;
+    DeviceStatus* d_status = nullptr;
+    DeviceStatus* h_status = nullptr;
+    uint32_t* h_iota = nullptr;
+    std::vector<int> free_rows;
+    std::unordered_map<int64_t, Object> objects;
+    std::map<uint64_t, ReduceOp> reduces;  // by creation order
+    std::map<uint64_t, BcastOp> bcasts;
+    std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
+    Journal journal;
+    bool work_in_flight = false;
+    hpl_stats_t stats{};
+    int occ_reduce[2][3] = {{0, 0, 0}, {0, 0, 0}};
+    int occ_fanout = 0;
+};
+
+namespace {
+
+inline uint32_t elem_size(int dtype) { return dtype == HPL_BF16 ? 2u : 4u; }
+
+inline uint32_t published_chunks(const hpl_ctx* c, const Object& o) {
+    if (o.ready_bytes >= o.bytes) return o.C;
+    return (uint32_t)(o.ready_bytes / c->cfg.chunk_bytes);
+}
+
+Object* find(hpl_ctx* c, int64_t id) {
+    auto it = c->objects.find(id);
+    return it == c->objects.end() ? nullptr : &it->second;
+}
+
+#define CUDA_TRY(x)                                  \
+    do {                                             \
+        if ((x) != cudaSuccess) return HPL_ERR_CUDA; \
+    } while (0)
+
+int alloc_row(hpl_ctx* c, Object& o) {
+    if (!c->device) return HPL_OK;
+    if (o.row >= 0) return HPL_OK;
+    if (c->free_rows.empty()) return HPL_ERR_NOMEM;
+    o.row = c->free_rows.back();
+    c->free_rows.pop_back();
+    DirRow& r = c->h_dir[o.row];
+    r.ptr = (unsigned long long)(uintptr_t)o.ptr;
+    r.bytes = o.bytes;
+    r.n_chunks = o.C;
+    // rows of library-produced copies are never polled: validity of their bytes is stream order
+    r.ready_chunks = (o.kind == OBJ_PLAIN) ? 0u : o.C;
+    r.dtype = (unsigned)o.dtype;
+    r.owner = (unsigned)o.worker;
+    CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->stream));
+    return HPL_OK;
+}
+
+// Publishes the chunk prefix of a put object in the device directory, ordered on `s`.
+int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
+    if (!c->device || o.row < 0) return HPL_OK;
+    CUDA_TRY(cudaMemcpyAsync(&c->d_dir[o.row].ready_chunks, &c->h_iota[chunks], sizeof(uint32_t), cudaMemcpyHostToDevice, s));
+    return HPL_OK;
+}
+
+int sync_and_check(hpl_ctx* c);
+int progress(hpl_ctx* c);
+
+void release_object_memory(hpl_ctx* c, Object& o) {
+    if (o.lib_owned && o.ptr) c->arena.release(o.ptr);
+    o.ptr = nullptr;
+    if (o.row >= 0) c->free_rows.push_back(o.row);
+    o.row = -1;
+}
+
+// ------------------------------------------------------------------------------------------ reduce planner
+struct ReducePlanCtx {
+    hpl_ctx* c;
+    ReduceOp* op;
+    uint32_t a, b;                 // chunk interval being planned
+    std::vector<uint32_t> ready;   // per position: chunks that may be consumed
+    std::vector<uint32_t> landed;  // per position: chunks known to be visible without polling
+    std::vector<char> done, avail;
+    std::vector<int> level_of;     // level at which the position's result becomes available in this pass
+    std::vector<PlannedReduceTask>* out;
+    int err = HPL_OK;
+};
+
+int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out) {
+    if (pos == 0) {
+        *out = find(c, op.target);
+        return HPL_OK;
+    }
+    if (op.partial_key[pos] != 0) {
+        *out = find(c, op.partial_key[pos]);
+        return HPL_OK;
+    }
+    Object o;
+    o.id = c->next_internal--;
+    o.kind = OBJ_PARTIAL;
+    o.bytes = op.elems * 4;
+    o.dtype = HPL_F32;
+    o.C = op.C;
+    o.lib_owned = true;
+    o.seq = c->seq++;
+    o.ptr = c->arena.alloc(o.bytes);
+    if (!o.ptr) return HPL_ERR_NOMEM;
+    o.ready_bytes = o.bytes;
+    int rc = alloc_row(c, o);
+    if (rc != HPL_OK) {
+        c->arena.release(o.ptr);
+        return rc;
+    }
+    op.partial_key[pos] = o.id;
+    auto ins = c->objects.emplace(o.id, o);
+    *out = &ins.first->second;
+    return HPL_OK;
+}
+
+// Emits the steps that leave the result of subtree `u` in accumulator `acc`.  Children that cannot be
+// fused (fusion switched off, or no accumulator left) are materialised first by tasks of a lower level.
+int ensure_result(ReducePlanCtx& p, int v);
+
+// One load step: the position's own object (partial == false) or its materialised partial result.
+void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial, uint8_t code, int acc) {
+    ReduceOp& op = *p.op;
+    ReduceStep st{};
+    st.code = code;
+    st.a = (uint8_t)acc;
+    if (partial) {
+        st.kind = SRC_F32;
+        st.row = (uint32_t)find(p.c, op.partial_key[q])->row;
+    } else {
+        st.kind = op.in_dtype == HPL_BF16 ? SRC_BF16 : SRC_F32;
+        st.row = (uint32_t)find(p.c, op.sched->object_at(q))->row;
+        if (p.landed[q] < p.b) task.poll = true;  // not yet known to be visible: the kernel polls its counter
+    }
+    task.steps.push_back(st);
+}
+
+void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& dep_level) {
+    ReduceTreeSchedule& s = *p.op->sched;
+    auto is_materialised = [&](int q) { return !s.is_leaf(q) && (p.done[q] || p.level_of[q] >= 0); };
+    task.n_acc = std::max(task.n_acc, acc + 1);
+    if (s.is_leaf(u)) {
+        emit_operand(p, task, u, false, OPC_LOAD, acc);
+        return;
+    }
+    const int c0 = s.first_child(u), nc = s.n_children(u);
+    for (int j = 0; j < nc; ++j) {
+        const int cj = c0 + j;
+        const int acc_j = j == 0 ? acc : acc + 1;            // where a fused subtree of this child would live
+        const uint8_t code = j == 0 ? OPC_LOAD : OPC_ADD_LOAD;
+        if (s.is_leaf(cj)) {
+            emit_operand(p, task, cj, false, code, acc);
+        } else {
+            if (!is_materialised(cj) && (!p.c->cfg.fuse || acc_j >= kMaxAcc)) ensure_result(p, cj);
+            if (p.err != HPL_OK) return;
+            if (is_materialised(cj)) {
+                if (p.level_of[cj] > dep_level) dep_level = p.level_of[cj];
+                emit_operand(p, task, cj, true, code, acc);
+            } else {
+                gen_steps(p, cj, acc_j, task, dep_level);
+                if (j > 0) {
+                    ReduceStep st{};
+                    st.code = OPC_ADD_ACC;
+                    st.a = (uint8_t)acc;
+                    st.b = (uint8_t)acc_j;
+                    task.steps.push_back(st);
+                }
+            }
+        }
+        if (j == 0) emit_operand(p, task, u, false, OPC_ADD_LOAD, acc);  // first child, then the node itself
+    }
+}
+
+// Plans the task that materialises the result of position v over [a, b); returns its level (>= 1).
+int ensure_result(ReducePlanCtx& p, int v) {
+    if (p.err != HPL_OK) return 0;
+    if (p.done[v]) return 0;
+    if (p.level_of[v] >= 0) return p.level_of[v];
+    Object* outbuf = nullptr;
+    int rc = ensure_partial_buffer(p.c, *p.op, v, &outbuf);
+    if (rc != HPL_OK) {
+        p.err = rc;
+        return 0;
+    }
+    PlannedReduceTask task;
+    task.pos = v;
+    task.a = p.a;
+    task.b = p.b;
+    task.n_acc = 1;
+    task.poll = false;
+    int dep = 0;
+    gen_steps(p, v, 0, task, dep);
+    task.level = dep + 1;
+    p.level_of[v] = task.level;
+    p.out->push_back(std::move(task));
+    return p.level_of[v];
+}
+
+void visit_for_progress(ReducePlanCtx& p, int v) {
+    ReduceTreeSchedule& s = *p.op->sched;
+    if (s.is_leaf(v) || p.done[v]) return;
+    if (p.avail[v]) {
+        ensure_result(p, v);
+        return;
+    }
+    const int c0 = s.first_child(v), nc = s.n_children(v);
+    for (int j = 0; j < nc; ++j) visit_for_progress(p, c0 + j);
+}
+
+int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
+    ReduceTreeSchedule& s = *op.sched;
+    const int k = s.k();
+    if (k <= 0) return HPL_OK;
+    std::vector<uint32_t> ready(k, 0), landed(k, 0);
+    std::vector<uint32_t> bp = {0u, op.C};
+    for (int p = 0; p < k; ++p) {
+        op.computed[p].breakpoints(bp);
+        const int64_t oid = s.object_at(p);
+        if (oid < 0) continue;
+        Object* o = find(c, oid);
+        if (!o || !o->alive || !o->ptr || o->row < 0) continue;
+        const uint32_t pub = published_chunks(c, *o);
+        landed[p] = std::min(pub, o->landed);
+        ready[p] = c->cfg.plan_ahead ? o->C : landed[p];
+        bp.push_back(ready[p]);
+        bp.push_back(landed[p]);
+    }
+    std::sort(bp.begin(), bp.end());
+    bp.erase(std::unique(bp.begin(), bp.end()), bp.end());
+
+    for (size_t i = 0; i + 1 < bp.size(); ++i) {
+        ReducePlanCtx p;
+        p.c = c;
+        p.op = &op;
+        p.a = bp[i];
+        p.b = bp[i + 1];
+        if (p.b > op.C) break;
+        p.ready = ready;
+        p.landed = landed;
+        p.done.assign(k, 0);
+        p.avail.assign(k, 0);
+        p.level_of.assign(k, -1);
+        std::vector<PlannedReduceTask> local;
+        p.out = &local;
+        for (int q = k - 1; q >= 0; --q) {
+            p.done[q] = op.computed[q].contains(p.a, p.b) ? 1 : 0;
+            bool av = ready[q] >= p.b;
+            if (!s.is_leaf(q)) {
+                const int c0 = s.first_child(q), nc = s.n_children(q);
+                for (int j = 0; j < nc && av; ++j) av = s.is_leaf(c0 + j) ? (ready[c0 + j] >= p.b) : (p.done[c0 + j] || p.avail[c0 + j]);
+            }
+            p.avail[q] = av ? 1 : 0;
+        }
+        if (s.is_leaf(0)) {
+            // k == 1: the target is a copy of the only member
+            if (!p.done[0] && p.avail[0]) ensure_result(p, 0);
+        } else {
+            visit_for_progress(p, 0);
+        }
+        if (p.err != HPL_OK) return p.err;
+        for (auto& t : local) {
+            op.computed[t.pos].add(t.a, t.b);
+            c->journal.r.push_back({op.target, t.pos, t.a, t.b});
+            // merge with the previous interval's task for the same position when the program is the same
+            bool merged = false;
+            for (auto& prev : tasks) {
+                if (prev.pos == t.pos && prev.b == t.a && prev.level == t.level && prev.poll == t.poll &&
+                    prev.steps.size() == t.steps.size() &&
+                    std::memcmp(prev.steps.data(), t.steps.data(), t.steps.size() * sizeof(ReduceStep)) == 0) {
+                    prev.b = t.b;
+                    merged = true;
+                    break;
+                }
+            }
+            if (!merged) tasks.push_back(std::move(t));
+        }
+    }
+    return HPL_OK;
+}
+
+int occ_index(int n_acc) { return n_acc <= 2 ? 0 : (n_acc <= 4 ? 1 : 2); }
+
+int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
+    if (tasks.empty()) return HPL_OK;
+    int max_level = 0;
+    for (auto& t : tasks) max_level = std::max(max_level, t.level);
+    const bool bf16 = op.in_dtype == HPL_BF16;
+    const uint32_t tpc_full = (op.chunk_elems + kTileElems - 1) / kTileElems;
+    for (int level = 1; level <= max_level; ++level) {
+        size_t i = 0;
+        std::vector<PlannedReduceTask*> lv;
+        for (auto& t : tasks)
+            if (t.level == level) lv.push_back(&t);
+        while (i < lv.size()) {
+            static thread_local ReduceWave w;
+            w.dir = c->d_dir;
+            w.status = c->d_status;
+            w.budget_ns = c->cfg.poll_budget_ns;
+            w.n_tasks = 0;
+            w.total_tiles = 0;
+            uint32_t n_steps = 0;
+            int n_acc = 1;
+            while (i < lv.size() && w.n_tasks < (uint32_t)kMaxTasksPerWave &&
+                   n_steps + lv[i]->steps.size() <= (size_t)kMaxStepsPerWave) {
+                PlannedReduceTask& t = *lv[i];
+                Object* out = nullptr;
+                int rc = ensure_partial_buffer(c, op, t.pos, &out);
+                if (rc != HPL_OK) return rc;
+                ReduceTask& d = w.tasks[w.n_tasks++];
+                d.out_ptr = (unsigned long long)(uintptr_t)out->ptr;
+                d.elems = op.elems;
+                d.chunk_elems = op.chunk_elems;
+                d.c_begin = t.a;
+                d.c_end = t.b;
+                d.tiles_per_chunk = tpc_full;
+                d.tile_begin = w.total_tiles;
+                d.step_begin = n_steps;
+                d.n_steps = (uint32_t)t.steps.size();
+                d.red_op = (uint32_t)op.red_op;
+                d.poll = t.poll ? 1u : 0u;
+                d.pad = 0;
+                std::memcpy(&w.steps[n_steps], t.steps.data(), t.steps.size() * sizeof(ReduceStep));
+                n_steps += d.n_steps;
+                w.total_tiles += (t.b - t.a) * tpc_full;
+                n_acc = std::max(n_acc, t.n_acc);
+                // accounting: bytes the task moves
+                uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
+                for (auto& st : t.steps)
+                    if (st.code != OPC_ADD_ACC) c->stats.bytes_read_planned += (e_hi - e_lo) * (st.kind == SRC_BF16 ? 2 : 4);
+                c->stats.bytes_written_planned += (e_hi - e_lo) * 4;
+                c->stats.reduce_tasks++;
+                ++i;
+            }
+            if (w.n_tasks == 0) return HPL_ERR_INVALID;  // a single task larger than a wave: tree too wide
+            int& occ = c->occ_reduce[bf16 ? 1 : 0][occ_index(n_acc)];
+            if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16);
+            int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
+            if (grid < 1) grid = 1;
+            if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
+            c->stats.kernel_launches++;
+            c->stats.tiles += w.total_tiles;
+            c->stats.last_kernel_grid = (uint64_t)grid;
+            c->work_in_flight = true;
+        }
+    }
+    return HPL_OK;
+}
+
+// ------------------------------------------------------------------------------------------ broadcast planner
+struct PlannedFanout {
+    int loc;  // location index read from
+    uint32_t a, b;
+    bool poll;
+    std::vector<int> dst;  // location indices written
+};
+
+int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+    BroadcastTreeSchedule& s = *op.sched;
+    const auto& locs = s.locations();
+    op.phys_have.resize(locs.size(), 0);
+    Object* src = find(c, op.src);
+    if (!src) return HPL_OK;
+    const uint32_t C = src->C;
+    uint32_t src_landed = 0, src_avail = 0;
+    if (src->alive && src->ptr && src->row >= 0) {
+        src_landed = std::min(published_chunks(c, *src), src->landed);
+        src_avail = c->cfg.plan_ahead ? C : src_landed;
+    }
+    std::vector<int64_t> pre(op.phys_have);  // what every copy holds before this pass
+    pre[0] = src_avail;
+    auto usable = [&](int x) {
+        if (x == 0) return src->alive && src->ptr != nullptr;
+        Object* o = find(c, locs[x].obj);
+        return locs[x].alive && o && o->alive && o->ptr && o->row >= 0;
+    };
+    std::vector<uint32_t> bp = {0u, src_avail};
+    for (size_t i = 1; i < locs.size(); ++i) bp.push_back((uint32_t)pre[i]);
+    std::sort(bp.begin(), bp.end());
+    bp.erase(std::unique(bp.begin(), bp.end()), bp.end());
+
+    std::vector<char> stuck(locs.size(), 0);
+    for (size_t bi = 0; bi + 1 < bp.size(); ++bi) {
+        const uint32_t a = bp[bi], b = bp[bi + 1];
+        std::map<int, std::vector<int>> groups;  // read location -> receivers
+        for (int r = 1; r < (int)locs.size(); ++r) {
+            if (stuck[r] || !usable(r) || locs[r].last_sender < 0) continue;
+            if (op.phys_have[r] != (int64_t)a) continue;  // needs this interval next
+            int loc = -1;
+            for (int x = locs[r].last_sender, hops = 0; x >= 0 && hops <= (int)locs.size(); x = locs[x].last_sender, ++hops) {
+                if (usable(x) && pre[x] >= (int64_t)b) {
+                    loc = x;
+                    break;
+                }
+                if (x == 0) break;
+            }
+            if (loc < 0) {
+                for (int x = 0; x < (int)locs.size(); ++x)
+                    if (x != r && usable(x) && pre[x] >= (int64_t)b) {
+                        loc = x;
+                        break;
+                    }
+            }
+            if (loc < 0) {
+                stuck[r] = 1;
+                continue;
+            }
+            groups[loc].push_back(r);
+            c->journal.b.push_back({op.src, r, op.phys_have[r]});
+            op.phys_have[r] = b;
+        }
+        for (auto& g : groups) {
+            const bool poll = (g.first == 0) && (src_landed < b);
+            bool merged = false;
+            for (auto& prev : tasks) {
+                if (prev.loc == g.first && prev.b == a && prev.poll == poll && prev.dst == g.second) {
+                    prev.b = b;
+                    merged = true;
+                    break;
+                }
+            }
+            if (!merged) tasks.push_back(PlannedFanout{g.first, a, b, poll, g.second});
+        }
+    }
+    return HPL_OK;
+}
+
+int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+    if (tasks.empty()) return HPL_OK;
+    Object* src = find(c, op.src);
+    const auto& locs = op.sched->locations();
+    const uint64_t chunk_bytes = c->cfg.chunk_bytes;
+    const uint32_t tpc = (uint32_t)((std::min<uint64_t>(chunk_bytes, src->bytes) + kFanoutTileBytes - 1) / kFanoutTileBytes);
+    size_t i = 0;
+    while (i < tasks.size()) {
+        static thread_local FanoutWave w;
+        w.dir = c->d_dir;
+        w.status = c->d_status;
+        w.budget_ns = c->cfg.poll_budget_ns;
+        w.n_tasks = 0;
+        w.total_tiles = 0;
+        uint32_t n_dst = 0;
+        while (i < tasks.size() && w.n_tasks < (uint32_t)kMaxFanoutTasks) {
+            PlannedFanout& t = tasks[i];
+            if (t.dst.size() > (size_t)kMaxFanoutDst) {
+                // more receivers than one task holds: split the receiver list
+                PlannedFanout rest = t;
+                rest.dst.assign(t.dst.begin() + kMaxFanoutDst, t.dst.end());
+                t.dst.resize(kMaxFanoutDst);
+                tasks.insert(tasks.begin() + i + 1, rest);
+                continue;
+            }
+            if (n_dst + tasks[i].dst.size() > (size_t)kMaxFanoutDst) break;
+            PlannedFanout& tt = tasks[i];
+            FanoutTask& d = w.tasks[w.n_tasks++];
+            Object* lo = tt.loc == 0 ? src : find(c, locs[tt.loc].obj);
+            d.src_row = (uint32_t)lo->row;
+            d.c_begin = tt.a;
+            d.c_end = tt.b;
+            d.tiles_per_chunk = tpc;
+            d.tile_begin = w.total_tiles;
+            d.dst_begin = n_dst;
+            d.n_dst = (uint32_t)tt.dst.size();
+            d.poll = tt.poll ? 1u : 0u;
+            d.bytes = src->bytes;
+            d.chunk_bytes = chunk_bytes;
+            for (int r : tt.dst) w.dst_rows[n_dst++] = (uint32_t)find(c, locs[r].obj)->row;
+            w.total_tiles += (tt.b - tt.a) * tpc;
+            const uint64_t b_lo = (uint64_t)tt.a * chunk_bytes, b_hi = std::min<uint64_t>((uint64_t)tt.b * chunk_bytes, src->bytes);
+            c->stats.bytes_read_planned += b_hi - b_lo;
+            c->stats.bytes_written_planned += (b_hi - b_lo) * tt.dst.size();
+            c->stats.fanout_tasks++;
+            ++i;
+        }
+        if (w.n_tasks == 0) return HPL_ERR_INVALID;
+        if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
+        int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
+        if (grid < 1) grid = 1;
+        if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
+        c->stats.kernel_launches++;
+        c->stats.tiles += w.total_tiles;
+        c->stats.last_kernel_grid = (uint64_t)grid;
+        c->work_in_flight = true;
+    }
+    return HPL_OK;
+}
+
+// ------------------------------------------------------------------------------------------ progress / sync
+int progress(hpl_ctx* c) {
+    if (!c->device) return HPL_OK;
+    if (c->copy_pending && !c->cfg.plan_ahead) {
+        // host objects: their chunks become usable once the main stream is ordered after the copies
+        CUDA_TRY(cudaEventRecord(c->copy_ev, c->copy_stream));
+        CUDA_TRY(cudaStreamWaitEvent(c->stream, c->copy_ev, 0));
+        c->copy_pending = false;
+        for (auto& kv : c->objects)
+            if (kv.second.from_host) kv.second.landed = published_chunks(c, kv.second);
+    }
+    for (auto& kv : c->bcasts) {
+        std::vector<PlannedFanout> tasks;
+        int rc = plan_bcast(c, kv.second, tasks);
+        if (rc != HPL_OK) return rc;
+        rc = launch_fanout_tasks(c, kv.second, tasks);
+        if (rc != HPL_OK) return rc;
+    }
+    for (auto& kv : c->reduces) {
+        std::vector<PlannedReduceTask> tasks;
+        int rc = plan_reduce(c, kv.second, tasks);
+        if (rc != HPL_OK) return rc;
+        rc = launch_reduce_tasks(c, kv.second, tasks);
+        if (rc != HPL_OK) return rc;
+    }
+    return HPL_OK;
+}
+
+void undo_journal(hpl_ctx* c) {
+    for (auto& e : c->journal.r) {
+        auto it = c->reduce_of_target.find(e.target);
+        if (it == c->reduce_of_target.end()) continue;
+        ReduceOp& op = c->reduces.at(it->second);
+        if (e.pos < (int)op.computed.size()) op.computed[e.pos].remove(e.a, e.b);
+    }
+    for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
+        auto f = c->bcast_of_src.find(it->src);
+        if (f == c->bcast_of_src.end()) continue;
+        BcastOp& op = c->bcasts.at(f->second);
+        if (it->loc < (int)op.phys_have.size()) op.phys_have[it->loc] = it->old_have;
+    }
+    c->journal.clear();
+}
+
+int sync_and_check(hpl_ctx* c) {
+    if (!c->device) return HPL_OK;
+    if (c->copy_pending) {
+        CUDA_TRY(cudaStreamSynchronize(c->copy_stream));
+        c->copy_pending = false;
+        for (auto& kv : c->objects)
+            if (kv.second.from_host) kv.second.landed = published_chunks(c, kv.second);
+    }
+    if (!c->work_in_flight) {
+        CUDA_TRY(cudaStreamSynchronize(c->stream));
+        c->journal.clear();
+        return HPL_OK;
+    }
+    CUDA_TRY(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->work_in_flight = false;
+    if (c->h_status->error) {
+        c->stats.device_timeouts++;
+        undo_journal(c);
+        CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus), c->stream));
+        CUDA_TRY(cudaStreamSynchronize(c->stream));
+        return HPL_ERR_TIMEOUT;
+    }
+    c->journal.clear();
+    return HPL_OK;
+}
+
+int after_event(hpl_ctx* c) { return c->cfg.eager ? progress(c) : HPL_OK; }
+
+int64_t delivered_of(hpl_ctx* c, int64_t oid) {
+    Object* o = find(c, oid);
+    return o ? (int64_t)published_chunks(c, *o) : 0;
+}
+
+void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv) {
+    const int k = op.sched->k();
+    if (inv.shrank) {
+        op.computed.resize(k);
+        op.partial_key.resize(k, 0);
+    }
+    for (int p : inv.positions)
+        if (p >= 0 && p < k) op.computed[p].clear();
+}
+
+void notify_arrival(hpl_ctx* c, Object& o) {
+    for (auto& kv : c->reduces)
+        if (kv.second.sched->has_source(o.id)) kv.second.sched->arrive(o.id);
+}
+
+int do_put_common(hpl_ctx* c, Object& o, uint64_t bytes, bool first) {
+    o.ready_bytes = bytes;
+    if (first) {
+        o.arrived = true;
+        o.t_arrival = (int64_t)c->now;
+        notify_arrival(c, o);
+    }
+    auto b = c->bcast_of_src.find(o.id);
+    if (b != c->bcast_of_src.end()) c->bcasts.at(b->second).sched->source_progress((int64_t)c->now, published_chunks(c, o));
+    return HPL_OK;
+}
+
+}  // namespace
+
+// ================================================================================================ C ABI
+extern "C" {
+
+const char* hpl_strerror(int code) {
+    switch (code) {
+        case HPL_OK: return "ok";
+        case HPL_ERR_INVALID: return "invalid argument";
+        case HPL_ERR_NOT_FOUND: return "unknown object";
+        case HPL_ERR_EXISTS: return "object id already exists";
+        case HPL_ERR_TIMEOUT: return "not complete (bounded wait expired or inputs missing)";
+        case HPL_ERR_INSUFFICIENT: return "no live source left";
+        case HPL_ERR_FAILED_WORKER: return "owned by a failed worker";
+        case HPL_ERR_CUDA: return "CUDA error or no device";
+        case HPL_ERR_NOMEM: return "arena exhausted";
+        default: return "unknown error";
+    }
+}
+
+int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
+    if (!cfg || !out) return HPL_ERR_INVALID;
+    if (cfg->chunk_bytes == 0 || cfg->chunk_bytes % 16 || cfg->reduce_degree < 1 || cfg->bcast_degree < 1) return HPL_ERR_INVALID;
+    hpl_ctx* c = new (std::nothrow) hpl_ctx();
+    if (!c) return HPL_ERR_NOMEM;
+    c->cfg = *cfg;
+    if (c->cfg.poll_budget_ns == 0) c->cfg.poll_budget_ns = 2000000000ull;
+    c->tau = cfg->virt_chunk_ns ? cfg->virt_chunk_ns : std::max<uint64_t>(1, cfg->chunk_bytes * 1000000000ull / (64ull << 30));
+    c->stream = (cudaStream_t)cuda_stream;
+    if (cfg->arena) {
+        const uint64_t need = sizeof(DirRow) * kMaxRows + sizeof(DeviceStatus) + 2 * kAlign;
+        if (cfg->arena_bytes < need) {
+            delete c;
+            return HPL_ERR_NOMEM;
+        }
+        int dev = 0;
+        cudaDeviceProp prop;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+            delete c;
+            return HPL_ERR_CUDA;
+        }
+        c->n_sm = prop.multiProcessorCount;
+        c->arena.init(cfg->arena, cfg->arena_bytes);
+        c->d_dir = (DirRow*)c->arena.alloc(sizeof(DirRow) * kMaxRows);
+        c->d_status = (DeviceStatus*)c->arena.alloc(sizeof(DeviceStatus));
+        bool ok = c->d_dir && c->d_status;
+        ok = ok && cudaHostAlloc((void**)&c->h_dir, sizeof(DirRow) * kMaxRows, cudaHostAllocDefault) == cudaSuccess;
+        ok = ok && cudaHostAlloc((void**)&c->h_status, sizeof(DeviceStatus), cudaHostAllocDefault) == cudaSuccess;
+        ok = ok && cudaHostAlloc((void**)&c->h_iota, sizeof(uint32_t) * (kMaxChunks + 1), cudaHostAllocDefault) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->copy_ev, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaMemsetAsync(c->d_dir, 0, sizeof(DirRow) * kMaxRows, c->stream) == cudaSuccess;
+        ok = ok && cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus), c->stream) == cudaSuccess;
+        if (!ok) {
+            if (c->h_dir) cudaFreeHost(c->h_dir);
+            if (c->h_status) cudaFreeHost(c->h_status);
+            if (c->h_iota) cudaFreeHost(c->h_iota);
+            if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+            if (c->copy_ev) cudaEventDestroy(c->copy_ev);
+            delete c;
+            return HPL_ERR_CUDA;
+        }
+        for (uint32_t i = 0; i <= kMaxChunks; ++i) c->h_iota[i] = i;
+        for (int r = (int)kMaxRows - 1; r >= 0; --r) c->free_rows.push_back(r);
+        c->device = true;
+    }
+    *out = c;
+    return HPL_OK;
+}
+
+int hpl_shutdown(hpl_ctx* c) {
+    if (!c) return HPL_ERR_INVALID;
+    if (c->device) {
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamSynchronize(c->stream);
+        cudaFreeHost(c->h_dir);
+        cudaFreeHost(c->h_status);
+        cudaFreeHost(c->h_iota);
+        cudaStreamDestroy(c->copy_stream);
+        cudaEventDestroy(c->copy_ev);
+    }
+    delete c;
+    return HPL_OK;
+}
+
+int hpl_advance(hpl_ctx* c, uint64_t t_ns) {
+    if (!c || t_ns < c->now) return HPL_ERR_INVALID;
+    c->now = t_ns;
+    for (auto& kv : c->bcasts) kv.second.sched->advance((int64_t)t_ns);
+    return HPL_OK;
+}
+
+int hpl_create(hpl_ctx* c, int64_t id, int32_t worker, uint64_t total_bytes, int32_t dtype) {
+    if (!c || id < 0 || worker < 0 || (dtype != HPL_F32 && dtype != HPL_BF16)) return HPL_ERR_INVALID;
+    if (total_bytes == 0 || total_bytes % elem_size(dtype)) return HPL_ERR_INVALID;
+    if (c->objects.count(id)) return HPL_ERR_EXISTS;
+    const uint64_t C = (total_bytes + c->cfg.chunk_bytes - 1) / c->cfg.chunk_bytes;
+    if (C > kMaxChunks) return HPL_ERR_INVALID;
+    Object o;
+    o.id = id;
+    o.worker = worker;
+    o.bytes = total_bytes;
+    o.dtype = dtype;
+    o.C = (uint32_t)C;
+    o.seq = c->seq++;
+    c->objects.emplace(id, o);
+    return HPL_OK;
+}
+
+static int put_checks(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes, Object** out) {
+    if (!c || !buf) return HPL_ERR_INVALID;
+    Object* o = find(c, id);
+    if (!o) return HPL_ERR_NOT_FOUND;
+    if (!o->alive) return HPL_ERR_FAILED_WORKER;
+    if (o->kind != OBJ_PLAIN) return HPL_ERR_INVALID;
+    if (bytes < o->ready_bytes || bytes > o->bytes) return HPL_ERR_INVALID;
+    *out = o;
+    return HPL_OK;
+}
+
+int hpl_put(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
+    Object* o = nullptr;
+    int rc = put_checks(c, id, buf, bytes, &o);
+    if (rc != HPL_OK) return rc;
+    if ((uintptr_t)buf % 16) return HPL_ERR_INVALID;
+    const bool first = !o->arrived;
+    if (!first && (o->ptr != buf || o->from_host)) return HPL_ERR_INVALID;
+    if (first) {
+        o->ptr = const_cast<void*>(buf);
+        rc = alloc_row(c, *o);
+        if (rc != HPL_OK) {
+            o->ptr = nullptr;
+            return rc;
+        }
+    }
+    const uint32_t before = published_chunks(c, *o);
+    do_put_common(c, *o, bytes, first);
+    const uint32_t after = published_chunks(c, *o);
+    if (after != before || first) {
+        rc = publish_counter(c, *o, after, c->stream);
+        if (rc != HPL_OK) return rc;
+    }
+    o->landed = after;
+    return after_event(c);
+}
+
+int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
+    Object* o = nullptr;
+    int rc = put_checks(c, id, buf, bytes, &o);
+    if (rc != HPL_OK) return rc;
+    if (!c->device) return HPL_ERR_CUDA;
+    const bool first = !o->arrived;
+    if (!first && !o->from_host) return HPL_ERR_INVALID;
+    if (first) {
+        o->ptr = c->arena.alloc(o->bytes);
+        if (!o->ptr) return HPL_ERR_NOMEM;
+        o->lib_owned = true;
+        o->from_host = true;
+        rc = alloc_row(c, *o);
+        if (rc != HPL_OK) {
+            c->arena.release(o->ptr);
+            o->ptr = nullptr;
+            o->lib_owned = false;
+            return rc;
+        }
+        // the row (pointer) must be in the directory before any copy-stream counter update can matter
+        CUDA_TRY(cudaEventRecord(c->copy_ev, c->stream));
+        CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
+    }
+    const uint64_t old_bytes = o->ready_bytes;
+    const uint64_t chunk = c->cfg.chunk_bytes;
+    // copy [old_bytes, bytes) in pieces that end on chunk boundaries, publishing each completed chunk
+    uint64_t off = old_bytes;
+    while (off < bytes) {
+        uint64_t end = std::min<uint64_t>((off / chunk + 1) * chunk, bytes);
+        CUDA_TRY(cudaMemcpyAsync((uint8_t*)o->ptr + off, (const uint8_t*)buf + off, end - off, cudaMemcpyHostToDevice, c->copy_stream));
+        c->stats.h2d_bytes += end - off;
+        uint32_t done = end >= o->bytes ? o->C : (uint32_t)(end / chunk);
+        if (end % chunk == 0 || end >= o->bytes) {
+            rc = publish_counter(c, *o, done, c->copy_stream);
+            if (rc != HPL_OK) return rc;
+        }
+        off = end;
+    }
+    c->copy_pending = true;
+    do_put_common(c, *o, bytes, first);
+    return after_event(c);
+}
+
+int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, int32_t k, int32_t op, int32_t dtype) {
+    if (!c || !src_ids || n < 1 || k < 1 || k > n || target < 0) return HPL_ERR_INVALID;
+    if (op < HPL_SUM || op > HPL_MAX || (dtype != HPL_F32 && dtype != HPL_BF16)) return HPL_ERR_INVALID;
+    if (c->objects.count(target)) return HPL_ERR_EXISTS;
+    std::vector<int64_t> srcs(src_ids, src_ids + n);
+    {
+        std::vector<int64_t> u = srcs;
+        std::sort(u.begin(), u.end());
+        if (std::adjacent_find(u.begin(), u.end()) != u.end()) return HPL_ERR_INVALID;
+    }
+    uint64_t bytes = 0;
+    int live = 0;
+    for (int64_t s : srcs) {
+        Object* o = find(c, s);
+        if (!o) return HPL_ERR_NOT_FOUND;
+        if (o->dtype != dtype || (bytes && o->bytes != bytes)) return HPL_ERR_INVALID;
+        bytes = o->bytes;
+        if (o->alive) ++live;
+    }
+    if (live < 1) return HPL_ERR_INSUFFICIENT;
+    const uint64_t elems = bytes / elem_size(dtype);
+
+    Object t;
+    t.id = target;
+    t.worker = -1;
+    t.bytes = elems * 4;
+    t.dtype = HPL_F32;
+    t.C = find(c, srcs[0])->C;
+    t.kind = OBJ_TARGET;
+    t.lib_owned = true;
+    t.seq = c->seq++;
+    if (c->device) {
+        t.ptr = c->arena.alloc(t.bytes);
+        if (!t.ptr) return HPL_ERR_NOMEM;
+        int rc = alloc_row(c, t);
+        if (rc != HPL_OK) {
+            c->arena.release(t.ptr);
+            return rc;
+        }
+    }
+    c->objects.emplace(target, t);
+
+    ReduceOp r;
+    r.target = target;
+    r.sched.reset(new ReduceTreeSchedule(srcs, k, c->cfg.reduce_degree));
+    r.red_op = op;
+    r.in_dtype = dtype;
+    r.elems = elems;
+    r.C = t.C;
+    r.chunk_elems = (uint32_t)(std::min<uint64_t>(c->cfg.chunk_bytes, bytes) / elem_size(dtype));
+    if (r.chunk_elems == 0) r.chunk_elems = 1;
+    r.seq = c->seq++;
+    auto dl = [c](int64_t o) { return delivered_of(c, o); };
+    for (int64_t s : srcs)
+        if (!find(c, s)->alive) r.sched->fail(s, 0, dl);  // sources lost before the call never take part
+    std::vector<std::pair<std::pair<int64_t, int>, int64_t>> arrived;
+    for (int i = 0; i < n; ++i) {
+        Object* o = find(c, srcs[i]);
+        if (o->alive && o->arrived) arrived.push_back({{o->t_arrival, i}, o->id});
+    }
+    std::sort(arrived.begin(), arrived.end());
+    for (auto& a : arrived) r.sched->arrive(a.second);
+    r.computed.assign(r.sched->k(), IntervalSet());
+    r.partial_key.assign(r.sched->k(), 0);
+    const uint64_t key = r.seq;
+    c->reduce_of_target[target] = key;
+    c->reduces.emplace(key, std::move(r));
+    return after_event(c);
+}
+
+int hpl_broadcast(hpl_ctx* c, int64_t src_id, const int64_t* dst_ids, int32_t n) {
+    if (!c || !dst_ids || n < 1) return HPL_ERR_INVALID;
+    Object* src = find(c, src_id);
+    if (!src) return HPL_ERR_NOT_FOUND;
+    if (c->bcast_of_src.count(src_id)) return HPL_ERR_EXISTS;
+    for (int i = 0; i < n; ++i) {
+        Object* d = find(c, dst_ids[i]);
+        if (!d) return HPL_ERR_NOT_FOUND;
+        if (d->bytes != src->bytes || d->dtype != src->dtype || d->kind != OBJ_PLAIN || d->arrived) return HPL_ERR_INVALID;
+        for (int j = 0; j < i; ++j)
+            if (dst_ids[j] == dst_ids[i]) return HPL_ERR_INVALID;
+    }
+    if (!src->alive) return HPL_ERR_FAILED_WORKER;
+    BcastOp b;
+    b.src = src_id;
+    b.sched.reset(new BroadcastTreeSchedule(src_id, src->C, c->cfg.bcast_degree, (int64_t)c->tau));
+    b.sched->advance((int64_t)c->now);
+    if (src->arrived) b.sched->source_progress((int64_t)c->now, published_chunks(c, *src));
+    b.dsts.assign(dst_ids, dst_ids + n);
+    b.seq = c->seq++;
+    for (int i = 0; i < n; ++i) {
+        Object* d = find(c, dst_ids[i]);
+        d->kind = OBJ_RECEIVER;
+        d->op_key = src_id;
+    }
+    c->bcast_of_src[src_id] = b.seq;
+    const uint64_t key = b.seq;
+    c->bcasts.emplace(key, std::move(b));
+    return after_event(c);
+}
+
+int hpl_join(hpl_ctx* c, int64_t dst_id, void* dst_buf) {
+    if (!c) return HPL_ERR_INVALID;
+    Object* d = find(c, dst_id);
+    if (!d) return HPL_ERR_NOT_FOUND;
+    if (d->kind != OBJ_RECEIVER) return HPL_ERR_NOT_FOUND;
+    if (!d->alive) return HPL_ERR_FAILED_WORKER;
+    if (c->device && (!dst_buf || (uintptr_t)dst_buf % 16)) return HPL_ERR_INVALID;
+    BcastOp& b = c->bcasts.at(c->bcast_of_src.at(d->op_key));
+    if (b.sched->index_of(dst_id) < 0) {
+        d->ptr = dst_buf;
+        d->ready_bytes = 0;
+        int rc = alloc_row(c, *d);
+        if (rc != HPL_OK) return rc;
+    }
+    b.sched->join((int64_t)c->now, dst_id);
+    return after_event(c);
+}
+
+int hpl_fail(hpl_ctx* c, int32_t worker) {
+    if (!c || worker < 0) return HPL_ERR_INVALID;
+    std::vector<Object*> lost;
+    for (auto& kv : c->objects)
+        if (kv.second.worker == worker && kv.second.alive) lost.push_back(&kv.second);
+    std::sort(lost.begin(), lost.end(), [](Object* a, Object* b) { return a->seq < b->seq; });
+    for (Object* o : lost) o->alive = false;
+    auto dl = [c](int64_t o) { return delivered_of(c, o); };
+    for (auto& kv : c->reduces) {
+        ReduceOp& op = kv.second;
+        for (Object* o : lost) {
+            if (!op.sched->has_source(o->id)) continue;
+            ReduceInvalidation inv = op.sched->fail(o->id, (int64_t)published_chunks(c, *o), dl);
+            apply_invalidation(op, inv);
+        }
+    }
+    for (auto& kv : c->bcasts) {
+        BcastOp& op = kv.second;
+        std::vector<int64_t> mine;
+        for (Object* o : lost)
+            if (o->id == op.src || (o->kind == OBJ_RECEIVER && o->op_key == op.src)) mine.push_back(o->id);
+        if (!mine.empty()) op.sched->fail((int64_t)c->now, mine);
+    }
+    return after_event(c);
+}
+
+int hpl_progress(hpl_ctx* c) {
+    if (!c) return HPL_ERR_INVALID;
+    return progress(c);
+}
+
+int hpl_sync(hpl_ctx* c) {
+    if (!c) return HPL_ERR_INVALID;
+    return sync_and_check(c);
+}
+
+int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
+    if (!c) return HPL_ERR_INVALID;
+    Object* o = find(c, id);
+    if (!o) return HPL_ERR_NOT_FOUND;
+    if (o->kind == OBJ_TARGET) {
+        ReduceOp& op = c->reduces.at(c->reduce_of_target.at(id));
+        if (op.sched->k() == 0) return HPL_ERR_INSUFFICIENT;
+        int rc = progress(c);   // whatever can run now runs, even if the target cannot complete yet
+        if (rc != HPL_OK) return rc;
+        if (!op.sched->full()) return HPL_ERR_TIMEOUT;
+        for (int p = 0; p < op.sched->k(); ++p) {
+            Object* m = find(c, op.sched->object_at(p));
+            if (!m || m->ready_bytes < m->bytes) return HPL_ERR_TIMEOUT;
+        }
+        if (!c->device) return HPL_ERR_CUDA;
+        if (!op.computed[0].contains(0, op.C)) return HPL_ERR_TIMEOUT;
+        rc = sync_and_check(c);
+        if (rc != HPL_OK) return rc;
+    } else if (o->kind == OBJ_RECEIVER) {
+        if (!o->alive) return HPL_ERR_FAILED_WORKER;
+        BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
+        const int li = op.sched->index_of(id);
+        if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
+        if (!op.sched->run_until_complete(id)) return HPL_ERR_TIMEOUT;
+        if ((uint64_t)op.sched->now() > c->now) c->now = (uint64_t)op.sched->now();
+        for (auto& kv : c->bcasts) kv.second.sched->advance((int64_t)c->now);
+        if (!c->device) return HPL_ERR_CUDA;
+        int rc = progress(c);
+        if (rc != HPL_OK) return rc;
+        if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) return HPL_ERR_TIMEOUT;
+        rc = sync_and_check(c);
+        if (rc != HPL_OK) return rc;
+    } else {
+        if (!o->alive) return HPL_ERR_FAILED_WORKER;
+        if (!o->arrived || o->ready_bytes < o->bytes) return HPL_ERR_TIMEOUT;
+        if (!c->device) return HPL_ERR_CUDA;
+        int rc = sync_and_check(c);
+        if (rc != HPL_OK) return rc;
+    }
+    if (dev_ptr) *dev_ptr = o->ptr;
+    if (bytes) *bytes = o->bytes;
+    return HPL_OK;
+}
+
+int hpl_get_host(hpl_ctx* c, int64_t id, void* dst, uint64_t cap) {
+    if (!c || !dst) return HPL_ERR_INVALID;
+    const void* p = nullptr;
+    uint64_t n = 0;
+    int rc = hpl_get(c, id, &p, &n);
+    if (rc != HPL_OK) return rc;
+    if (cap < n) return HPL_ERR_INVALID;
+    CUDA_TRY(cudaMemcpyAsync(dst, p, n, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->stats.d2h_bytes += n;
+    return HPL_OK;
+}
+
+int hpl_delete(hpl_ctx* c, int64_t id) {
+    if (!c) return HPL_ERR_INVALID;
+    Object* o = find(c, id);
+    if (!o || id < 0) return HPL_ERR_NOT_FOUND;
+    if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
+    for (auto& kv : c->reduces)
+        if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
+    if (c->device) {
+        // rows and arena memory are recycled only when nothing enqueued can still read them
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamSynchronize(c->stream);
+    }
+    if (o->kind == OBJ_TARGET) {
+        const uint64_t key = c->reduce_of_target.at(id);
+        ReduceOp& op = c->reduces.at(key);
+        for (int64_t pk : op.partial_key)
+            if (pk != 0) {
+                Object* po = find(c, pk);
+                if (po) {
+                    release_object_memory(c, *po);
+                    c->objects.erase(pk);
+                }
+            }
+        c->reduces.erase(key);
+        c->reduce_of_target.erase(id);
+    }
+    auto b = c->bcast_of_src.find(id);
+    if (b != c->bcast_of_src.end()) {
+        BcastOp& op = c->bcasts.at(b->second);
+        for (int64_t d : op.dsts) {
+            Object* r = find(c, d);
+            if (r) {
+                release_object_memory(c, *r);
+                c->objects.erase(d);
+            }
+        }
+        c->bcasts.erase(b->second);
+        c->bcast_of_src.erase(b);
+    }
+    o = find(c, id);
+    release_object_memory(c, *o);
+    c->objects.erase(id);
+    return HPL_OK;
+}
+
+int hpl_schedule_dump(hpl_ctx* c, int64_t op_id, int64_t* words, uint64_t cap, uint64_t* len) {
+    if (!c || !len) return HPL_ERR_INVALID;
+    std::vector<int64_t> w;
+    auto r = c->reduce_of_target.find(op_id);
+    auto b = c->bcast_of_src.find(op_id);
+    if (r != c->reduce_of_target.end())
+        c->reduces.at(r->second).sched->dump(op_id, w);
+    else if (b != c->bcast_of_src.end())
+        c->bcasts.at(b->second).sched->dump(w);
+    else
+        return HPL_ERR_NOT_FOUND;
+    *len = w.size();
+    if (!words || cap < w.size()) return HPL_ERR_INVALID;
+    std::memcpy(words, w.data(), w.size() * sizeof(int64_t));
+    return HPL_OK;
+}
+
+int hpl_stats(hpl_ctx* c, hpl_stats_t* out) {
+    if (!c || !out) return HPL_ERR_INVALID;
+    c->stats.arena_used = c->arena.used;
+    *out = c->stats;
+    return HPL_OK;
+}
+
+}  // extern "C"

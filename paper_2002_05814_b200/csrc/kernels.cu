@@ -1,0 +1,388 @@
+// sm_100a kernels of the reduce / broadcast hot path.
+//
+//  reduce_wave_kernel  -- persistent grid over the tiles of a wave of subtree tasks.  A task is a
+//      fused evaluation of a subtree of the reduce tree (arXiv 2002.05814, Section 3.4.2) over a
+//      range of chunks: a short program of LOAD / ADD_LOAD / ADD_ACC steps, executed per tile with
+//      the accumulators in registers, in exactly the association order of the tree, fp32, no
+//      contraction, no fast-math.  Before a chunk is touched the progress counters of its operands
+//      are polled in the device directory (bounded wait), which is how a chunk that is still being
+//      copied into the store is consumed as soon as it lands (Section 3.3).
+//  fanout_wave_kernel  -- reads each tile of a chunk once and stores it to every receiver of the
+//      task (Section 3.4.1: the receivers of one sender subtree), same polling.
+//
+// Global reads are 16 bytes per thread, coalesced and L2-only (.cg) because every byte is used once.
+// The reduce kernel stages its operand tiles through shared memory with cp.async, three steps ahead
+// of the adds, so that about 48 KiB per CTA are in flight without holding registers.
+#include <cuda_runtime.h>
+
+#include "device_types.h"
+
+namespace hpl {
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ unsigned int load_acquire_sys(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Waits until dir[row].ready_chunks > chunk.  Bounded twice: by the wave's time budget measured from
+// the kernel's start and by an iteration cap.  On expiry records the wait in *status and returns false.
+__device__ bool wait_chunk(const DirRow* dir, DeviceStatus* status, unsigned int row, unsigned int chunk,
+                           unsigned long long t_start, unsigned long long budget_ns) {
+    const unsigned int* flag = &dir[row].ready_chunks;
+    if (load_acquire_sys(flag) > chunk) return true;
+    atomicAdd(&status->waits, 1ull);
+    const unsigned long long max_iter = budget_ns / 128ull + 1024ull;
+    for (unsigned long long it = 0; it < max_iter; ++it) {
+        __nanosleep(200);
+        if (load_acquire_sys(flag) > chunk) return true;
+        if (*reinterpret_cast<volatile unsigned int*>(&status->abort)) return false;
+        if (global_timer_ns() - t_start > budget_ns) break;
+    }
+    if (atomicCAS(&status->error, 0u, 1u) == 0u) {
+        status->row = row;
+        status->chunk = chunk;
+    }
+    __threadfence();
+    *reinterpret_cast<volatile unsigned int*>(&status->abort) = 1u;
+    return false;
+}
+
+__device__ __forceinline__ float combine(float a, float b, unsigned int red_op) {
+    if (red_op == 0) return __fadd_rn(a, b);
+    if (red_op == 1) return (b < a) ? b : a;
+    return (a < b) ? b : a;
+}
+
+// ---- staging.  Every load step of a task is brought from global memory to shared memory with
+// cp.async (16 bytes per instruction, L2 only), kStages steps ahead of its use.  A thread only ever
+// reads back the bytes it copied itself, so no barrier is needed: cp.async.wait_group orders them.
+// Shared layout: [stage][vector j][thread] of 16-byte vectors (conflict free).
+//   F32 task:  vector j (of 4) of thread t holds elements (j*256 + t)*4 .. +3 of the tile.
+//   BF16 task: group j (of 2) of thread t holds elements (j*256 + t)*8 .. +7: one vector for a bf16
+//              operand, two (slots 2j, 2j+1) for an fp32 operand (a materialised partial result).
+constexpr int kStages = 4;
+constexpr int kStageBytes = 4 * kReduceThreads * 16;
+constexpr int kReduceSmemBytes = kStages * kStageBytes;
+
+__device__ __forceinline__ void cp_async16(unsigned int smem_addr, const void* gptr, unsigned int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <bool BF16>
+struct TileCtx {
+    const ReduceStep* steps;
+    const unsigned long long* s_ptr;   // operand base addresses of the task's steps (shared memory)
+    unsigned int smem_base;            // shared-window address of the staging area
+    unsigned int n, pc, red_op, t;
+    unsigned long long e0;             // first element of the tile
+    unsigned int count;                // elements in the tile
+
+    // bytes of a 16-byte vector starting at element `off` of the tile that lie inside it
+    __device__ __forceinline__ unsigned int in_bounds_bytes(unsigned int off, unsigned int elem_bytes, unsigned int per_vec) const {
+        if (off >= count) return 0u;
+        const unsigned int left = count - off;
+        return (left >= per_vec ? per_vec : left) * elem_bytes;
+    }
+
+    __device__ __forceinline__ void issue(unsigned int i) {
+        if (i < n) {
+            const ReduceStep st = steps[i];
+            if (st.code != OPC_ADD_ACC) {
+                const unsigned int stage = smem_base + (i % kStages) * kStageBytes;
+                const unsigned long long base = s_ptr[i];
+                if (!BF16) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned int off = (j * kReduceThreads + t) * 4;
+                        const unsigned int nb = in_bounds_bytes(off, 4, 4);
+                        const float* g = reinterpret_cast<const float*>(base) + (nb ? e0 + off : 0ull);
+                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
+                    }
+                } else if (st.kind == SRC_BF16) {
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const unsigned int off = (j * kReduceThreads + t) * 8;
+                        const unsigned int nb = in_bounds_bytes(off, 2, 8);
+                        const unsigned short* g = reinterpret_cast<const unsigned short*>(base) + (nb ? e0 + off : 0ull);
+                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned int off = ((j >> 1) * kReduceThreads + t) * 8 + (j & 1) * 4;
+                        const unsigned int nb = in_bounds_bytes(off, 4, 4);
+                        const float* g = reinterpret_cast<const float*>(base) + (nb ? e0 + off : 0ull);
+                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
+                    }
+                }
+            }
+        }
+        cp_async_commit();  // one group per step, empty or not, keeps the group count equal to the step count
+    }
+
+    // Consumes step pc: starts the copy kStages-1 steps ahead, waits for this step's bytes, widens to fp32.
+    __device__ __forceinline__ void fetch(const ReduceStep st, float (&x)[16]) {
+        issue(pc + kStages - 1);
+        cp_async_wait<kStages - 1>();
+        const unsigned int stage = smem_base + (pc % kStages) * kStageBytes;
+        uint4 v[4];
+        const int nv = (BF16 && st.kind == SRC_BF16) ? 2 : 4;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (j < nv) {
+                const unsigned int a = stage + (j * kReduceThreads + t) * 16;
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w) : "r"(a));
+            }
+        }
+        if (!BF16 || st.kind == SRC_F32) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                x[j * 4 + 0] = __uint_as_float(v[j].x);
+                x[j * 4 + 1] = __uint_as_float(v[j].y);
+                x[j * 4 + 2] = __uint_as_float(v[j].z);
+                x[j * 4 + 3] = __uint_as_float(v[j].w);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const unsigned int w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    x[j * 8 + i * 2 + 0] = __uint_as_float(w[i] << 16);  // widening bf16 -> fp32 is exact
+                    x[j * 8 + i * 2 + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+                }
+            }
+        }
+        ++pc;
+    }
+
+    __device__ __forceinline__ void skip() {  // an ADD_ACC step: no bytes, but its (empty) group is counted
+        issue(pc + kStages - 1);
+        ++pc;
+    }
+};
+
+// Runs the steps that belong to accumulator L, starting at a LOAD into L, until a step that belongs to
+// a shallower accumulator.  A step into L+1 opens a fused child subtree: one more level of this
+// function, whose accumulator is a separate set of registers, closed by ADD_ACC(L, L+1).
+template <int L, int A, bool BF16>
+__device__ __forceinline__ void eval_level(TileCtx<BF16>& cx, float (&acc)[16]) {
+    while (cx.pc < cx.n) {
+        const ReduceStep st = cx.steps[cx.pc];
+        if (L > 0 && (int)st.a < L) return;
+        if (st.a == L) {
+            float x[16];
+            cx.fetch(st, x);
+            if (st.code == OPC_LOAD) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = x[i];
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = combine(acc[i], x[i], cx.red_op);
+            }
+        } else {
+            if constexpr (L + 1 < A) {
+                float sub[16];
+                eval_level<L + 1, A, BF16>(cx, sub);
+                cx.skip();  // the ADD_ACC(L, L+1) that closes the subtree
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = combine(acc[i], sub[i], cx.red_op);
+            } else {
+                cx.skip();  // unreachable for a well-formed task (the planner bounds the depth by A)
+            }
+        }
+    }
+}
+
+template <int A, bool BF16>
+__global__ void __launch_bounds__(kReduceThreads) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
+    extern __shared__ __align__(16) unsigned char s_stage[];
+    __shared__ unsigned long long s_ptr[kMaxStepsPerWave];
+    const unsigned int t = threadIdx.x;
+    const unsigned long long t_start = global_timer_ns();
+    int cached_task = -1;
+
+    for (unsigned int g = blockIdx.x; g < w.total_tiles; g += gridDim.x) {
+        int ti = 0;
+        while (ti + 1 < (int)w.n_tasks && g >= w.tasks[ti + 1].tile_begin) ++ti;
+        const ReduceTask& task = w.tasks[ti];
+        if (ti != cached_task) {
+            __syncthreads();  // everyone is done with the previous task's pointers
+            for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
+                const ReduceStep st = w.steps[task.step_begin + i];
+                s_ptr[i] = st.code == OPC_ADD_ACC ? 0ull : w.dir[st.row].ptr;
+            }
+            cached_task = ti;
+            __syncthreads();
+        }
+        const unsigned int lt = g - task.tile_begin;
+        const unsigned int c = task.c_begin + lt / task.tiles_per_chunk;
+        const unsigned int j = lt % task.tiles_per_chunk;
+        const unsigned long long e0 = (unsigned long long)c * task.chunk_elems + (unsigned long long)j * kTileElems;
+        unsigned long long e1 = e0 + kTileElems;
+        const unsigned long long chunk_end = (unsigned long long)(c + 1) * task.chunk_elems;
+        if (e1 > chunk_end) e1 = chunk_end;
+        if (e1 > task.elems) e1 = task.elems;
+        if (e0 >= e1) continue;
+
+        if (task.poll) {
+            int ok = 1;
+            for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
+                const ReduceStep st = w.steps[task.step_begin + i];
+                if (st.code != OPC_ADD_ACC) ok &= wait_chunk(w.dir, w.status, st.row, c, t_start, w.budget_ns) ? 1 : 0;
+            }
+            if (!__syncthreads_and(ok)) return;
+        }
+
+        TileCtx<BF16> cx;
+        cx.steps = &w.steps[task.step_begin];
+        cx.s_ptr = s_ptr;
+        cx.smem_base = (unsigned int)__cvta_generic_to_shared(s_stage);
+        cx.n = task.n_steps;
+        cx.pc = 0;
+        cx.red_op = task.red_op;
+        cx.t = t;
+        cx.e0 = e0;
+        cx.count = (unsigned int)(e1 - e0);
+#pragma unroll
+        for (int i = 0; i < kStages - 1; ++i) cx.issue(i);
+
+        float acc[16];
+        eval_level<0, A, BF16>(cx, acc);
+        cp_async_wait<0>();
+
+        float* out = reinterpret_cast<float*>(task.out_ptr) + e0;
+        const unsigned int count = cx.count;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const unsigned int off = BF16 ? ((q >> 1) * kReduceThreads + t) * 8 + (q & 1) * 4 : (q * kReduceThreads + t) * 4;
+            if (off + 4 <= count) {
+                *reinterpret_cast<float4*>(out + off) = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
+            } else {
+                for (int i = 0; i < 4; ++i)
+                    if (off + i < count) out[off + i] = acc[q * 4 + i];
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ fan-out
+__global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __grid_constant__ FanoutWave w) {
+    __shared__ unsigned long long s_dst[kMaxFanoutDst];
+    __shared__ unsigned long long s_src;
+    const unsigned int t = threadIdx.x;
+    const unsigned long long t_start = global_timer_ns();
+    int cached_task = -1;
+
+    for (unsigned int g = blockIdx.x; g < w.total_tiles; g += gridDim.x) {
+        int ti = 0;
+        while (ti + 1 < (int)w.n_tasks && g >= w.tasks[ti + 1].tile_begin) ++ti;
+        const FanoutTask& task = w.tasks[ti];
+        if (ti != cached_task) {
+            __syncthreads();
+            for (unsigned int i = t; i < task.n_dst; i += kFanoutThreads) s_dst[i] = w.dir[w.dst_rows[task.dst_begin + i]].ptr;
+            if (t == 0) s_src = w.dir[task.src_row].ptr;
+            cached_task = ti;
+            __syncthreads();
+        }
+        const unsigned int lt = g - task.tile_begin;
+        const unsigned int c = task.c_begin + lt / task.tiles_per_chunk;
+        const unsigned int j = lt % task.tiles_per_chunk;
+        const unsigned long long b0 = (unsigned long long)c * task.chunk_bytes + (unsigned long long)j * kFanoutTileBytes;
+        unsigned long long b1 = b0 + kFanoutTileBytes;
+        const unsigned long long chunk_end = (unsigned long long)(c + 1) * task.chunk_bytes;
+        if (b1 > chunk_end) b1 = chunk_end;
+        if (b1 > task.bytes) b1 = task.bytes;
+        if (b0 >= b1) continue;
+
+        if (task.poll) {
+            int ok = 1;
+            if (t == 0) ok = wait_chunk(w.dir, w.status, task.src_row, c, t_start, w.budget_ns) ? 1 : 0;
+            if (!__syncthreads_and(ok)) return;
+        }
+
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(s_src) + b0;
+        const unsigned int count = (unsigned int)(b1 - b0);
+        const unsigned int n_dst = task.n_dst;
+        if (count == kFanoutTileBytes) {
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = __ldcg(reinterpret_cast<const uint4*>(src) + q * kFanoutThreads + t);
+            for (unsigned int r = 0; r < n_dst; ++r) {
+                uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(s_dst[r]) + b0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) __stcs(dst + q * kFanoutThreads + t, v[q]);
+            }
+        } else {
+            const unsigned int n_vec = count / 16;
+            for (unsigned int q = t; q < n_vec; q += kFanoutThreads) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(src) + q);
+                for (unsigned int r = 0; r < n_dst; ++r)
+                    __stcs(reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(s_dst[r]) + b0) + q, v);
+            }
+            for (unsigned int b = n_vec * 16 + t; b < count; b += kFanoutThreads) {
+                const unsigned char v = src[b];
+                for (unsigned int r = 0; r < n_dst; ++r) (reinterpret_cast<unsigned char*>(s_dst[r]) + b0)[b] = v;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ launchers
+template <int A, bool BF16>
+static int launch_reduce_t(const ReduceWave& w, int grid, cudaStream_t s) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kReduceSmemBytes);
+        if (e != cudaSuccess) return (int)e;
+        attr_set = true;
+    }
+    reduce_wave_kernel<A, BF16><<<grid, kReduceThreads, kReduceSmemBytes, s>>>(w);
+    return (int)cudaGetLastError();
+}
+
+int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, int grid, void* stream) {
+    cudaStream_t s = (cudaStream_t)stream;
+    if (n_acc <= 2) return bf16 ? launch_reduce_t<2, true>(w, grid, s) : launch_reduce_t<2, false>(w, grid, s);
+    if (n_acc <= 4) return bf16 ? launch_reduce_t<4, true>(w, grid, s) : launch_reduce_t<4, false>(w, grid, s);
+    return bf16 ? launch_reduce_t<kMaxAcc, true>(w, grid, s) : launch_reduce_t<kMaxAcc, false>(w, grid, s);
+}
+
+int launch_fanout_wave(const FanoutWave& w, int grid, void* stream) {
+    fanout_wave_kernel<<<grid, kFanoutThreads, 0, (cudaStream_t)stream>>>(w);
+    return (int)cudaGetLastError();
+}
+
+template <int A, bool BF16>
+static int occ_t() {
+    int n = 0;
+    if (cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kReduceSmemBytes) != cudaSuccess) return 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reduce_wave_kernel<A, BF16>, kReduceThreads, kReduceSmemBytes) != cudaSuccess) return 1;
+    return n < 1 ? 1 : n;
+}
+
+int reduce_ctas_per_sm(int n_acc, bool bf16) {
+    if (n_acc <= 2) return bf16 ? occ_t<2, true>() : occ_t<2, false>();
+    if (n_acc <= 4) return bf16 ? occ_t<4, true>() : occ_t<4, false>();
+    return bf16 ? occ_t<kMaxAcc, true>() : occ_t<kMaxAcc, false>();
+}
+
+int fanout_ctas_per_sm() {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fanout_wave_kernel, kFanoutThreads, 0) != cudaSuccess) return 1;
+    return n < 1 ? 1 : n;
+}
+
+}  // namespace hpl

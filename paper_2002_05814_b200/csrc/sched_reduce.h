@@ -1,0 +1,79 @@
+// Reduce schedule builder (host side, no CUDA): tree shape, arrival-order placement, k-of-m
+// selection and failure edits of Hoplite's Reduce (arXiv 2002.05814, Sections 3.4.2 and 3.5.2).
+//
+// The tree over k objects is the complete d-ary tree on positions 0..k-1 in level order.  An
+// arriving object takes the first open position of the generalised in-order traversal (first
+// child's subtree, the node, then the other children's subtrees).  Arrivals beyond k wait as
+// spares.  A failed member leaves at once: the oldest spare replaces it, else the position stays
+// open for the next arrival while enough live sources remain, else the tree shrinks by its last
+// position and the object there (if any) moves into the opening.  Ancestors of every touched
+// position lose their partial results.
+#pragma once
+#include <cstdint>
+#include <functional>
+#include <unordered_map>
+#include <vector>
+
+namespace hpl {
+
+enum { RED_EDIT_REPLACE = 1, RED_EDIT_HOLE = 2, RED_EDIT_SHRINK = 3 };
+
+struct ReduceEdit {
+    int64_t epoch, kind, pos, old_obj, new_obj, moved_from, hi_failed, hi_moved;
+    std::vector<int> cleared;
+};
+
+// What an edit means for materialised results: positions whose own partial must be recomputed.
+struct ReduceInvalidation {
+    std::vector<int> positions;   // includes the vacated position itself and all cleared ancestors
+    bool shrank = false;          // the last position disappeared
+};
+
+class ReduceTreeSchedule {
+public:
+    ReduceTreeSchedule(const std::vector<int64_t>& srcs, int k, int d);
+
+    int k() const { return k_; }
+    int k_requested() const { return k0_; }
+    int d() const { return d_; }
+    int64_t object_at(int pos) const { return at_[pos]; }
+    int position_of(int64_t obj) const;
+    bool has_source(int64_t obj) const { return alive_.count(obj) != 0; }
+    bool full() const;
+    int live() const;
+    const std::vector<int64_t>& sources() const { return srcs_; }
+
+    int parent(int p) const { return p == 0 ? -1 : (p - 1) / d_; }
+    int first_child(int p) const { return d_ * p + 1; }
+    int n_children(int p) const;
+    bool is_leaf(int p) const { return (int64_t)d_ * p + 1 >= k_; }
+
+    // events; each returns the positions whose materialised results are no longer valid
+    void arrive(int64_t obj);
+    ReduceInvalidation fail(int64_t obj, int64_t delivered_chunks, const std::function<int64_t(int64_t)>& delivered_of);
+
+    void dump(int64_t target, std::vector<int64_t>& w) const;
+
+private:
+    int first_open() const;
+    void assign(int64_t obj, int pos);
+    void shrink(int p, int64_t old_obj, int64_t hi_failed, const std::function<int64_t(int64_t)>& delivered_of,
+                ReduceInvalidation& inv);
+    std::vector<int> strict_ancestors(int p) const;
+
+    std::vector<int64_t> srcs_;
+    int k0_, k_, d_;
+    int64_t epoch_ = 0;
+    std::unordered_map<int64_t, bool> alive_;
+    std::unordered_map<int64_t, bool> arrived_;
+    std::unordered_map<int64_t, int> pos_;
+    std::vector<int64_t> at_;
+    std::vector<int64_t> spares_;
+    std::vector<std::pair<int64_t, int>> placements_;
+    std::vector<ReduceEdit> edits_;
+};
+
+// Positions of the complete d-ary tree on k nodes in generalised in-order.
+std::vector<int> generalised_inorder(int k, int d);
+
+}  // namespace hpl

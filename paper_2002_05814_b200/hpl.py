@@ -1,0 +1,199 @@
+"""ctypes binding of ``include/hpl.h``: the same calls, argument marshalling only.
+
+Every step of the hot path runs inside the library; nothing here computes.  Device pointers
+are plain integers (e.g. ``tensor.data_ptr()``), host buffers anything exposing the buffer
+protocol or an integer address.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HPL_OK = 0
+HPL_ERR_INVALID, HPL_ERR_NOT_FOUND, HPL_ERR_EXISTS, HPL_ERR_TIMEOUT = -1, -2, -3, -4
+HPL_ERR_INSUFFICIENT, HPL_ERR_FAILED_WORKER, HPL_ERR_CUDA, HPL_ERR_NOMEM = -5, -6, -7, -8
+HPL_F32, HPL_BF16 = 0, 1
+HPL_SUM, HPL_MIN, HPL_MAX = 0, 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libhpl.so")
+
+
+class Config(C.Structure):
+    """Mirror of ``hpl_config``."""
+    _fields_ = [("chunk_bytes", C.c_uint64), ("reduce_degree", C.c_int32), ("bcast_degree", C.c_int32),
+                ("virt_chunk_ns", C.c_uint64), ("poll_budget_ns", C.c_uint64), ("eager", C.c_int32),
+                ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("reserved", C.c_int32),
+                ("arena", C.c_void_p), ("arena_bytes", C.c_uint64)]
+
+
+class Stats(C.Structure):
+    """Mirror of ``hpl_stats_t``."""
+    _fields_ = [(n, C.c_uint64) for n in ("kernel_launches", "reduce_tasks", "fanout_tasks", "tiles",
+                                          "bytes_read_planned", "bytes_written_planned", "device_timeouts",
+                                          "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid")] + \
+               [("reserved", C.c_uint64 * 5)]
+
+
+class HplError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {code} ({_strerror(code)})")
+
+
+def _strerror(code: int) -> str:
+    try:
+        return load_library().hpl_strerror(code).decode()
+    except Exception:  # pragma: no cover
+        return "?"
+
+
+def load_library():
+    """Loads ``libhpl.so``.  There is no fallback: a missing library is an error."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `python -m paper_2002_05814_b200.build`")
+    lib = C.CDLL(path)
+    P, I32, I64, U64, VP = C.POINTER, C.c_int32, C.c_int64, C.c_uint64, C.c_void_p
+    sig = {
+        "hpl_init": [P(Config), VP, P(VP)],
+        "hpl_shutdown": [VP],
+        "hpl_advance": [VP, U64],
+        "hpl_create": [VP, I64, I32, U64, I32],
+        "hpl_put": [VP, I64, VP, U64],
+        "hpl_put_host": [VP, I64, VP, U64],
+        "hpl_reduce": [VP, I64, P(I64), I32, I32, I32, I32],
+        "hpl_broadcast": [VP, I64, P(I64), I32],
+        "hpl_join": [VP, I64, VP],
+        "hpl_get": [VP, I64, P(VP), P(U64)],
+        "hpl_get_host": [VP, I64, VP, U64],
+        "hpl_fail": [VP, I32],
+        "hpl_delete": [VP, I64],
+        "hpl_progress": [VP],
+        "hpl_sync": [VP],
+        "hpl_schedule_dump": [VP, I64, P(I64), U64, P(U64)],
+        "hpl_stats": [VP, P(Stats)],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.hpl_strerror.argtypes = [C.c_int]
+    lib.hpl_strerror.restype = C.c_char_p
+    _LIB = lib
+    return lib
+
+
+def _addr(buf) -> int:
+    if isinstance(buf, int):
+        return buf
+    if hasattr(buf, "data_ptr"):        # torch tensor (host or device)
+        return buf.data_ptr()
+    if hasattr(buf, "ctypes"):          # numpy array
+        return buf.ctypes.data
+    return C.addressof(C.c_char.from_buffer(buf))
+
+
+class Context:
+    """One ``hpl_ctx``.  Methods are the C calls of the same name; errors raise :class:`HplError`
+    unless the method is documented to return the code."""
+
+    def __init__(self, chunk_bytes: int, reduce_degree: int = 2, bcast_degree: int = 2, *, arena=0,
+                 arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
+                 eager: bool = False, plan_ahead: bool = False, fuse: bool = True):
+        self._lib = load_library()
+        cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
+                     int(plan_ahead), int(fuse), 0, _addr(arena) if arena else None, arena_bytes)
+        self._h = C.c_void_p()
+        self._check(self._lib.hpl_init(C.byref(cfg), C.c_void_p(stream or None), C.byref(self._h)), "hpl_init")
+
+    def _check(self, rc: int, what: str) -> int:
+        if rc != HPL_OK:
+            raise HplError(rc, what)
+        return rc
+
+    def shutdown(self):
+        if self._h:
+            self._lib.hpl_shutdown(self._h)
+            self._h = C.c_void_p()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.shutdown()
+
+    def advance(self, t_ns: int):
+        self._check(self._lib.hpl_advance(self._h, t_ns), "hpl_advance")
+
+    def create(self, object_id: int, worker: int, total_bytes: int, dtype: int = HPL_F32):
+        self._check(self._lib.hpl_create(self._h, object_id, worker, total_bytes, dtype), "hpl_create")
+
+    def put(self, object_id: int, dev_buf, nbytes: int):
+        self._check(self._lib.hpl_put(self._h, object_id, C.c_void_p(_addr(dev_buf)), nbytes), "hpl_put")
+
+    def put_host(self, object_id: int, host_buf, nbytes: int):
+        self._check(self._lib.hpl_put_host(self._h, object_id, C.c_void_p(_addr(host_buf)), nbytes), "hpl_put_host")
+
+    def reduce(self, target_id: int, src_ids, k_first_ready: int, op: int = HPL_SUM, dtype: int = HPL_F32):
+        arr = (C.c_int64 * len(src_ids))(*src_ids)
+        self._check(self._lib.hpl_reduce(self._h, target_id, arr, len(src_ids), k_first_ready, op, dtype), "hpl_reduce")
+
+    def broadcast(self, src_id: int, dst_ids):
+        arr = (C.c_int64 * len(dst_ids))(*dst_ids)
+        self._check(self._lib.hpl_broadcast(self._h, src_id, arr, len(dst_ids)), "hpl_broadcast")
+
+    def join(self, dst_id: int, dev_buf=0):
+        self._check(self._lib.hpl_join(self._h, dst_id, C.c_void_p(_addr(dev_buf) if dev_buf is not None else None)), "hpl_join")
+
+    def get(self, object_id: int):
+        """Returns ``(device_pointer, nbytes)``."""
+        p, n = C.c_void_p(), C.c_uint64()
+        self._check(self._lib.hpl_get(self._h, object_id, C.byref(p), C.byref(n)), "hpl_get")
+        return p.value, n.value
+
+    def try_get(self, object_id: int):
+        """As :meth:`get` but returns ``(code, device_pointer, nbytes)`` instead of raising."""
+        p, n = C.c_void_p(), C.c_uint64()
+        rc = self._lib.hpl_get(self._h, object_id, C.byref(p), C.byref(n))
+        return rc, p.value, n.value
+
+    def get_host(self, object_id: int, host_buf, cap: int):
+        self._check(self._lib.hpl_get_host(self._h, object_id, C.c_void_p(_addr(host_buf)), cap), "hpl_get_host")
+
+    def fail(self, worker: int):
+        self._check(self._lib.hpl_fail(self._h, worker), "hpl_fail")
+
+    def delete(self, object_id: int):
+        self._check(self._lib.hpl_delete(self._h, object_id), "hpl_delete")
+
+    def progress(self):
+        self._check(self._lib.hpl_progress(self._h), "hpl_progress")
+
+    def sync(self) -> int:
+        """Returns the code (HPL_OK or HPL_ERR_TIMEOUT) instead of raising on a timeout."""
+        rc = self._lib.hpl_sync(self._h)
+        if rc not in (HPL_OK, HPL_ERR_TIMEOUT):
+            raise HplError(rc, "hpl_sync")
+        return rc
+
+    def schedule_dump(self, op_id: int) -> list[int]:
+        n = C.c_uint64()
+        rc = self._lib.hpl_schedule_dump(self._h, op_id, None, 0, C.byref(n))
+        if rc == HPL_ERR_NOT_FOUND:
+            raise HplError(rc, "hpl_schedule_dump")
+        buf = (C.c_int64 * n.value)()
+        self._check(self._lib.hpl_schedule_dump(self._h, op_id, buf, n.value, C.byref(n)), "hpl_schedule_dump")
+        return list(buf)
+
+    def stats(self) -> dict:
+        st = Stats()
+        self._check(self._lib.hpl_stats(self._h, C.byref(st)), "hpl_stats")
+        return {name: getattr(st, name) for name, _ in Stats._fields_ if name != "reserved"}

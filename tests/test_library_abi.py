@@ -1,0 +1,71 @@
+"""The C-ABI library loads on a machine without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2002_05814_b200 as hpl
+from paper_2002_05814_b200 import build as hpl_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    hpl_build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "hpl.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hpl_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = _declared()
+    assert {"hpl_put", "hpl_reduce", "hpl_broadcast", "hpl_get", "hpl_fail"} <= set(names)
+    lib = ctypes.CDLL(hpl.lib_path())
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_error_strings_and_argument_checks():
+    lib = hpl.load_library()
+    for code in range(0, -9, -1):
+        assert lib.hpl_strerror(code)
+    with pytest.raises(hpl.HplError) as ei:
+        hpl.Context(chunk_bytes=24)            # not a multiple of 16
+    assert ei.value.code == hpl.HPL_ERR_INVALID
+    with hpl.Context(chunk_bytes=64) as c:     # schedule-only context: no device memory given
+        c.create(1, 0, 256)
+        with pytest.raises(hpl.HplError) as ei:
+            c.create(1, 0, 256)
+        assert ei.value.code == hpl.HPL_ERR_EXISTS
+        with pytest.raises(hpl.HplError) as ei:
+            c.create(2, 0, 255)                 # not a whole number of elements
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+        with pytest.raises(hpl.HplError) as ei:
+            c.put(3, 16, 4)
+        assert ei.value.code == hpl.HPL_ERR_NOT_FOUND
+        with pytest.raises(hpl.HplError) as ei:
+            c.put(1, 8, 4)                      # misaligned
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+        c.put(1, 16, 128)
+        with pytest.raises(hpl.HplError) as ei:
+            c.put(1, 16, 64)                    # the prefix never shrinks
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+        with pytest.raises(hpl.HplError) as ei:
+            c.advance(5), c.advance(4)
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+        with pytest.raises(hpl.HplError) as ei:
+            c.reduce(9, [1, 1], 1)
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+        rc, _, _ = c.try_get(1)
+        assert rc == hpl.HPL_ERR_TIMEOUT        # partial object
+        c.put(1, 16, 256)
+        rc, _, _ = c.try_get(1)
+        assert rc == hpl.HPL_ERR_CUDA           # complete, but this context has no device
+        with pytest.raises(hpl.HplError) as ei:
+            c.put_host(1, bytearray(256), 256)
+        assert ei.value.code in (hpl.HPL_ERR_CUDA, hpl.HPL_ERR_INVALID)

@@ -1,0 +1,193 @@
+"""Schedules built by the library (host code, no GPU needed) against the oracle, bit for bit, on
+randomised timelines of puts, joins, failures and gets."""
+import numpy as np
+import pytest
+
+import paper_2002_05814_b200 as hpl
+from oracle.store import OracleStore, StoreError, OK, ERR_TIMEOUT
+from paper_2002_05814_b200 import build as hpl_build
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    hpl_build.build()
+
+
+CHUNK = 64
+
+
+class Pair:
+    """Drives the oracle and a schedule-only library context with the same events."""
+
+    def __init__(self, d_reduce, d_bcast, tau):
+        self.o = OracleStore(CHUNK, d_reduce, d_bcast, tau)
+        self.c = hpl.Context(CHUNK, d_reduce, d_bcast, virt_chunk_ns=tau)
+        self.data = {}
+        self.addr = {}
+
+    def close(self):
+        self.c.shutdown()
+
+    def both(self, name, *args, oracle_args=None):
+        ro = OK
+        try:
+            getattr(self.o, name)(*(oracle_args if oracle_args is not None else args))
+        except StoreError as e:
+            ro = e.code
+        rl = OK
+        try:
+            getattr(self.c, name)(*args)
+        except hpl.HplError as e:
+            rl = e.code
+        assert ro == rl, (name, args, ro, rl)
+        return ro
+
+    def create(self, oid, worker, nbytes):
+        self.data[oid] = np.zeros(nbytes // 4, np.float32)
+        self.addr[oid] = 4096 * (oid + 1)
+        return self.both("create", oid, worker, nbytes, 0)
+
+    def put(self, oid, nbytes):
+        ro = OK
+        try:
+            self.o.put(oid, self.data[oid], nbytes)
+        except StoreError as e:
+            ro = e.code
+        rl = OK
+        try:
+            self.c.put(oid, self.addr[oid], nbytes)
+        except hpl.HplError as e:
+            rl = e.code
+        assert ro == rl, ("put", oid, nbytes, ro, rl)
+
+    def join(self, oid):
+        ro = OK
+        try:
+            self.o.join(oid)
+        except StoreError as e:
+            ro = e.code
+        rl = OK
+        try:
+            self.c.join(oid, None)
+        except hpl.HplError as e:
+            rl = e.code
+        assert ro == rl, ("join", oid, ro, rl)
+
+    def get(self, oid):
+        ro = OK
+        try:
+            self.o.get(oid)
+        except StoreError as e:
+            ro = e.code
+        rl, _, _ = self.c.try_get(oid)
+        if ro == OK:
+            assert rl == hpl.HPL_ERR_CUDA, (oid, rl)   # would succeed with a device
+        else:
+            assert rl == ro, ("get", oid, ro, rl)
+        return ro
+
+    def compare(self, op_id):
+        assert self.c.schedule_dump(op_id) == self.o.dump(op_id)
+
+
+def _reduce_timeline(seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(1, 13))
+    k = int(rng.integers(1, n + 1))
+    d = int(rng.integers(1, 5))
+    nbytes = int(rng.integers(1, 9)) * 64 - (0 if rng.random() < 0.7 else 60)
+    p = Pair(d, 1, 7)
+    n_workers = max(1, int(rng.integers(1, n + 1)))
+    for i in range(n):
+        p.create(i, int(rng.integers(0, n_workers)), nbytes)
+    t = 0
+    called = False
+    order = list(rng.permutation(n))
+    prefix = {i: 0 for i in range(n)}
+    steps = int(rng.integers(n, 4 * n + 4))
+    for s in range(steps):
+        t += int(rng.integers(0, 20))
+        p.both("advance", t)
+        r = rng.random()
+        if not called and (r < 0.25 or s == steps // 2):
+            if p.both("reduce", 1000, list(range(n)), k, 0, 0) != OK:
+                p.close()
+                return        # refused alike by both (e.g. no live source left)
+            called = True
+        elif r < 0.7 and order:
+            i = int(order[0])
+            full = rng.random() < 0.6
+            nb = nbytes if full else int(rng.integers(prefix[i], nbytes + 1))
+            nb -= nb % 4
+            nb = max(nb, prefix[i])
+            if nb == 0:
+                nb = nbytes
+            p.put(i, nb)
+            prefix[i] = nb
+            if nb == nbytes:
+                order.pop(0)
+        elif r < 0.85:
+            p.both("fail", int(rng.integers(0, n_workers)))
+        elif called:
+            p.get(1000)
+        if called:
+            p.compare(1000)
+    if called:
+        p.get(1000)
+        p.compare(1000)
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(8))
+def test_reduce_schedules_match_on_random_timelines(block):
+    for seed in range(block * 150, (block + 1) * 150):
+        _reduce_timeline(seed)
+
+
+def _bcast_timeline(seed):
+    rng = np.random.default_rng(seed)
+    R = int(rng.integers(1, 14))
+    d = int(rng.integers(1, 4))
+    tau = int(rng.integers(1, 30))
+    nbytes = int(rng.integers(1, 12)) * 64
+    p = Pair(2, d, tau)
+    n_workers = int(rng.integers(1, R + 2))
+    p.create(0, int(rng.integers(0, n_workers)) if rng.random() < 0.3 else 99, nbytes)
+    for j in range(1, R + 1):
+        p.create(j, int(rng.integers(0, n_workers)), nbytes)
+    t = 0
+    src_pref = 0
+    if rng.random() < 0.5:
+        src_pref = nbytes if rng.random() < 0.6 else int(rng.integers(0, nbytes // 64 + 1)) * 64
+        if src_pref:
+            p.put(0, src_pref)
+    p.both("broadcast", 0, list(range(1, R + 1)))
+    joiners = list(rng.permutation(np.arange(1, R + 1)))
+    for s in range(int(rng.integers(R, 4 * R + 6))):
+        t += int(rng.integers(0, 3 * tau))
+        p.both("advance", t)
+        t = max(t, p.o.now)
+        r = rng.random()
+        if r < 0.45 and joiners:
+            p.join(int(joiners.pop(0)))
+        elif r < 0.6 and src_pref < nbytes:
+            src_pref = nbytes if rng.random() < 0.5 else min(nbytes, src_pref + 64)
+            p.put(0, src_pref)
+        elif r < 0.75:
+            p.both("fail", int(rng.integers(0, n_workers)))
+        else:
+            p.get(int(rng.integers(1, R + 1)))
+            t = max(t, p.o.now)
+        p.compare(0)
+    if src_pref < nbytes:
+        p.put(0, nbytes)
+    for j in range(1, R + 1):
+        p.get(j)
+        p.compare(0)
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(8))
+def test_broadcast_schedules_match_on_random_timelines(block):
+    for seed in range(block * 150, (block + 1) * 150):
+        _bcast_timeline(seed)
