@@ -1,0 +1,270 @@
+"""Parity of the CUDA reduce path with the oracle (through the C ABI), element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_05814_b200 as hpl
+import workloads as wl
+from oracle import values as ov
+from oracle.store import DT_F32, DT_BF16
+from tests.harness import Pair, gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2002_05814_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _norm_err(got32, ref64):
+    return float(np.max(np.abs(got32.astype(np.float64) - ref64)) / np.max(np.abs(ref64)))
+
+
+def test_cfg1_eight_objects_of_1mib_all_ready():
+    w = wl.workload("cfg1")
+    p = Pair(w.chunk_bytes, w.degree)
+    for i in range(8):
+        p.create(i, i, gen(w.dist, w.seed + i, i, w.elems))
+        p.put(i)
+    p.reduce(100, list(range(8)), 8)
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    ref = ov.naive_sum_f64(list(range(8)), p.host)
+    assert _norm_err(got, ref) <= 1e-5 * math.ceil(math.log2(8))
+    st = p.c.stats()
+    assert st["kernel_launches"] == 1 and st["reduce_tasks"] == 1      # the whole tree fused into one pass
+    assert st["bytes_read_planned"] == 8 << 20 and st["bytes_written_planned"] == 1 << 20
+    p.close()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+@pytest.mark.parametrize("k,d,elems,chunk", [
+    (1, 2, 256, 4096), (2, 2, 255, 4096), (3, 2, 4097, 1 << 14), (5, 3, 40_001, 1 << 14),
+    (8, 2, 100_003, 64 << 10), (8, 1, 70_000, 64 << 10), (9, 8, 33_333, 64 << 10),
+    (16, 4, 12_289, 16 << 10), (13, 2, 3 * 4096 + 1, 16 << 10), (31, 2, 5000, 4096),
+])
+def test_shapes_tails_and_degrees_f32(k, d, elems, chunk, fuse):
+    p = Pair(chunk, d, fuse=fuse)
+    order = list(np.random.default_rng(k * 7 + d).permutation(k))
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 77, i, elems))
+    p.reduce(100, list(range(k)), k)
+    for t, i in enumerate(order):
+        p.advance(10 * t)
+        p.put(int(i))
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert _norm_err(got, ov.naive_sum_f64(list(range(k)), p.host)) <= 1e-5 * max(1, math.ceil(math.log2(max(k, 2))))
+    p.close()
+
+
+@pytest.mark.parametrize("k,d,elems,chunk", [(4, 2, 4096 * 3 + 5, 16 << 10), (64, 4, 20_000, 8 << 10), (7, 2, 9, 4096),
+                                             (10, 3, 8 * 4096 + 3, 32 << 10)])
+def test_bf16_inputs_fp32_accumulate(k, d, elems, chunk):
+    p = Pair(chunk, d)
+    for i in range(k):
+        p.create(i, i, gen(("normal", 0.02), 5, i, elems, "bf16"))
+        p.put(i)
+    p.reduce(100, list(range(k)), k, 0, DT_BF16)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert _norm_err(got, ov.naive_sum_f64(list(range(k)), p.host)) <= 1e-5 * math.ceil(math.log2(max(k, 2)))
+    p.close()
+
+
+def test_bf16_partials_are_fp32_when_progress_comes_between_arrivals():
+    k, elems = 8, 3 * 4096 + 11
+    p = Pair(16 << 10, 2)
+    for i in range(k):
+        p.create(i, i, gen(("normal", 0.02), 6, i, elems, "bf16"))
+    p.reduce(100, list(range(k)), k, 0, DT_BF16)
+    for t, i in enumerate([3, 1, 0, 2, 7, 6, 5, 4]):
+        p.advance(t + 1)
+        p.put(i)
+        p.progress()
+    p.check_target_bits(100)
+    assert p.c.stats()["kernel_launches"] >= 3
+    p.close()
+
+
+@pytest.mark.parametrize("op", [hpl.HPL_MIN, hpl.HPL_MAX])
+def test_min_max(op):
+    p = Pair(16 << 10, 2)
+    for i in range(6):
+        p.create(i, i, gen(("uniform",), 9, i, 10_001))
+        p.put(i)
+    p.reduce(100, list(range(6)), 6, op)
+    got = p.check_target_bits(100).cpu().numpy()
+    ref = p.host[0]
+    for i in range(1, 6):
+        ref = (np.minimum if op == hpl.HPL_MIN else np.maximum)(ref, p.host[i])
+    assert np.array_equal(got, ref)
+    p.close()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+def test_progress_between_arrivals_materialises_and_reuses_partials(fuse):
+    """Objects arrive one by one and the library is asked to progress after each: subtrees are
+    reduced as soon as they are complete, later passes read those partial results."""
+    k, n, d, elems = 8, 12, 2, 50_000
+    p = Pair(64 << 10, d, fuse=fuse)
+    for i in range(n):
+        p.create(i, i, gen(("normal", 1e-3), 3, i, elems))
+    p.reduce(100, list(range(n)), k)
+    order = [5, 0, 11, 3, 7, 2, 9, 1, 4, 6, 8, 10]
+    launches = []
+    for t, i in enumerate(order):
+        p.advance(1000 * (t + 1))
+        p.put(i)
+        p.progress()
+        launches.append(p.c.stats()["kernel_launches"])
+    assert launches[1] >= 1            # the first two arrivals already form a complete subtree
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    members = order[:k]
+    assert _norm_err(got, ov.naive_sum_f64(members, p.host)) <= 1e-5 * 3
+    if fuse:
+        st = p.c.stats()
+        assert st["bytes_read_planned"] > k * elems * 4      # partial results were re-read: the price of early progress
+    p.close()
+
+
+def test_partial_puts_chunk_by_chunk():
+    k, elems, chunk = 4, 5 * 4096 + 100, 16 << 10      # 6 chunks, the last one short
+    p = Pair(chunk, 2)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 4, i, elems))
+    p.reduce(100, list(range(k)), k)
+    nbytes = elems * 4
+    t = 0
+    for step in range(1, 7):
+        for i in range(k):
+            t += 5
+            p.advance(t)
+            p.put(i, min(nbytes, step * chunk - (8 if (i + step) % 2 else 0)))   # some prefixes end inside a chunk
+            p.progress()
+    for i in range(k):
+        p.put(i, nbytes)
+    p.check_schedule(100)
+    p.check_target_bits(100)
+    assert p.c.stats()["kernel_launches"] >= 5
+    p.close()
+
+
+def test_integer_inputs_equal_brute_force_sum():
+    k, elems = 32, 30_000
+    p = Pair(32 << 10, 2)
+    for i in range(k):
+        p.create(i, i, gen(("smallint", 1000), 8, i, elems))
+        p.put(i)
+    p.reduce(100, list(range(k)), k)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert np.array_equal(got.astype(np.float64), ov.naive_sum_f64(list(range(k)), p.host))
+    p.close()
+
+
+# ------------------------------------------------------------------------------- failures
+@pytest.mark.parametrize("fuse", [True, False])
+@pytest.mark.parametrize("size", [1 << 10, 1 << 14, 1 << 18, 1 << 22])
+def test_cfg5_shape_worker_7_fails_after_40_percent(size, fuse):
+    """32 objects, no spare: worker 7 delivers 40 % of its chunks, the tree is used, then it fails;
+    the result is the sum over the 31 survivors."""
+    chunk = min(64 << 10, size)                      # scaled-down chunk so that small sizes still have many chunks
+    elems = size // 4
+    C = wl.n_chunks(size, chunk)
+    h = int(0.4 * C)
+    p = Pair(chunk, 2, fuse=fuse, arena_bytes=512 << 20)
+    for i in range(32):
+        p.create(i, i, gen(("smallint", 500), 12, i, elems))
+    p.reduce(100, list(range(32)), 32)
+    for i in range(32):
+        p.put(i, size if i != 7 else h * chunk)
+    p.progress()                                      # chunks below h are reduced with worker 7's data in them
+    before = p.c.stats()
+    p.advance(10)
+    p.fail(7)
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    survivors = [i for i in range(32) if i != 7]
+    assert np.array_equal(got.astype(np.float64), ov.naive_sum_f64(survivors, p.host))
+    after = p.c.stats()
+    if h > 0:
+        assert before["kernel_launches"] >= 1
+        redo = after["bytes_read_planned"] - before["bytes_read_planned"]
+        if not fuse:   # healthy partial results are kept: only the two root paths are recomputed below chunk h
+            assert redo < 31 * size
+    p.close()
+
+
+def test_failed_member_is_replaced_by_a_spare_and_by_a_later_arrival():
+    elems = 20_000
+    for spare_first in (True, False):
+        p = Pair(16 << 10, 2)
+        for i in range(10):
+            p.create(i, i, gen(("uniform",), 21, i, elems))
+        p.reduce(100, list(range(10)), 6)
+        for i in range(6):
+            p.advance(i + 1)
+            p.put(i)
+        p.progress()
+        if spare_first:
+            p.advance(20)
+            p.put(6)
+        p.advance(30)
+        p.fail(1)
+        if not spare_first:
+            rc, _, _ = p.c.try_get(100)
+            assert rc == hpl.HPL_ERR_TIMEOUT
+            p.advance(40)
+            p.put(6)
+        p.check_schedule(100)
+        got = p.check_target_bits(100).cpu().numpy()
+        assert _norm_err(got, ov.naive_sum_f64([0, 2, 3, 4, 5, 6], p.host)) <= 1e-5 * 3
+        p.close()
+
+
+def test_every_single_failure_position_small():
+    elems = 3000
+    for victim in range(7):
+        for d in (1, 2, 3):
+            p = Pair(4096, d, arena_bytes=16 << 20)
+            for i in range(7):
+                p.create(i, i, gen(("smallint", 50), 2, i, elems))
+            p.reduce(100, list(range(7)), 7)
+            for i in range(7):
+                p.put(i)
+            p.progress()
+            p.fail(victim)
+            p.check_schedule(100)
+            got = p.check_target_bits(100).cpu().numpy()
+            assert np.array_equal(got.astype(np.float64), ov.naive_sum_f64([i for i in range(7) if i != victim], p.host))
+            p.close()
+
+
+def test_reduce_with_missing_source_times_out_then_completes():
+    p = Pair(16 << 10, 2)
+    for i in range(3):
+        p.create(i, i, gen(("uniform",), 1, i, 10_000))
+    p.reduce(100, [0, 1, 2], 3)
+    p.put(0)
+    p.put(1)
+    rc, _, _ = p.c.try_get(100)
+    assert rc == hpl.HPL_ERR_TIMEOUT
+    p.put(2)
+    p.check_target_bits(100)
+    p.close()
+
+
+def test_deep_and_wide_trees():
+    for k, d in ((64, 1), (64, 64), (200, 2), (100, 3)):
+        p = Pair(8 << 10, d, arena_bytes=64 << 20)
+        for i in range(k):
+            p.create(i, i, gen(("uniform",), 6, i, 6000))
+            p.put(i)
+        p.reduce(1000, list(range(k)), k)
+        p.check_target_bits(1000)
+        p.close()
