@@ -1,0 +1,494 @@
+#!/usr/bin/env python
+"""Benchmark of the chunk-pipelined reduce / broadcast hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload cfg4] [--impl ours|reference]
+
+One step is one pass of the whole path over one batch of synthetic objects of the chosen workload:
+directory updates on Put, arrival ordering and tree formation, the kernels, Get.  The default workload
+is the policy round (broadcast a 64 MiB bf16 object to 64 receivers, then sum 64 returned bf16 objects
+in fp32, chunk 2 MiB, degree 4): the largest single-GPU configuration that uses both collectives.
+Inputs are resident in HBM before the timed region; every step is bracketed by CUDA events on the
+library's stream and the K steps by a barrier + synchronize.  Rank 0 prints one JSON line.
+
+With N > 1 every rank runs the same workload on its own GPU (independent rounds: the path has no
+exchange step between GPUs), the time is the maximum over ranks and the value the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads as wl  # noqa: E402
+
+MiB = 1 << 20
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------------------- helpers
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines: list[str] = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes(w: wl.Workload) -> dict:
+    """Bytes the method must move: every selected source read once and the result written once; the
+    broadcast source read once and every receiver written once."""
+    S = w.object_bytes
+    out = {"reduce": 0, "broadcast": 0}
+    if w.kind in ("reduce", "round"):
+        out["reduce"] = w.k * S + w.elems * 4
+    if w.kind == "ft_reduce":
+        out["reduce"] = (w.k - 1) * S + w.elems * 4          # the survivors and the result
+    if w.kind in ("broadcast", "round"):
+        out["broadcast"] = S + w.n_receivers * S
+    return out
+
+
+# ----------------------------------------------------------------------------------------- our arm
+class Runner:
+    """Holds the device buffers of one workload and runs steps through the C ABI."""
+
+    def __init__(self, w: wl.Workload, device, host_buffers: bool = False, plan_ahead: bool = False):
+        import torch
+        import paper_2002_05814_b200 as hpl
+
+        self.torch, self.hpl, self.w = torch, hpl, w
+        self.dt = hpl.HPL_BF16 if w.dtype == "bf16" else hpl.HPL_F32
+        S = w.object_bytes
+        self.host_buffers = host_buffers
+        n_src = w.n_objects
+        arena_bytes = 64 * MiB + 2 * w.elems * 4 + (n_src + 2) * S * (1 if host_buffers else 0)
+        if w.kind == "ft_reduce":
+            arena_bytes += 4 * w.elems * 4
+        self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
+        self.ctx = hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=arena_bytes,
+                               stream=torch.cuda.current_stream().cuda_stream, time_kernels=True,
+                               plan_ahead=plan_ahead)
+        self.src = [wl.values_torch(w.dist, w.seed + i, i, 0, w.elems, w.dtype, device=device) for i in range(n_src)]
+        self.policy = None
+        self.recv = []
+        if w.n_receivers:
+            self.policy = wl.values_torch(w.dist, w.seed + 1000, 1000, 0, w.elems, w.dtype, device=device)
+            self.recv = [torch.empty(S, dtype=torch.uint8, device=device) for _ in range(w.n_receivers)]
+        self.host_src, self.host_policy, self.host_out, self.host_recv = [], None, None, None
+        if host_buffers:
+            n_distinct = min(n_src, 8)      # pinned host images; objects beyond the 8th reuse them (same bytes to copy)
+            self.host_src = [self.src[i].cpu().pin_memory() for i in range(n_distinct)]
+            if self.policy is not None:
+                self.host_policy = self.policy.cpu().pin_memory()
+                self.host_recv = torch.empty(S, dtype=torch.uint8).pin_memory()
+            if n_src:
+                self.host_out = torch.empty(w.elems, dtype=torch.float32).pin_memory()
+        self.round = 0
+        self.t = 0
+        torch.cuda.synchronize()
+
+    def close(self):
+        self.ctx.shutdown()
+
+    # one pass of the whole path; returns (h2d bytes, d2h bytes) of the step
+    def step(self):
+        w, ctx, r = self.w, self.ctx, self.round
+        base = 0
+        S = w.object_bytes
+        h2d = d2h = 0
+        self.t += 1_000_000_000
+        ctx.advance(self.t)
+        ids_to_delete = []
+        if w.kind in ("broadcast", "round"):
+            src_id = base + 5000
+            dsts = [base + 6000 + j for j in range(w.n_receivers)]
+            ctx.create(src_id, 900, S, self.dt)
+            if self.host_buffers:
+                ctx.put_host(src_id, self.host_policy.data_ptr(), S)
+                h2d += S
+            else:
+                ctx.put(src_id, self.policy.data_ptr(), S)
+            for j, dd in enumerate(dsts):
+                ctx.create(dd, 1000 + j, S, self.dt)
+            ctx.broadcast(src_id, dsts)
+            if w.kind == "broadcast":
+                offs = wl.uniform_offsets_ns(w.seed + r, w.n_receivers, w.extra["join_window_ns"])
+                order = sorted(range(w.n_receivers), key=lambda j: (offs[j], j))
+                for j in order:
+                    ctx.advance(self.t + offs[j])
+                    ctx.join(dsts[j], self.recv[j].data_ptr())
+                self.t += w.extra["join_window_ns"]
+            else:
+                for j, dd in enumerate(dsts):
+                    ctx.join(dd, self.recv[j].data_ptr())
+            for dd in dsts:
+                ctx.get(dd)
+            if self.host_buffers:
+                ctx.get_host(dsts[-1], self.host_recv.data_ptr(), S)
+                d2h += S
+            self.t = max(self.t, 0)
+            ids_to_delete.append(src_id)
+        self.mid_event()
+        if w.kind in ("reduce", "round", "ft_reduce"):
+            n = w.n_objects
+            ids = [base + i for i in range(n)]
+            tgt = base + 9000
+            for i in ids:
+                ctx.create(i, i, S, self.dt)
+            if w.kind == "reduce" and "mean_arrival_ns" in w.extra:
+                arr = wl.exponential_arrivals_ns(w.seed + r, n, w.extra["mean_arrival_ns"])
+            else:
+                arr = [0] * n
+            order = sorted(range(n), key=lambda i: (arr[i], i))
+            ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
+            tmax = 0
+            for i in order:
+                ctx.advance(max(self.t + arr[i], self.t + tmax))
+                tmax = max(tmax, arr[i])
+                nbytes = S
+                if w.kind == "ft_reduce" and i == w.extra["fail_worker"]:
+                    C = wl.n_chunks(S, w.chunk_bytes)
+                    nbytes = int(w.extra["fail_fraction"] * C) * w.chunk_bytes
+                    if nbytes == 0:
+                        continue
+                if self.host_buffers:
+                    ctx.put_host(ids[i], self.host_src[i % len(self.host_src)].data_ptr(), nbytes)
+                    h2d += nbytes
+                else:
+                    ctx.put(ids[i], self.src[i].data_ptr(), nbytes)
+            self.t += tmax
+            if w.kind == "ft_reduce":
+                ctx.progress()                       # chunks delivered by every worker are reduced before the failure
+                self.t += 1
+                ctx.advance(self.t)
+                ctx.fail(w.extra["fail_worker"])
+            if self.host_buffers:
+                ctx.get_host(tgt, self.host_out.data_ptr(), w.elems * 4)
+                d2h += w.elems * 4
+            else:
+                ctx.get(tgt)
+            ids_to_delete += [tgt] + ids
+        self.end_event()
+        for i in ids_to_delete:
+            ctx.delete(i)
+        self.round += 1
+        return h2d, d2h
+
+    def mid_event(self):
+        pass
+
+    def end_event(self):
+        pass
+
+
+def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
+    torch = runner.torch
+    for _ in range(warmup):
+        runner.step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    cur = {"i": 0}
+    runner.mid_event = lambda: ev[cur["i"]][1].record()
+    runner.end_event = lambda: ev[cur["i"]][2].record()
+    st0 = runner.ctx.stats()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    h2d = d2h = 0
+    for i in range(steps):
+        cur["i"] = i
+        ev[i][0].record()
+        a, b = runner.step()
+        h2d, d2h = a, b
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    st1 = runner.ctx.stats()
+    runner.mid_event = runner.end_event = lambda: None
+    bc = [e[0].elapsed_time(e[1]) for e in ev]
+    rd = [e[1].elapsed_time(e[2]) for e in ev]
+    tot = [e[0].elapsed_time(e[2]) for e in ev]
+    delta = {k: st1[k] - st0[k] for k in st1}
+    return {"bcast_ms": bc, "reduce_ms": rd, "total_ms": tot, "wall_ms": wall_ms, "stats": delta,
+            "h2d": h2d, "d2h": d2h}
+
+
+def gbs(nbytes, ms):
+    return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+
+
+# ----------------------------------------------------------------------------------------- oracle arm
+def oracle_sample(w: wl.Workload, budget_s: float = 12.0):
+    """Times the oracle, as it stands, on a bounded sample of the workload: the same objects cut to a
+    window of their elements (same chunk size, same tree, same timeline).  Returns GB/s on the
+    algorithmic bytes of the sample."""
+    from oracle.store import OracleStore, DT_F32, DT_BF16
+
+    frac = 16
+    elems = max(4096, (w.elems // frac) // 8 * 8)
+    dt = DT_BF16 if w.dtype == "bf16" else DT_F32
+    distinct = [wl.values_np(w.dist, w.seed + i, i, 0, elems, w.dtype) for i in range(min(8, max(1, w.n_objects)))]
+    S = distinct[0].nbytes
+    sw = wl.Workload(**{**w.__dict__, "elems": elems})
+    ab = algorithmic_bytes(sw)
+    total_bytes = ab["reduce"] + ab["broadcast"]
+    reps, t_total = 0, 0.0
+    while t_total < budget_s and reps < 200:
+        o = OracleStore(w.chunk_bytes, w.degree, w.degree)
+        t0 = time.perf_counter()
+        if w.kind in ("broadcast", "round"):
+            o.create(5000, 900, S, dt)
+            o.put(5000, distinct[0], S)
+            dsts = [6000 + j for j in range(w.n_receivers)]
+            for j, dd in enumerate(dsts):
+                o.create(dd, 1000 + j, S, dt)
+            o.broadcast(5000, dsts)
+            offs = wl.uniform_offsets_ns(w.seed + reps, w.n_receivers, w.extra.get("join_window_ns", 1))
+            for j in sorted(range(w.n_receivers), key=lambda j: (offs[j], j)):
+                o.advance(max(o.now, offs[j] if w.kind == "broadcast" else 0))
+                o.join(dsts[j])
+            for dd in dsts:
+                o.get(dd)
+        if w.kind in ("reduce", "round", "ft_reduce"):
+            n = w.n_objects
+            for i in range(n):
+                o.create(i, i, S, dt)
+            arr = wl.exponential_arrivals_ns(w.seed + reps, n, w.extra["mean_arrival_ns"]) if "mean_arrival_ns" in w.extra else [0] * n
+            o.reduce(9000, list(range(n)), w.k, 0, dt)
+            base = o.now
+            for i in sorted(range(n), key=lambda i: (arr[i], i)):
+                o.advance(max(o.now, base + arr[i]))
+                nbytes = S
+                if w.kind == "ft_reduce" and i == w.extra["fail_worker"]:
+                    nbytes = int(w.extra["fail_fraction"] * wl.n_chunks(S, w.chunk_bytes)) * w.chunk_bytes
+                    if nbytes == 0:
+                        continue
+                o.put(i, distinct[i % len(distinct)], nbytes)
+            if w.kind == "ft_reduce":
+                o.fail(w.extra["fail_worker"])
+            o.get(9000)
+        t_total += time.perf_counter() - t0
+        reps += 1
+    value = total_bytes * reps / t_total / 1e9
+    sample = (f"{reps} pass(es) of the oracle over the first {elems} of {w.elems} elements of every object "
+              f"({total_bytes * reps / 1e9:.2f} GB algorithmic, {t_total:.1f} s, numpy single thread)")
+    return value, sample, t_total / reps * 1e3
+
+
+# ----------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--size", type=int, default=64 * MiB, help="object bytes for cfg5")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads measured briefly and reported under 'also'")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = wl.cfg5_at(args.size) if args.workload == "cfg5" else wl.workload(args.workload)
+    ab = algorithmic_bytes(w)
+    step_bytes = ab["reduce"] + ab["broadcast"]
+    name = {"cfg1": "cfg1 reduce 8 x 1 MiB fp32", "cfg2": "cfg2 broadcast 64 MiB fp32 to 16 receivers",
+            "cfg3": "cfg3 async-SGD reduce, first 8 of 16 x 97.5 MiB fp32",
+            "cfg4": "cfg4 policy round: broadcast 64 MiB bf16 to 64 receivers + fp32 sum of 64 x 64 MiB bf16",
+            "cfg5": f"cfg5 fault-tolerant reduce of 32 x {args.size} B fp32, worker 7 fails at 40%"}[w.name]
+    config = {"workload": name, "chunk_bytes": w.chunk_bytes, "degree": w.degree, "object_bytes": w.object_bytes,
+              "algorithmic_bytes_per_step": step_bytes, "l2": "inputs larger than L2 (no flush)",
+              "timed_region": "first Put of the step to the last Get, CUDA events on the library's stream; Delete outside"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        value, sample, ms = oracle_sample(w, budget_s=max(5.0, 4.0 * (args.steps + args.warmup)))
+        line = {"impl": "reference", "metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value,
+                "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": config, "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+                "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    from paper_2002_05814_b200 import build as hpl_build
+
+    if rank == 0 or world == 1:
+        hpl_build.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        torch.cuda.set_device(local)
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+        dist.barrier()
+    else:
+        torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+
+    sampler = ClockSampler(local)
+    runner = Runner(w, device)
+    sampler.start()
+    res = time_steps(runner, args.steps, args.warmup, dist)
+    clocks = sampler.stop()
+    runner.close()
+    del runner
+    torch.cuda.empty_cache()
+
+    total_ms = float(np.sum(res["total_ms"]))
+    if dist is not None:
+        tmax = torch.tensor([total_ms, res["wall_ms"]], device=device, dtype=torch.float64)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms, wall_ms = float(tmax[0]), float(tmax[1])
+    else:
+        wall_ms = res["wall_ms"]
+    value = gbs(step_bytes * args.steps * world, total_ms)
+    peak, peak_kind = measured_peak()
+    st = res["stats"]
+
+    def roof(kind_ns, kind_launches, per_launch_bytes):
+        if st[kind_launches] == 0:
+            return None
+        avg_ms = st[kind_ns] / st[kind_launches] / 1e6
+        ach = gbs(per_launch_bytes, avg_ms)
+        return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": None,
+                "peak_kind": f"of {peak_kind} (copy bandwidth)", "avg_launch_ms": avg_ms, "launches": st[kind_launches],
+                "algorithmic_bytes_per_launch": per_launch_bytes, "frac_of_8TBs_nominal": ach / 8000.0}
+
+    r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * args.steps / max(1, st["reduce_launches"])) if ab["reduce"] else None
+    r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * args.steps / max(1, st["fanout_launches"])) if ab["broadcast"] else None
+    line = {"metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value, "unit": "GB/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.dtype == "f32" else "f32 (bf16 inputs widened)", "data": "synthetic",
+            "config": config, "clocks": clocks, "gpu_launches": int(st["kernel_launches"]),
+            "wall_ms_per_step": wall_ms / args.steps,
+            "frac_of_hbm_peak": {"measured_copy": value / world / peak, "nominal_8TBs": value / world / 8000.0},
+            "roofline": r_red if r_red is not None else r_fan}
+    if r_red is not None and r_fan is not None:
+        line["roofline_fanout"] = r_fan
+    if ab["reduce"]:
+        line["reduce"] = {"GBps": gbs(ab["reduce"] * args.steps, float(np.sum(res["reduce_ms"]))), "ms": float(np.mean(res["reduce_ms"])),
+                          "ms_std": float(np.std(res["reduce_ms"]))}
+    if ab["broadcast"]:
+        line["broadcast"] = {"GBps": gbs(ab["broadcast"] * args.steps, float(np.sum(res["bcast_ms"]))), "ms": float(np.mean(res["bcast_ms"])),
+                             "ms_std": float(np.std(res["bcast_ms"]))}
+
+    if rank == 0 and world == 1 and args.also:
+        also = {}
+        for nm in [x for x in args.also.split(",") if x and x != w.name]:
+            ww = wl.workload(nm)
+            rr = Runner(ww, device)
+            r2 = time_steps(rr, 5, 3)
+            rr.close()
+            del rr
+            torch.cuda.empty_cache()
+            a2 = algorithmic_bytes(ww)
+            b2 = a2["reduce"] + a2["broadcast"]
+            g = gbs(b2 * 5, float(np.sum(r2["total_ms"])))
+            s2 = r2["stats"]
+            kn, kl = ("reduce_kernel_ns", "reduce_launches") if a2["reduce"] else ("fanout_kernel_ns", "fanout_launches")
+            kern = gbs(b2 * 5 / max(1, s2[kl]), s2[kn] / max(1, s2[kl]) / 1e6)
+            also[nm] = {"GBps": g, "ms_per_step": float(np.mean(r2["total_ms"])), "kernel_GBps": kern,
+                        "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / 5}
+        line["also"] = also
+
+    if not args.no_e2e:
+        e_steps = max(1, min(args.steps, 3))
+        rr = Runner(w, device, host_buffers=True, plan_ahead=True)
+        r3 = time_steps(rr, e_steps, 1, dist)
+        rr.close()
+        del rr
+        torch.cuda.empty_cache()
+        e_ms = float(np.sum(r3["total_ms"]))
+        if dist is not None:
+            tm = torch.tensor([e_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            e_ms = float(tm[0])
+        line["e2e"] = {"value": gbs(step_bytes * e_steps * world, e_ms), "unit": "GB/s", "h2d_bytes_per_step": int(r3["h2d"]),
+                       "d2h_bytes_per_step": int(r3["d2h"]), "ms_per_step": e_ms / e_steps,
+                       "how": "hpl_put_host from pinned host memory, chunks consumed by polling kernels as they land; hpl_get_host of the result"}
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        v, sample, _ = oracle_sample(w)
+        line["cpu_baseline"] = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

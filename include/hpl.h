@@ -66,7 +66,8 @@ typedef struct hpl_config {
                                  kernels poll the directory's progress counters for them (bounded) */
     int32_t  fuse;            /* 1: a subtree whose inputs are all ready is reduced in registers in one pass
                                  (same association, same bits); 0: every tree node writes its partial result */
-    int32_t  reserved;
+    int32_t  time_kernels;    /* 1: CUDA events are recorded around every kernel launch on the context's stream and
+                                 summed into hpl_stats_t at the next wait (for benchmarks) */
     void*    arena;           /* device memory the library may use for the directory, partial results, reduce
                                  targets and copies of host objects; owned by the caller, must outlive the
                                  context.  NULL = schedule-only context (no device work; hpl_get fails). */
@@ -171,7 +172,11 @@ typedef struct hpl_stats_t {
     uint64_t h2d_bytes;            /* copied by hpl_put_host */
     uint64_t d2h_bytes;            /* copied by hpl_get_host */
     uint64_t last_kernel_grid;     /* CTAs of the most recent launch */
-    uint64_t reserved[5];
+    uint64_t reduce_launches;      /* launches of the reduce kernel */
+    uint64_t fanout_launches;      /* launches of the fan-out kernel */
+    uint64_t reduce_kernel_ns;     /* summed device time of reduce launches (time_kernels = 1; updated by waits) */
+    uint64_t fanout_kernel_ns;
+    uint64_t reserved[1];
 } hpl_stats_t;
 
 int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);

@@ -210,6 +210,9 @@ struct hpl_ctx {
     hpl_stats_t stats{};
     int occ_reduce[2][3] = {{0, 0, 0}, {0, 0, 0}};
     int occ_fanout = 0;
+    struct Timed { cudaEvent_t a, b; int kind; };
+    std::vector<Timed> timed;            // event pairs of launches not yet read back
+    std::vector<cudaEvent_t> event_pool;
 };
 
 namespace {
@@ -258,6 +261,50 @@ int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
 
 int sync_and_check(hpl_ctx* c);
 int progress(hpl_ctx* c);
+
+cudaEvent_t take_event(hpl_ctx* c) {
+    if (!c->event_pool.empty()) {
+        cudaEvent_t e = c->event_pool.back();
+        c->event_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+// Brackets one launch with events when kernel timing is on (kind 0 = reduce, 1 = fan-out).
+struct LaunchTimer {
+    hpl_ctx* c;
+    int kind;
+    cudaEvent_t a = nullptr, b = nullptr;
+    LaunchTimer(hpl_ctx* ctx, int k) : c(ctx), kind(k) {
+        if (c->cfg.time_kernels) {
+            a = take_event(c);
+            b = take_event(c);
+            if (a) cudaEventRecord(a, c->stream);
+        }
+    }
+    ~LaunchTimer() {
+        if (a && b) {
+            cudaEventRecord(b, c->stream);
+            c->timed.push_back({a, b, kind});
+        }
+    }
+};
+
+void collect_kernel_times(hpl_ctx* c) {   // call only after the stream has been waited for
+    for (auto& t : c->timed) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) {
+            const uint64_t ns = (uint64_t)((double)ms * 1e6);
+            if (t.kind == 0) c->stats.reduce_kernel_ns += ns; else c->stats.fanout_kernel_ns += ns;
+        }
+        c->event_pool.push_back(t.a);
+        c->event_pool.push_back(t.b);
+    }
+    c->timed.clear();
+}
 
 void release_object_memory(hpl_ctx* c, Object& o) {
     if (o.lib_owned && o.ptr) c->arena.release(o.ptr);
@@ -532,8 +579,12 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16);
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
             if (grid < 1) grid = 1;
-            if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
+            {
+                LaunchTimer timer(c, 0);
+                if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
+            }
             c->stats.kernel_launches++;
+            c->stats.reduce_launches++;
             c->stats.tiles += w.total_tiles;
             c->stats.last_kernel_grid = (uint64_t)grid;
             c->work_in_flight = true;
@@ -671,8 +722,12 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
-        if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
+        {
+            LaunchTimer timer(c, 1);
+            if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
+        }
         c->stats.kernel_launches++;
+        c->stats.fanout_launches++;
         c->stats.tiles += w.total_tiles;
         c->stats.last_kernel_grid = (uint64_t)grid;
         c->work_in_flight = true;
@@ -740,6 +795,7 @@ int sync_and_check(hpl_ctx* c) {
     CUDA_TRY(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->work_in_flight = false;
+    collect_kernel_times(c);
     if (c->h_status->error) {
         c->stats.device_timeouts++;
         undo_journal(c);
@@ -860,6 +916,8 @@ int hpl_shutdown(hpl_ctx* c) {
     if (c->device) {
         cudaStreamSynchronize(c->copy_stream);
         cudaStreamSynchronize(c->stream);
+        collect_kernel_times(c);
+        for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
         cudaFreeHost(c->h_dir);
         cudaFreeHost(c->h_status);
         cudaFreeHost(c->h_iota);

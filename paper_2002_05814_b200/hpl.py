@@ -27,7 +27,7 @@ class Config(C.Structure):
     """Mirror of ``hpl_config``."""
     _fields_ = [("chunk_bytes", C.c_uint64), ("reduce_degree", C.c_int32), ("bcast_degree", C.c_int32),
                 ("virt_chunk_ns", C.c_uint64), ("poll_budget_ns", C.c_uint64), ("eager", C.c_int32),
-                ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("reserved", C.c_int32),
+                ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_uint64)]
 
 
@@ -35,8 +35,10 @@ class Stats(C.Structure):
     """Mirror of ``hpl_stats_t``."""
     _fields_ = [(n, C.c_uint64) for n in ("kernel_launches", "reduce_tasks", "fanout_tasks", "tiles",
                                           "bytes_read_planned", "bytes_written_planned", "device_timeouts",
-                                          "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid")] + \
-               [("reserved", C.c_uint64 * 5)]
+                                          "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
+                                          "reduce_launches", "fanout_launches", "reduce_kernel_ns",
+                                          "fanout_kernel_ns")] + \
+               [("reserved", C.c_uint64 * 1)]
 
 
 class HplError(RuntimeError):
@@ -107,10 +109,10 @@ class Context:
 
     def __init__(self, chunk_bytes: int, reduce_degree: int = 2, bcast_degree: int = 2, *, arena=0,
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
-                 eager: bool = False, plan_ahead: bool = False, fuse: bool = True):
+                 eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
-                     int(plan_ahead), int(fuse), 0, _addr(arena) if arena else None, arena_bytes)
+                     int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes)
         self._h = C.c_void_p()
         self._check(self._lib.hpl_init(C.byref(cfg), C.c_void_p(stream or None), C.byref(self._h)), "hpl_init")
 
