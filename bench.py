@@ -190,7 +190,8 @@ class Runner:
             if self.host_buffers:
                 ctx.get_host(dsts[-1], self.host_recv.data_ptr(), S)
                 d2h += S
-            self.t = max(self.t, 0)
+            self.t += 100_000_000          # the Gets let virtual time run until the copies had landed
+            ctx.advance(self.t)
             ids_to_delete.append(src_id)
         self.mid_event()
         if w.kind in ("reduce", "round", "ft_reduce"):
