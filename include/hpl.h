@@ -183,6 +183,30 @@ int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);
 
 const char* hpl_strerror(int code);
 
+/* Reduce for callers that cannot allocate device memory.  The paper has no counterpart: this is an
+ * addition for users of this library who run where cudaMalloc is off limits -- allocator callbacks,
+ * serving loops that have frozen their memory map, processes whose device memory all belongs to someone
+ * else -- and who therefore cannot hand hpl_init an arena either.  It needs no context.
+ *
+ * Computes out[j] = op over the n objects src_bufs[0..n-1] (device pointers, 16-byte aligned, `elems`
+ * elements of `dtype` each; the array src_bufs itself is host memory), all complete, taken as arriving in
+ * index order, in the association order of the degree-`degree` tree -- the same bits hpl_reduce gives for
+ * those arrivals.  `out`: device, fp32, `elems` elements, 16-byte aligned.  The work is enqueued on
+ * `cuda_stream` and not waited for.
+ *
+ * The few KiB of device memory the kernel needs besides inputs and output (directory rows of the operands,
+ * status record) are a fixed array inside the library image, held by every GPU that loads the library until
+ * the process exits.  Hence the limits: n <= HPL_NOALLOC_MAX_SOURCES and elems <= HPL_NOALLOC_MAX_ELEMS;
+ * a tree deeper than the kernel can fuse in registers (8 accumulators) is refused too.  Anything beyond
+ * returns HPL_ERR_INVALID and does nothing.  No cudaMalloc / cudaFree / allocating routine is called.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and the SM count;
+ * make that first call outside any stream capture.  All calls share the one array and each call rewrites
+ * it: two calls whose kernels may overlap on the GPU (different streams, no ordering) race -- order them. */
+#define HPL_NOALLOC_MAX_SOURCES 256
+#define HPL_NOALLOC_MAX_ELEMS   (1ull << 32)
+int hpl_reduce_noalloc(const void* const* src_bufs, int32_t n, int32_t degree, int32_t op, int32_t dtype,
+                       uint64_t elems, void* out, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhpl.so")
-SOURCES = ["hpl.cpp", "sched_reduce.cpp", "sched_bcast.cpp", "kernels.cu"]
+SOURCES = ["hpl.cpp", "sched_reduce.cpp", "sched_bcast.cpp", "kernels.cu", "noalloc.cu"]
 HEADERS = ["device_types.h", "sched_reduce.h", "sched_bcast.h", os.path.join("..", "..", "include", "hpl.h")]
 
 

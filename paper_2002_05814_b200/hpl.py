@@ -87,6 +87,8 @@ def load_library():
         fn = getattr(lib, name)
         fn.argtypes = args
         fn.restype = C.c_int
+    lib.hpl_reduce_noalloc.argtypes = [P(VP), I32, I32, I32, I32, U64, VP, VP]
+    lib.hpl_reduce_noalloc.restype = C.c_int
     lib.hpl_strerror.argtypes = [C.c_int]
     lib.hpl_strerror.restype = C.c_char_p
     _LIB = lib
@@ -199,3 +201,12 @@ class Context:
         st = Stats()
         self._check(self._lib.hpl_stats(self._h, C.byref(st)), "hpl_stats")
         return {name: getattr(st, name) for name, _ in Stats._fields_ if name != "reserved"}
+
+
+def reduce_noalloc(src_ptrs, degree: int, op: int, dtype: int, elems: int, out_ptr: int, stream: int = 0) -> int:
+    """``hpl_reduce_noalloc``: the tree reduce for callers that cannot allocate device memory (no context,
+    no arena; its small scratch is a fixed array inside the library).  ``src_ptrs``: device addresses of the
+    complete objects in arrival order; ``out_ptr``: device fp32 buffer.  Returns the library's code."""
+    lib = load_library()
+    arr = (C.c_void_p * len(src_ptrs))(*src_ptrs)
+    return lib.hpl_reduce_noalloc(arr, len(src_ptrs), degree, op, dtype, elems, C.c_void_p(out_ptr), C.c_void_p(stream or None))
