@@ -138,6 +138,7 @@ struct Object {
     void* ptr = nullptr;
     bool lib_owned = false;
     bool from_host = false;
+    bool async_counter = false;   // its counter travels on a side stream: kernels poll it until a wait confirms it
     uint64_t ready_bytes = 0;  // published prefix
     uint32_t landed = 0;       // chunks whose counter update is ordered before later launches on the main stream
     bool alive = true;
@@ -187,10 +188,11 @@ struct BcastOp {
 
 struct hpl_ctx {
     hpl_config cfg{};
-    cudaStream_t stream = nullptr, copy_stream = nullptr;
-    cudaEvent_t copy_ev = nullptr;
+    cudaStream_t stream = nullptr, copy_stream = nullptr, ctl_stream = nullptr;
+    cudaEvent_t copy_ev = nullptr, ctl_ev = nullptr;
     bool device = false;
     bool copy_pending = false;
+    bool ctl_pending = false;   // directory updates on the control stream not yet ordered before the main stream
     int n_sm = 0;
     uint64_t now = 0, tau = 1, seq = 0;
     int64_t next_internal = -1;  // ids of partial buffers: negative, never visible outside
@@ -248,7 +250,19 @@ int alloc_row(hpl_ctx* c, Object& o) {
     r.ready_chunks = (o.kind == OBJ_PLAIN) ? 0u : o.C;
     r.dtype = (unsigned)o.dtype;
     r.owner = (unsigned)o.worker;
-    CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->stream));
+    // With plan-ahead a kernel that polls may occupy the main stream for a while, so directory rows travel
+    // on the control stream (tiny copies only) and the main stream is ordered after it before each launch.
+    cudaStream_t s = c->cfg.plan_ahead ? c->ctl_stream : c->stream;
+    CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, s));
+    if (c->cfg.plan_ahead) c->ctl_pending = true;
+    return HPL_OK;
+}
+
+int order_main_after_control(hpl_ctx* c) {
+    if (!c->ctl_pending) return HPL_OK;
+    CUDA_TRY(cudaEventRecord(c->ctl_ev, c->ctl_stream));
+    CUDA_TRY(cudaStreamWaitEvent(c->stream, c->ctl_ev, 0));
+    c->ctl_pending = false;
     return HPL_OK;
 }
 
@@ -738,13 +752,17 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
 // ------------------------------------------------------------------------------------------ progress / sync
 int progress(hpl_ctx* c) {
     if (!c->device) return HPL_OK;
+    {
+        int rc = order_main_after_control(c);
+        if (rc != HPL_OK) return rc;
+    }
     if (c->copy_pending && !c->cfg.plan_ahead) {
         // host objects: their chunks become usable once the main stream is ordered after the copies
         CUDA_TRY(cudaEventRecord(c->copy_ev, c->copy_stream));
         CUDA_TRY(cudaStreamWaitEvent(c->stream, c->copy_ev, 0));
         c->copy_pending = false;
         for (auto& kv : c->objects)
-            if (kv.second.from_host) kv.second.landed = published_chunks(c, kv.second);
+            if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
     for (auto& kv : c->bcasts) {
         std::vector<PlannedFanout> tasks;
@@ -781,11 +799,13 @@ void undo_journal(hpl_ctx* c) {
 
 int sync_and_check(hpl_ctx* c) {
     if (!c->device) return HPL_OK;
-    if (c->copy_pending) {
+    if (c->copy_pending || c->ctl_pending) {
+        CUDA_TRY(cudaStreamSynchronize(c->ctl_stream));
         CUDA_TRY(cudaStreamSynchronize(c->copy_stream));
         c->copy_pending = false;
+        c->ctl_pending = false;
         for (auto& kv : c->objects)
-            if (kv.second.from_host) kv.second.landed = published_chunks(c, kv.second);
+            if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
     if (!c->work_in_flight) {
         CUDA_TRY(cudaStreamSynchronize(c->stream));
@@ -891,15 +911,20 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         ok = ok && cudaHostAlloc((void**)&c->h_status, sizeof(DeviceStatus), cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaHostAlloc((void**)&c->h_iota, sizeof(uint32_t) * (kMaxChunks + 1), cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&c->ctl_stream, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->copy_ev, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->ctl_ev, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaMemsetAsync(c->d_dir, 0, sizeof(DirRow) * kMaxRows, c->stream) == cudaSuccess;
         ok = ok && cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus), c->stream) == cudaSuccess;
+        ok = ok && cudaStreamSynchronize(c->stream) == cudaSuccess;   // side streams must not overtake the clearing
         if (!ok) {
             if (c->h_dir) cudaFreeHost(c->h_dir);
             if (c->h_status) cudaFreeHost(c->h_status);
             if (c->h_iota) cudaFreeHost(c->h_iota);
             if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+            if (c->ctl_stream) cudaStreamDestroy(c->ctl_stream);
             if (c->copy_ev) cudaEventDestroy(c->copy_ev);
+            if (c->ctl_ev) cudaEventDestroy(c->ctl_ev);
             delete c;
             return HPL_ERR_CUDA;
         }
@@ -914,6 +939,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
 int hpl_shutdown(hpl_ctx* c) {
     if (!c) return HPL_ERR_INVALID;
     if (c->device) {
+        cudaStreamSynchronize(c->ctl_stream);
         cudaStreamSynchronize(c->copy_stream);
         cudaStreamSynchronize(c->stream);
         collect_kernel_times(c);
@@ -922,7 +948,9 @@ int hpl_shutdown(hpl_ctx* c) {
         cudaFreeHost(c->h_status);
         cudaFreeHost(c->h_iota);
         cudaStreamDestroy(c->copy_stream);
+        cudaStreamDestroy(c->ctl_stream);
         cudaEventDestroy(c->copy_ev);
+        cudaEventDestroy(c->ctl_ev);
     }
     delete c;
     return HPL_OK;
@@ -981,11 +1009,22 @@ int hpl_put(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
     const uint32_t before = published_chunks(c, *o);
     do_put_common(c, *o, bytes, first);
     const uint32_t after = published_chunks(c, *o);
-    if (after != before || first) {
-        rc = publish_counter(c, *o, after, c->stream);
-        if (rc != HPL_OK) return rc;
+    if (c->device && c->cfg.plan_ahead) {
+        // the counter goes out on the control stream, which no polling kernel can hold up; until a wait
+        // confirms it, kernels poll for this object's chunks
+        o->async_counter = true;
+        if (after != before || first) {
+            rc = publish_counter(c, *o, after, c->ctl_stream);
+            if (rc != HPL_OK) return rc;
+            c->ctl_pending = true;
+        }
+    } else {
+        if (after != before || first) {
+            rc = publish_counter(c, *o, after, c->stream);
+            if (rc != HPL_OK) return rc;
+        }
+        o->landed = after;
     }
-    o->landed = after;
     return after_event(c);
 }
 
@@ -1001,6 +1040,7 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
         if (!o->ptr) return HPL_ERR_NOMEM;
         o->lib_owned = true;
         o->from_host = true;
+        o->async_counter = true;
         rc = alloc_row(c, *o);
         if (rc != HPL_OK) {
             c->arena.release(o->ptr);
@@ -1009,7 +1049,8 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
             return rc;
         }
         // the row (pointer) must be in the directory before any copy-stream counter update can matter
-        CUDA_TRY(cudaEventRecord(c->copy_ev, c->stream));
+        cudaStream_t row_stream = c->cfg.plan_ahead ? c->ctl_stream : c->stream;
+        CUDA_TRY(cudaEventRecord(c->copy_ev, row_stream));
         CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
     }
     const uint64_t old_bytes = o->ready_bytes;
@@ -1253,6 +1294,7 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
         if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
     if (c->device) {
         // rows and arena memory are recycled only when nothing enqueued can still read them
+        cudaStreamSynchronize(c->ctl_stream);
         cudaStreamSynchronize(c->copy_stream);
         cudaStreamSynchronize(c->stream);
     }

@@ -1,0 +1,121 @@
+"""Chunks consumed while they are still arriving: host objects copied into the store chunk by chunk,
+kernels that poll the directory's progress counters, and the bound on every such wait."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_05814_b200 as hpl
+from oracle import values as ov
+from oracle.store import DT_F32, DT_BF16
+from tests.harness import Pair, gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2002_05814_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _pinned(a: np.ndarray) -> torch.Tensor:
+    t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a)
+    return t.pin_memory()
+
+
+@pytest.mark.parametrize("plan_ahead", [True, False])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_host_objects_are_copied_in_reduced_and_read_back(plan_ahead, dtype):
+    k, elems, chunk = 8, 300_003 if dtype == "f32" else 300_008, 64 << 10
+    p = Pair(chunk, 2, plan_ahead=plan_ahead, arena_bytes=128 << 20)
+    code = DT_BF16 if dtype == "bf16" else DT_F32
+    host = {}
+    for i in range(k):
+        a = gen(("normal", 0.02), 70, i, elems, dtype)
+        p.host[i] = a
+        host[i] = _pinned(a)
+        p.c.create(i, i, a.nbytes, code)
+        p.o.create(i, i, a.nbytes, code)
+    p.c.reduce(100, list(range(k)), k, 0, code)
+    p.o.reduce(100, list(range(k)), k, 0, code)
+    for i in range(k):
+        half = (a.nbytes // 2) // chunk * chunk
+        p.c.put_host(i, host[i].data_ptr(), half)          # the copy is published in two instalments
+        p.o.put(i, p.host[i], half)
+    if plan_ahead:
+        p.c.progress()                                       # the kernel starts before the objects are complete
+    for i in range(k):
+        p.c.put_host(i, host[i].data_ptr(), p.host[i].nbytes)
+        p.o.put(i, p.host[i], p.host[i].nbytes)
+    out = torch.empty(elems, dtype=torch.float32).pin_memory()
+    p.c.get_host(100, out.data_ptr(), elems * 4)
+    want = p.o.get(100)
+    assert np.array_equal(out.numpy().view(np.uint32), want.view(np.uint32))
+    st = p.c.stats()
+    assert st["h2d_bytes"] == k * p.host[0].nbytes and st["d2h_bytes"] == elems * 4 and st["device_timeouts"] == 0
+    p.check_schedule(100)
+    p.close()
+
+
+def test_host_source_is_broadcast_while_it_is_copied_in():
+    nbytes, R = 3 << 20, 6
+    p = Pair(256 << 10, 2, 2, plan_ahead=True, arena_bytes=64 << 20)
+    a = gen(("uniform",), 71, 0, nbytes // 4)
+    p.host[0] = a
+    pin = _pinned(a)
+    p.c.create(0, 99, nbytes, DT_F32)
+    p.o.create(0, 99, nbytes, DT_F32)
+    for j in range(1, R + 1):
+        p.create(j, j, nbytes=nbytes, dtype=DT_F32)
+    p.broadcast(0, list(range(1, R + 1)))
+    p.c.put_host(0, pin.data_ptr(), 1 << 20)
+    p.o.put(0, a, 1 << 20)
+    for j in range(1, R + 1):
+        p.join(j)
+    p.c.progress()
+    p.c.put_host(0, pin.data_ptr(), nbytes)
+    p.o.put(0, a, nbytes)
+    for j in range(1, R + 1):
+        p.check_receiver_bytes(j)
+    assert p.c.stats()["device_timeouts"] == 0
+    p.close()
+
+
+def test_polling_kernel_picks_up_chunks_published_while_it_runs():
+    k, elems, chunk = 4, 64 * 4096, 16 << 10                 # 16 chunks
+    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=5_000_000_000)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 72, i, elems))
+    p.reduce(100, list(range(k)), k)
+    for i in range(k):
+        p.put(i, 4 * chunk)                                  # a quarter of every object
+    p.progress()                                             # planned for all 16 chunks: the kernel now waits at chunk 4
+    for step in (8, 12, 16):
+        for i in range(k):
+            p.put(i, step * chunk)                           # counters travel on the control stream
+    p.check_target_bits(100)
+    st = p.c.stats()
+    assert st["device_timeouts"] == 0 and st["kernel_launches"] == 1
+    p.close()
+
+
+def test_a_wait_nothing_ends_runs_out_and_the_context_stays_usable():
+    k, elems, chunk = 3, 10 * 4096, 16 << 10
+    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=3_000_000)    # 3 ms
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 73, i, elems))
+    p.reduce(100, list(range(k)), k)
+    p.put(0)
+    p.put(1)
+    p.put(2, 2 * chunk)                                      # object 2 stops at chunk 2 and nothing advances it
+    rc, _, _ = p.c.try_get(100)
+    assert rc == hpl.HPL_ERR_TIMEOUT                          # the host already knows the target cannot complete
+    assert p.c.sync() == hpl.HPL_ERR_TIMEOUT                  # ... and the kernel's bounded wait has run out
+    assert p.c.stats()["device_timeouts"] == 1
+    x = torch.ones(1024, device="cuda")                       # the device is fine
+    assert float(x.sum()) == 1024.0
+    p.put(2)                                                  # the rest arrives: everything is planned again
+    p.check_target_bits(100)
+    assert p.c.sync() == hpl.HPL_OK
+    p.close()
