@@ -127,7 +127,7 @@ class Runner:
         n_src = w.n_objects
         arena_bytes = 64 * MiB + 2 * w.elems * 4 + (n_src + 2) * S * (1 if host_buffers else 0)
         if w.kind == "ft_reduce":
-            arena_bytes += 4 * w.elems * 4
+            arena_bytes += 8 * w.elems * 4       # partial results of the subtrees beside the failing worker's root path
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
         self.ctx = hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=arena_bytes,
                                stream=torch.cuda.current_stream().cuda_stream, time_kernels=True,
