@@ -83,7 +83,7 @@ def test_host_source_is_broadcast_while_it_is_copied_in():
 
 
 def test_polling_kernel_picks_up_chunks_published_while_it_runs():
-    k, elems, chunk = 4, 64 * 4096, 16 << 10                 # 16 chunks
+    k, elems, chunk = 4, 16 * 4096, 16 << 10                 # 16 chunks of 4096 elements
     p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=5_000_000_000)
     for i in range(k):
         p.create(i, i, gen(("uniform",), 72, i, elems))
