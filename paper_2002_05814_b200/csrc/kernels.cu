@@ -11,8 +11,8 @@
 //      task (Section 3.4.1: the receivers of one sender subtree), same polling.
 //
 // Global reads are 16 bytes per thread, coalesced and L2-only (.cg) because every byte is used once.
-// The reduce kernel stages its operand tiles through shared memory with cp.async, three steps ahead
-// of the adds, so that about 48 KiB per CTA are in flight without holding registers.
+// The reduce kernel stages its operand tiles through shared memory with cp.async, several steps ahead
+// of the adds, so that 80 KiB and more per SM are in flight without holding registers.
 #include <cuda_runtime.h>
 
 #include "device_types.h"
@@ -67,9 +67,16 @@ __device__ __forceinline__ float combine(float a, float b, unsigned int red_op) 
 //   F32 task:  vector j (of 4) of thread t holds elements (j*256 + t)*4 .. +3 of the tile.
 //   BF16 task: group j (of 2) of thread t holds elements (j*256 + t)*8 .. +7: one vector for a bf16
 //              operand, two (slots 2j, 2j+1) for an fp32 operand (a materialised partial result).
-constexpr int kStages = 4;
+// Stage count per kernel variant: with up to 4 accumulators two CTAs share an SM (6 stages each, 5 steps =
+// 40-80 KiB per CTA in flight); the 8-accumulator variant needs the whole register file of an SM for one
+// CTA and gets 12 stages instead.
 constexpr int kStageBytes = 4 * kReduceThreads * 16;
-constexpr int kReduceSmemBytes = kStages * kStageBytes;
+template <int A>
+struct StagesFor {
+    static constexpr int value = A <= 4 ? 6 : 12;
+    static constexpr int min_ctas = A <= 4 ? 2 : 1;
+    static constexpr int smem_bytes = value * kStageBytes;
+};
 
 __device__ __forceinline__ void cp_async16(unsigned int smem_addr, const void* gptr, unsigned int src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(src_bytes) : "memory");
@@ -80,7 +87,7 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <bool BF16>
+template <bool BF16, int kStages>
 struct TileCtx {
     const ReduceStep* steps;
     const unsigned long long* s_ptr;   // operand base addresses of the task's steps (shared memory)
@@ -178,7 +185,7 @@ struct TileCtx {
 // a shallower accumulator.  A step into L+1 opens a fused child subtree: one more level of this
 // function, whose accumulator is a separate set of registers, closed by ADD_ACC(L, L+1).
 template <int L, int A, bool BF16>
-__device__ __forceinline__ void eval_level(TileCtx<BF16>& cx, float (&acc)[16]) {
+__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& cx, float (&acc)[16]) {
     while (cx.pc < cx.n) {
         const ReduceStep st = cx.steps[cx.pc];
         if (L > 0 && (int)st.a < L) return;
@@ -207,7 +214,8 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16>& cx, float (&acc)[16]) 
 }
 
 template <int A, bool BF16>
-__global__ void __launch_bounds__(kReduceThreads) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
+__global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
+    constexpr int kStages = StagesFor<A>::value;
     extern __shared__ __align__(16) unsigned char s_stage[];
     __shared__ unsigned long long s_ptr[kMaxStepsPerWave];
     const unsigned int t = threadIdx.x;
@@ -246,7 +254,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_wave_kernel(const __gri
             if (!__syncthreads_and(ok)) return;
         }
 
-        TileCtx<BF16> cx;
+        TileCtx<BF16, kStages> cx;
         cx.steps = &w.steps[task.step_begin];
         cx.s_ptr = s_ptr;
         cx.smem_base = (unsigned int)__cvta_generic_to_shared(s_stage);
@@ -345,11 +353,11 @@ template <int A, bool BF16>
 static int launch_reduce_t(const ReduceWave& w, int grid, cudaStream_t s) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kReduceSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, StagesFor<A>::smem_bytes);
         if (e != cudaSuccess) return (int)e;
         attr_set = true;
     }
-    reduce_wave_kernel<A, BF16><<<grid, kReduceThreads, kReduceSmemBytes, s>>>(w);
+    reduce_wave_kernel<A, BF16><<<grid, kReduceThreads, StagesFor<A>::smem_bytes, s>>>(w);
     return (int)cudaGetLastError();
 }
 
@@ -368,8 +376,8 @@ int launch_fanout_wave(const FanoutWave& w, int grid, void* stream) {
 template <int A, bool BF16>
 static int occ_t() {
     int n = 0;
-    if (cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kReduceSmemBytes) != cudaSuccess) return 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reduce_wave_kernel<A, BF16>, kReduceThreads, kReduceSmemBytes) != cudaSuccess) return 1;
+    if (cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, StagesFor<A>::smem_bytes) != cudaSuccess) return 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reduce_wave_kernel<A, BF16>, kReduceThreads, StagesFor<A>::smem_bytes) != cudaSuccess) return 1;
     return n < 1 ? 1 : n;
 }
 
