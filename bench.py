@@ -350,6 +350,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--size", type=int, default=64 * MiB, help="object bytes for cfg5")
+    ap.add_argument("--shrink", type=int, default=1, help="divide the object size by this (profiling captures on a smaller case)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads measured briefly and reported under 'also'")
@@ -359,12 +360,16 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     w = wl.cfg5_at(args.size) if args.workload == "cfg5" else wl.workload(args.workload)
+    if args.shrink > 1:
+        w.elems = max(8, w.elems // args.shrink // 8 * 8)
     ab = algorithmic_bytes(w)
     step_bytes = ab["reduce"] + ab["broadcast"]
     name = {"cfg1": "cfg1 reduce 8 x 1 MiB fp32", "cfg2": "cfg2 broadcast 64 MiB fp32 to 16 receivers",
             "cfg3": "cfg3 async-SGD reduce, first 8 of 16 x 97.5 MiB fp32",
             "cfg4": "cfg4 policy round: broadcast 64 MiB bf16 to 64 receivers + fp32 sum of 64 x 64 MiB bf16",
             "cfg5": f"cfg5 fault-tolerant reduce of 32 x {args.size} B fp32, worker 7 fails at 40%"}[w.name]
+    if args.shrink > 1:
+        name += f" [objects shrunk {args.shrink}x]"
     config = {"workload": name, "chunk_bytes": w.chunk_bytes, "degree": w.degree, "object_bytes": w.object_bytes,
               "algorithmic_bytes_per_step": step_bytes, "l2": "inputs larger than L2 (no flush)",
               "timed_region": "first Put of the step to the last Get, CUDA events on the library's stream; Delete outside"}
