@@ -452,7 +452,7 @@ def main():
 
     if rank == 0 and world == 1 and args.also:
         also = {}
-        for nm in [x for x in args.also.split(",") if x and x != w.name]:
+        for nm in [x for x in args.also.split(",") if x and x != "none" and x != w.name]:
             ww = wl.workload(nm)
             rr = Runner(ww, device)
             r2 = time_steps(rr, 5, 3)
