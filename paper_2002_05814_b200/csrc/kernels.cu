@@ -61,9 +61,9 @@ __device__ __forceinline__ float combine(float a, float b, unsigned int red_op) 
 }
 
 // ---- staging.  Every load step of a task is brought from global memory to shared memory with
-// cp.async (16 bytes per instruction, L2 only), kStages steps ahead of its use.  A thread only ever
+// cp.async (16 bytes per instruction, L2 only), several steps ahead of its use.  A thread only ever
 // reads back the bytes it copied itself, so no barrier is needed: cp.async.wait_group orders them.
-// Shared layout: [stage][vector j][thread] of 16-byte vectors (conflict free).
+// Shared layout of one stage: [vector j][thread] of 16-byte vectors (conflict free).
 //   F32 task:  vector j (of 4) of thread t holds elements (j*256 + t)*4 .. +3 of the tile.
 //   BF16 task: group j (of 2) of thread t holds elements (j*256 + t)*8 .. +7: one vector for a bf16
 //              operand, two (slots 2j, 2j+1) for an fp32 operand (a materialised partial result).
@@ -71,6 +71,7 @@ __device__ __forceinline__ float combine(float a, float b, unsigned int red_op) 
 // 40-80 KiB per CTA in flight); the 8-accumulator variant needs the whole register file of an SM for one
 // CTA and gets 12 stages instead.
 constexpr int kStageBytes = 4 * kReduceThreads * 16;
+constexpr int kVecStride = kReduceThreads * 16;   // bytes between a thread's consecutive vectors, in shared and (mostly) global
 template <int A>
 struct StagesFor {
     static constexpr int value = A <= 4 ? 6 : 12;
@@ -78,105 +79,162 @@ struct StagesFor {
     static constexpr int smem_bytes = value * kStageBytes;
 };
 
-__device__ __forceinline__ void cp_async16(unsigned int smem_addr, const void* gptr, unsigned int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(src_bytes) : "memory");
+// A step as the kernel keeps it in shared memory: operand base address in the low 56 bits, and on top
+// code (2 bits), accumulator (3 bits), operand kind (1 bit).
+constexpr int kRecShift = 56;
+__device__ __forceinline__ unsigned long long make_rec(const ReduceStep st, unsigned long long ptr) {
+    const unsigned long long meta = (unsigned long long)st.code | ((unsigned long long)st.a << 2) | ((unsigned long long)st.kind << 5);
+    return (ptr & ((1ull << kRecShift) - 1)) | (meta << kRecShift);
+}
+__device__ __forceinline__ unsigned int rec_meta(unsigned long long rec) { return (unsigned int)(rec >> kRecShift); }
+__device__ __forceinline__ unsigned int meta_code(unsigned int m) { return m & 3u; }
+__device__ __forceinline__ unsigned int meta_acc(unsigned int m) { return (m >> 2) & 7u; }
+__device__ __forceinline__ bool meta_is_bf16(unsigned int m) { return (m & 32u) != 0; }
+
+__device__ __forceinline__ void cp_async16(unsigned int smem_addr, unsigned long long gaddr) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gaddr) : "memory");
+}
+__device__ __forceinline__ void cp_async16_partial(unsigned int smem_addr, unsigned long long gaddr, unsigned int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gaddr), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
+__device__ __forceinline__ unsigned long long ld_shared_u64(unsigned int addr) {
+    unsigned long long v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr));
+    return v;
+}
 
-template <bool BF16, int kStages>
+// Sixteen fp32 values of a thread as eight register pairs, so that sums can use the packed fp32 add of
+// sm_100 (two IEEE round-to-nearest adds per instruction; same bits as two scalar adds).
+struct Acc {
+    unsigned long long p[8];
+};
+__device__ __forceinline__ unsigned long long pack2(unsigned int lo, unsigned int hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, unsigned int& lo, unsigned int& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ void combine_acc(Acc& a, const Acc& x, unsigned int red_op) {
+    if (red_op == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a.p[i] = add2(a.p[i], x.p[i]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            unsigned int al, ah, xl, xh;
+            unpack2(a.p[i], al, ah);
+            unpack2(x.p[i], xl, xh);
+            const float l = combine(__uint_as_float(al), __uint_as_float(xl), red_op);
+            const float h = combine(__uint_as_float(ah), __uint_as_float(xh), red_op);
+            a.p[i] = pack2(__float_as_uint(l), __float_as_uint(h));
+        }
+    }
+}
+
+template <bool BF16, int kStages, bool FULL>
 struct TileCtx {
-    const ReduceStep* steps;
-    const unsigned long long* s_ptr;   // operand base addresses of the task's steps (shared memory)
-    unsigned int smem_base;            // shared-window address of the staging area
-    unsigned int n, pc, red_op, t;
-    unsigned long long e0;             // first element of the tile
-    unsigned int count;                // elements in the tile
+    unsigned int rec_base;             // shared-window address of the step records
+    unsigned int n, pc, red_op;
+    unsigned int issue_idx;            // next step whose copy is to be started
+    unsigned int issue_stage, cons_stage, stage_lo, stage_end;   // this thread's slot in the stage ring
+    unsigned long long goff_main;      // byte offset of this thread's first vector for the wave's source dtype
+    unsigned long long goff_f32;       // (BF16 waves) the same for an fp32 operand
+    unsigned int count, t;             // ragged tiles: elements in the tile, thread index
 
-    // bytes of a 16-byte vector starting at element `off` of the tile that lie inside it
-    __device__ __forceinline__ unsigned int in_bounds_bytes(unsigned int off, unsigned int elem_bytes, unsigned int per_vec) const {
-        if (off >= count) return 0u;
-        const unsigned int left = count - off;
-        return (left >= per_vec ? per_vec : left) * elem_bytes;
+    // ragged tiles: bytes of a 16-byte vector starting at element `off` of the tile that lie inside it
+    __device__ __forceinline__ unsigned int inside(unsigned int off, unsigned int per_vec, unsigned int elem_bytes) const {
+        const unsigned int left = off < count ? count - off : 0u;
+        return (left < per_vec ? left : per_vec) * elem_bytes;
     }
 
-    __device__ __forceinline__ void issue(unsigned int i) {
-        if (i < n) {
-            const ReduceStep st = steps[i];
-            if (st.code != OPC_ADD_ACC) {
-                const unsigned int stage = smem_base + (i % kStages) * kStageBytes;
-                const unsigned long long base = s_ptr[i];
-                if (!BF16) {
+    __device__ __forceinline__ void advance(unsigned int& stage) {
+        stage += kStageBytes;
+        if (stage == stage_end) stage = stage_lo;
+    }
+
+    __device__ __forceinline__ void issue() {
+        if (issue_idx < n) {
+            const unsigned long long rec = ld_shared_u64(rec_base + issue_idx * 8);
+            const unsigned int m = rec_meta(rec);
+            if (meta_code(m) != OPC_ADD_ACC) {
+                const unsigned long long ptr = rec & ((1ull << kRecShift) - 1);
+                if (!BF16 || meta_is_bf16(m)) {
+                    const unsigned long long g = ptr + goff_main;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const unsigned int off = (j * kReduceThreads + t) * 4;
-                        const unsigned int nb = in_bounds_bytes(off, 4, 4);
-                        const float* g = reinterpret_cast<const float*>(base) + (nb ? e0 + off : 0ull);
-                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
-                    }
-                } else if (st.kind == SRC_BF16) {
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const unsigned int off = (j * kReduceThreads + t) * 8;
-                        const unsigned int nb = in_bounds_bytes(off, 2, 8);
-                        const unsigned short* g = reinterpret_cast<const unsigned short*>(base) + (nb ? e0 + off : 0ull);
-                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
+                    for (int j = 0; j < (BF16 ? 2 : 4); ++j) {
+                        if (FULL) {
+                            cp_async16(issue_stage + j * kVecStride, g + j * kVecStride);
+                        } else {
+                            const unsigned int nb = BF16 ? inside((j * kReduceThreads + t) * 8, 8, 2) : inside((j * kReduceThreads + t) * 4, 4, 4);
+                            cp_async16_partial(issue_stage + j * kVecStride, nb ? g + j * kVecStride : ptr, nb);
+                        }
                     }
                 } else {
+                    const unsigned long long g = ptr + goff_f32;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const unsigned int off = ((j >> 1) * kReduceThreads + t) * 8 + (j & 1) * 4;
-                        const unsigned int nb = in_bounds_bytes(off, 4, 4);
-                        const float* g = reinterpret_cast<const float*>(base) + (nb ? e0 + off : 0ull);
-                        cp_async16(stage + (j * kReduceThreads + t) * 16, g, nb);
+                        const unsigned int go = (j >> 1) * (2 * kVecStride) + (j & 1) * 16;
+                        if (FULL) {
+                            cp_async16(issue_stage + j * kVecStride, g + go);
+                        } else {
+                            const unsigned int nb = inside(((j >> 1) * kReduceThreads + t) * 8 + (j & 1) * 4, 4, 4);
+                            cp_async16_partial(issue_stage + j * kVecStride, nb ? g + go : ptr, nb);
+                        }
                     }
                 }
             }
         }
         cp_async_commit();  // one group per step, empty or not, keeps the group count equal to the step count
+        ++issue_idx;
+        advance(issue_stage);
     }
 
     // Consumes step pc: starts the copy kStages-1 steps ahead, waits for this step's bytes, widens to fp32.
-    __device__ __forceinline__ void fetch(const ReduceStep st, float (&x)[16]) {
-        issue(pc + kStages - 1);
+    __device__ __forceinline__ void fetch(unsigned int m, Acc& x) {
+        issue();
         cp_async_wait<kStages - 1>();
-        const unsigned int stage = smem_base + (pc % kStages) * kStageBytes;
         uint4 v[4];
-        const int nv = (BF16 && st.kind == SRC_BF16) ? 2 : 4;
+        const bool half = BF16 && meta_is_bf16(m);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (j < nv) {
-                const unsigned int a = stage + (j * kReduceThreads + t) * 16;
+            if (j < 2 || !BF16 || !half) {
+                const unsigned int a = cons_stage + j * kVecStride;
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w) : "r"(a));
             }
         }
-        if (!BF16 || st.kind == SRC_F32) {
+        if (!half) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                x[j * 4 + 0] = __uint_as_float(v[j].x);
-                x[j * 4 + 1] = __uint_as_float(v[j].y);
-                x[j * 4 + 2] = __uint_as_float(v[j].z);
-                x[j * 4 + 3] = __uint_as_float(v[j].w);
+                x.p[j * 2 + 0] = pack2(v[j].x, v[j].y);
+                x.p[j * 2 + 1] = pack2(v[j].z, v[j].w);
             }
         } else {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const unsigned int w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    x[j * 8 + i * 2 + 0] = __uint_as_float(w[i] << 16);  // widening bf16 -> fp32 is exact
-                    x[j * 8 + i * 2 + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-                }
+                for (int i = 0; i < 4; ++i) x.p[j * 4 + i] = pack2(w[i] << 16, w[i] & 0xFFFF0000u);  // bf16 -> fp32 is exact
             }
         }
+        advance(cons_stage);
         ++pc;
     }
 
     __device__ __forceinline__ void skip() {  // an ADD_ACC step: no bytes, but its (empty) group is counted
-        issue(pc + kStages - 1);
+        issue();
+        advance(cons_stage);
         ++pc;
     }
 };
@@ -184,28 +242,27 @@ struct TileCtx {
 // Runs the steps that belong to accumulator L, starting at a LOAD into L, until a step that belongs to
 // a shallower accumulator.  A step into L+1 opens a fused child subtree: one more level of this
 // function, whose accumulator is a separate set of registers, closed by ADD_ACC(L, L+1).
-template <int L, int A, bool BF16>
-__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& cx, float (&acc)[16]) {
+template <int L, int A, bool BF16, bool FULL>
+__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value, FULL>& cx, Acc& acc) {
     while (cx.pc < cx.n) {
-        const ReduceStep st = cx.steps[cx.pc];
-        if (L > 0 && (int)st.a < L) return;
-        if (st.a == L) {
-            float x[16];
-            cx.fetch(st, x);
-            if (st.code == OPC_LOAD) {
+        const unsigned int m = rec_meta(ld_shared_u64(cx.rec_base + cx.pc * 8));
+        const unsigned int a = meta_acc(m);
+        if (L > 0 && (int)a < L) return;
+        if ((int)a == L) {
+            Acc x;
+            cx.fetch(m, x);
+            if (meta_code(m) == OPC_LOAD) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) acc[i] = x[i];
+                for (int i = 0; i < 8; ++i) acc.p[i] = x.p[i];
             } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) acc[i] = combine(acc[i], x[i], cx.red_op);
+                combine_acc(acc, x, cx.red_op);
             }
         } else {
             if constexpr (L + 1 < A) {
-                float sub[16];
-                eval_level<L + 1, A, BF16>(cx, sub);
+                Acc sub;
+                eval_level<L + 1, A, BF16, FULL>(cx, sub);
                 cx.skip();  // the ADD_ACC(L, L+1) that closes the subtree
-#pragma unroll
-                for (int i = 0; i < 16; ++i) acc[i] = combine(acc[i], sub[i], cx.red_op);
+                combine_acc(acc, sub, cx.red_op);
             } else {
                 cx.skip();  // unreachable for a well-formed task (the planner bounds the depth by A)
             }
@@ -213,13 +270,59 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& c
     }
 }
 
+template <int A, bool BF16, bool FULL>
+__device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int stage_base, const ReduceTask& task, unsigned long long e0,
+                                         unsigned int count, unsigned int t) {
+    constexpr int kStages = StagesFor<A>::value;
+    TileCtx<BF16, kStages, FULL> cx;
+    cx.rec_base = rec_base;
+    cx.n = task.n_steps;
+    cx.pc = 0;
+    cx.red_op = task.red_op;
+    cx.issue_idx = 0;
+    cx.stage_lo = stage_base + t * 16;
+    cx.stage_end = cx.stage_lo + kStages * kStageBytes;
+    cx.issue_stage = cx.cons_stage = cx.stage_lo;
+    if (!BF16) {
+        cx.goff_main = e0 * 4ull + t * 16ull;
+        cx.goff_f32 = cx.goff_main;
+    } else {
+        cx.goff_main = e0 * 2ull + t * 16ull;
+        cx.goff_f32 = e0 * 4ull + t * 32ull;
+    }
+    cx.count = count;
+    cx.t = t;
+#pragma unroll
+    for (int i = 0; i < kStages - 1; ++i) cx.issue();
+
+    Acc acc;
+    eval_level<0, A, BF16, FULL>(cx, acc);
+    cp_async_wait<0>();
+
+    float* out = reinterpret_cast<float*>(task.out_ptr) + e0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const unsigned int off = BF16 ? ((q >> 1) * kReduceThreads + t) * 8 + (q & 1) * 4 : (q * kReduceThreads + t) * 4;
+        unsigned int r[4];
+        unpack2(acc.p[q * 2 + 0], r[0], r[1]);
+        unpack2(acc.p[q * 2 + 1], r[2], r[3]);
+        if (FULL || off + 4 <= count) {
+            *reinterpret_cast<uint4*>(out + off) = make_uint4(r[0], r[1], r[2], r[3]);
+        } else {
+            for (int i = 0; i < 4; ++i)
+                if (off + i < count) out[off + i] = __uint_as_float(r[i]);
+        }
+    }
+}
+
 template <int A, bool BF16>
 __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
-    constexpr int kStages = StagesFor<A>::value;
     extern __shared__ __align__(16) unsigned char s_stage[];
-    __shared__ unsigned long long s_ptr[kMaxStepsPerWave];
+    __shared__ unsigned long long s_rec[kMaxStepsPerWave];
     const unsigned int t = threadIdx.x;
     const unsigned long long t_start = global_timer_ns();
+    const unsigned int rec_base = (unsigned int)__cvta_generic_to_shared(s_rec);
+    const unsigned int stage_base = (unsigned int)__cvta_generic_to_shared(s_stage);
     int cached_task = -1;
 
     for (unsigned int g = blockIdx.x; g < w.total_tiles; g += gridDim.x) {
@@ -227,10 +330,10 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
         while (ti + 1 < (int)w.n_tasks && g >= w.tasks[ti + 1].tile_begin) ++ti;
         const ReduceTask& task = w.tasks[ti];
         if (ti != cached_task) {
-            __syncthreads();  // everyone is done with the previous task's pointers
+            __syncthreads();  // everyone is done with the previous task's records
             for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
                 const ReduceStep st = w.steps[task.step_begin + i];
-                s_ptr[i] = st.code == OPC_ADD_ACC ? 0ull : w.dir[st.row].ptr;
+                s_rec[i] = make_rec(st, st.code == OPC_ADD_ACC ? 0ull : w.dir[st.row].ptr);
             }
             cached_task = ti;
             __syncthreads();
@@ -254,35 +357,11 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
             if (!__syncthreads_and(ok)) return;
         }
 
-        TileCtx<BF16, kStages> cx;
-        cx.steps = &w.steps[task.step_begin];
-        cx.s_ptr = s_ptr;
-        cx.smem_base = (unsigned int)__cvta_generic_to_shared(s_stage);
-        cx.n = task.n_steps;
-        cx.pc = 0;
-        cx.red_op = task.red_op;
-        cx.t = t;
-        cx.e0 = e0;
-        cx.count = (unsigned int)(e1 - e0);
-#pragma unroll
-        for (int i = 0; i < kStages - 1; ++i) cx.issue(i);
-
-        float acc[16];
-        eval_level<0, A, BF16>(cx, acc);
-        cp_async_wait<0>();
-
-        float* out = reinterpret_cast<float*>(task.out_ptr) + e0;
-        const unsigned int count = cx.count;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const unsigned int off = BF16 ? ((q >> 1) * kReduceThreads + t) * 8 + (q & 1) * 4 : (q * kReduceThreads + t) * 4;
-            if (off + 4 <= count) {
-                *reinterpret_cast<float4*>(out + off) = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
-            } else {
-                for (int i = 0; i < 4; ++i)
-                    if (off + i < count) out[off + i] = acc[q * 4 + i];
-            }
-        }
+        const unsigned int count = (unsigned int)(e1 - e0);
+        if (count == kTileElems)
+            run_tile<A, BF16, true>(rec_base, stage_base, task, e0, count, t);
+        else
+            run_tile<A, BF16, false>(rec_base, stage_base, task, e0, count, t);
     }
 }
 
