@@ -143,7 +143,7 @@ __device__ __forceinline__ void combine_acc(Acc& a, const Acc& x, unsigned int r
     }
 }
 
-template <bool BF16, int kStages, bool FULL>
+template <bool BF16, int kStages>
 struct TileCtx {
     unsigned int rec_base;             // shared-window address of the step records
     unsigned int n, pc, red_op;
@@ -151,9 +151,10 @@ struct TileCtx {
     unsigned int issue_stage, cons_stage, stage_lo, stage_end;   // this thread's slot in the stage ring
     unsigned long long goff_main;      // byte offset of this thread's first vector for the wave's source dtype
     unsigned long long goff_f32;       // (BF16 waves) the same for an fp32 operand
-    unsigned int count, t;             // ragged tiles: elements in the tile, thread index
+    unsigned int count, t;             // elements in the tile, thread index
+    unsigned int nb_main[BF16 ? 2 : 4];  // bytes of each of this thread's vectors that lie inside the tile (16 unless ragged)
 
-    // ragged tiles: bytes of a 16-byte vector starting at element `off` of the tile that lie inside it
+    // bytes of a 16-byte vector starting at element `off` of the tile that lie inside it
     __device__ __forceinline__ unsigned int inside(unsigned int off, unsigned int per_vec, unsigned int elem_bytes) const {
         const unsigned int left = off < count ? count - off : 0u;
         return (left < per_vec ? left : per_vec) * elem_bytes;
@@ -174,24 +175,16 @@ struct TileCtx {
                     const unsigned long long g = ptr + goff_main;
 #pragma unroll
                     for (int j = 0; j < (BF16 ? 2 : 4); ++j) {
-                        if (FULL) {
-                            cp_async16(issue_stage + j * kVecStride, g + j * kVecStride);
-                        } else {
-                            const unsigned int nb = BF16 ? inside((j * kReduceThreads + t) * 8, 8, 2) : inside((j * kReduceThreads + t) * 4, 4, 4);
-                            cp_async16_partial(issue_stage + j * kVecStride, nb ? g + j * kVecStride : ptr, nb);
-                        }
+                        // a vector that lies (partly) beyond the tile copies fewer bytes, or none, and is zero-filled
+                        cp_async16_partial(issue_stage + j * kVecStride, g + j * kVecStride, nb_main[j]);
                     }
                 } else {
                     const unsigned long long g = ptr + goff_f32;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const unsigned int go = (j >> 1) * (2 * kVecStride) + (j & 1) * 16;
-                        if (FULL) {
-                            cp_async16(issue_stage + j * kVecStride, g + go);
-                        } else {
-                            const unsigned int nb = inside(((j >> 1) * kReduceThreads + t) * 8 + (j & 1) * 4, 4, 4);
-                            cp_async16_partial(issue_stage + j * kVecStride, nb ? g + go : ptr, nb);
-                        }
+                        const unsigned int nb = inside(((j >> 1) * kReduceThreads + t) * 8 + (j & 1) * 4, 4, 4);
+                        cp_async16_partial(issue_stage + j * kVecStride, g + go, nb);
                     }
                 }
             }
@@ -242,8 +235,8 @@ struct TileCtx {
 // Runs the steps that belong to accumulator L, starting at a LOAD into L, until a step that belongs to
 // a shallower accumulator.  A step into L+1 opens a fused child subtree: one more level of this
 // function, whose accumulator is a separate set of registers, closed by ADD_ACC(L, L+1).
-template <int L, int A, bool BF16, bool FULL>
-__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value, FULL>& cx, Acc& acc) {
+template <int L, int A, bool BF16>
+__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& cx, Acc& acc) {
     while (cx.pc < cx.n) {
         const unsigned int m = rec_meta(ld_shared_u64(cx.rec_base + cx.pc * 8));
         const unsigned int a = meta_acc(m);
@@ -260,7 +253,7 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value, FU
         } else {
             if constexpr (L + 1 < A) {
                 Acc sub;
-                eval_level<L + 1, A, BF16, FULL>(cx, sub);
+                eval_level<L + 1, A, BF16>(cx, sub);
                 cx.skip();  // the ADD_ACC(L, L+1) that closes the subtree
                 combine_acc(acc, sub, cx.red_op);
             } else {
@@ -270,11 +263,11 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value, FU
     }
 }
 
-template <int A, bool BF16, bool FULL>
+template <int A, bool BF16>
 __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int stage_base, const ReduceTask& task, unsigned long long e0,
                                          unsigned int count, unsigned int t) {
     constexpr int kStages = StagesFor<A>::value;
-    TileCtx<BF16, kStages, FULL> cx;
+    TileCtx<BF16, kStages> cx;
     cx.rec_base = rec_base;
     cx.n = task.n_steps;
     cx.pc = 0;
@@ -293,10 +286,13 @@ __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int sta
     cx.count = count;
     cx.t = t;
 #pragma unroll
+    for (int j = 0; j < (BF16 ? 2 : 4); ++j)
+        cx.nb_main[j] = BF16 ? cx.inside((j * kReduceThreads + t) * 8, 8, 2) : cx.inside((j * kReduceThreads + t) * 4, 4, 4);
+#pragma unroll
     for (int i = 0; i < kStages - 1; ++i) cx.issue();
 
     Acc acc;
-    eval_level<0, A, BF16, FULL>(cx, acc);
+    eval_level<0, A, BF16>(cx, acc);
     cp_async_wait<0>();
 
     float* out = reinterpret_cast<float*>(task.out_ptr) + e0;
@@ -306,7 +302,7 @@ __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int sta
         unsigned int r[4];
         unpack2(acc.p[q * 2 + 0], r[0], r[1]);
         unpack2(acc.p[q * 2 + 1], r[2], r[3]);
-        if (FULL || off + 4 <= count) {
+        if (off + 4 <= count) {
             *reinterpret_cast<uint4*>(out + off) = make_uint4(r[0], r[1], r[2], r[3]);
         } else {
             for (int i = 0; i < 4; ++i)
@@ -358,10 +354,7 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
         }
 
         const unsigned int count = (unsigned int)(e1 - e0);
-        if (count == kTileElems)
-            run_tile<A, BF16, true>(rec_base, stage_base, task, e0, count, t);
-        else
-            run_tile<A, BF16, false>(rec_base, stage_base, task, e0, count, t);
+        run_tile<A, BF16>(rec_base, stage_base, task, e0, count, t);
     }
 }
 
