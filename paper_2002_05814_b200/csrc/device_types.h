@@ -30,7 +30,7 @@ struct DeviceStatus {
 constexpr int kTileElems = 4096;        // elements of the reduce output per tile (one CTA iteration)
 constexpr int kReduceThreads = 256;
 constexpr int kMaxAcc = 8;              // accumulators (tree depth that can be fused in registers)
-constexpr int kFanoutTileBytes = 16384;
+constexpr int kFanoutTileBytes = 32768;
 constexpr int kFanoutThreads = 256;
 
 enum : uint8_t { OPC_LOAD = 0, OPC_ADD_LOAD = 1, OPC_ADD_ACC = 2 };

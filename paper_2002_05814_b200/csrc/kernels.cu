@@ -7,8 +7,8 @@
 //      contraction, no fast-math.  Before a chunk is touched the progress counters of its operands
 //      are polled in the device directory (bounded wait), which is how a chunk that is still being
 //      copied into the store is consumed as soon as it lands (Section 3.3).
-//  fanout_wave_kernel  -- reads each tile of a chunk once and stores it to every receiver of the
-//      task (Section 3.4.1: the receivers of one sender subtree), same polling.
+//  fanout_wave_kernel  -- reads each tile of a chunk once into shared memory and writes it to every
+//      receiver of the task with bulk copies (Section 3.4.1: the receivers of one sender subtree), same polling.
 //
 // Global reads are 16 bytes per thread, coalesced and L2-only (.cg) because every byte is used once.
 // The reduce kernel stages its operand tiles through shared memory with cp.async, several steps ahead
@@ -359,12 +359,26 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
 }
 
 // ------------------------------------------------------------------------------------------ fan-out
+// A tile is loaded once (16-byte loads, L2 only) into one of two shared-memory buffers and then written to
+// every receiver with one bulk copy per receiver (shared -> global, cp.async.bulk, issued by the first 64
+// threads): large contiguous writes reach a higher HBM write rate than per-thread stores, and the next
+// tile's load overlaps the draining stores.  The only waits are on the CTA's own bulk copies
+// (cp.async.bulk.wait_group), which always complete.
+constexpr int kFanoutIssuers = 64;
+constexpr int kFanoutSmemBytes = 2 * kFanoutTileBytes;
+
+__device__ __forceinline__ void bulk_store(unsigned long long gdst, unsigned int smem_src, unsigned int bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
+}
+
 __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __grid_constant__ FanoutWave w) {
+    extern __shared__ __align__(128) unsigned char s_tile[];
     __shared__ unsigned long long s_dst[kMaxFanoutDst];
     __shared__ unsigned long long s_src;
     const unsigned int t = threadIdx.x;
     const unsigned long long t_start = global_timer_ns();
     int cached_task = -1;
+    unsigned int buf = 0;
 
     for (unsigned int g = blockIdx.x; g < w.total_tiles; g += gridDim.x) {
         int ti = 0;
@@ -390,34 +404,48 @@ __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __gri
         if (task.poll) {
             int ok = 1;
             if (t == 0) ok = wait_chunk(w.dir, w.status, task.src_row, c, t_start, w.budget_ns) ? 1 : 0;
-            if (!__syncthreads_and(ok)) return;
+            if (!__syncthreads_and(ok)) break;
         }
 
+        // the bulk copies that read this buffer two tiles ago must have finished reading it
+        if (t < kFanoutIssuers) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        __syncthreads();
+
+        unsigned char* tile = s_tile + buf * kFanoutTileBytes;
         const unsigned char* src = reinterpret_cast<const unsigned char*>(s_src) + b0;
         const unsigned int count = (unsigned int)(b1 - b0);
-        const unsigned int n_dst = task.n_dst;
-        if (count == kFanoutTileBytes) {
-            uint4 v[4];
+        const unsigned int n_vec = count / 16;
+        constexpr int kVecPerThread = kFanoutTileBytes / 16 / kFanoutThreads;
+        uint4 v[kVecPerThread];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) v[q] = __ldcg(reinterpret_cast<const uint4*>(src) + q * kFanoutThreads + t);
-            for (unsigned int r = 0; r < n_dst; ++r) {
-                uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(s_dst[r]) + b0);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) __stcs(dst + q * kFanoutThreads + t, v[q]);
-            }
-        } else {
-            const unsigned int n_vec = count / 16;
-            for (unsigned int q = t; q < n_vec; q += kFanoutThreads) {
-                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(src) + q);
-                for (unsigned int r = 0; r < n_dst; ++r)
-                    __stcs(reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(s_dst[r]) + b0) + q, v);
-            }
-            for (unsigned int b = n_vec * 16 + t; b < count; b += kFanoutThreads) {
-                const unsigned char v = src[b];
-                for (unsigned int r = 0; r < n_dst; ++r) (reinterpret_cast<unsigned char*>(s_dst[r]) + b0)[b] = v;
-            }
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const unsigned int i = q * kFanoutThreads + t;
+            if (i < n_vec) v[q] = __ldcg(reinterpret_cast<const uint4*>(src) + i);
         }
+#pragma unroll
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const unsigned int i = q * kFanoutThreads + t;
+            if (i < n_vec) reinterpret_cast<uint4*>(tile)[i] = v[q];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tile visible to the bulk-copy engine
+        __syncthreads();
+        const unsigned int n_dst = task.n_dst;
+        if (t < kFanoutIssuers) {
+            if (n_vec) {
+                const unsigned int sa = (unsigned int)__cvta_generic_to_shared(tile);
+                for (unsigned int r = t; r < n_dst; r += kFanoutIssuers) bulk_store(s_dst[r] + b0, sa, n_vec * 16);
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        // the last bytes of an object whose size is not a multiple of 16
+        for (unsigned int b = n_vec * 16 + t; b < count; b += kFanoutThreads) {
+            const unsigned char x = src[b];
+            for (unsigned int r = 0; r < n_dst; ++r) (reinterpret_cast<unsigned char*>(s_dst[r]) + b0)[b] = x;
+        }
+        buf ^= 1u;
     }
+    // shared memory must stay valid until the bulk copies have read it, and the writes must be complete
+    if (t < kFanoutIssuers) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------------ launchers
@@ -441,7 +469,13 @@ int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, int grid, void
 }
 
 int launch_fanout_wave(const FanoutWave& w, int grid, void* stream) {
-    fanout_wave_kernel<<<grid, kFanoutThreads, 0, (cudaStream_t)stream>>>(w);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(fanout_wave_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFanoutSmemBytes);
+        if (e != cudaSuccess) return (int)e;
+        attr_set = true;
+    }
+    fanout_wave_kernel<<<grid, kFanoutThreads, kFanoutSmemBytes, (cudaStream_t)stream>>>(w);
     return (int)cudaGetLastError();
 }
 
@@ -461,7 +495,9 @@ int reduce_ctas_per_sm(int n_acc, bool bf16) {
 
 int fanout_ctas_per_sm() {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fanout_wave_kernel, kFanoutThreads, 0) != cudaSuccess) return 1;
+    if (cudaFuncSetAttribute(fanout_wave_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFanoutSmemBytes) != cudaSuccess) return 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fanout_wave_kernel, kFanoutThreads, kFanoutSmemBytes) != cudaSuccess) return 1;
+    if (n > 2) n = 2;   // two CTAs per SM already saturate the write path
     return n < 1 ? 1 : n;
 }
 
