@@ -202,6 +202,9 @@ struct hpl_ctx {
     DeviceStatus* d_status = nullptr;
     DeviceStatus* h_status = nullptr;
     uint32_t* h_iota = nullptr;
+    DirRow* h_stage = nullptr;           // pinned snapshots of directory rows on their way to the device
+    uint32_t stage_cursor = 0;
+    std::vector<int> dirty_rows;         // rows changed on the host since the last flush (batched mode)
     std::vector<int> free_rows;
     std::unordered_map<int64_t, Object> objects;
     std::map<uint64_t, ReduceOp> reduces;  // by creation order
@@ -252,9 +255,40 @@ int alloc_row(hpl_ctx* c, Object& o) {
     r.owner = (unsigned)o.worker;
     // With plan-ahead a kernel that polls may occupy the main stream for a while, so directory rows travel
     // on the control stream (tiny copies only) and the main stream is ordered after it before each launch.
-    cudaStream_t s = c->cfg.plan_ahead ? c->ctl_stream : c->stream;
-    CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, s));
-    if (c->cfg.plan_ahead) c->ctl_pending = true;
+    if (c->cfg.plan_ahead) {
+        CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->ctl_stream));
+        c->ctl_pending = true;
+    } else {
+        c->dirty_rows.push_back(o.row);   // travels with the next flush, before the next launch
+    }
+    return HPL_OK;
+}
+
+constexpr uint32_t kStageRows = 4 * kMaxRows;
+
+// Batched mode (no plan-ahead): all rows changed since the last flush go to the device in one copy per run of
+// consecutive rows, from an immutable pinned snapshot, ordered on the main stream before whatever is
+// launched next.  A Put is then a few stores on the host; its cost on the device is amortised over the batch.
+int flush_directory(hpl_ctx* c) {
+    if (c->dirty_rows.empty()) return HPL_OK;
+    std::sort(c->dirty_rows.begin(), c->dirty_rows.end());
+    c->dirty_rows.erase(std::unique(c->dirty_rows.begin(), c->dirty_rows.end()), c->dirty_rows.end());
+    size_t i = 0;
+    while (i < c->dirty_rows.size()) {
+        size_t j = i + 1;
+        while (j < c->dirty_rows.size() && c->dirty_rows[j] == c->dirty_rows[j - 1] + 1) ++j;
+        const uint32_t n = (uint32_t)(j - i);
+        if (c->stage_cursor + n > kStageRows) {
+            CUDA_TRY(cudaStreamSynchronize(c->stream));   // every earlier snapshot has been consumed
+            c->stage_cursor = 0;
+        }
+        DirRow* snap = c->h_stage + c->stage_cursor;
+        std::memcpy(snap, c->h_dir + c->dirty_rows[i], n * sizeof(DirRow));
+        CUDA_TRY(cudaMemcpyAsync(c->d_dir + c->dirty_rows[i], snap, n * sizeof(DirRow), cudaMemcpyHostToDevice, c->stream));
+        c->stage_cursor += n;
+        i = j;
+    }
+    c->dirty_rows.clear();
     return HPL_OK;
 }
 
@@ -269,6 +303,11 @@ int order_main_after_control(hpl_ctx* c) {
 // Publishes the chunk prefix of a put object in the device directory, ordered on `s`.
 int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
     if (!c->device || o.row < 0) return HPL_OK;
+    c->h_dir[o.row].ready_chunks = chunks;   // the host mirror always holds the published value
+    if (s == c->stream && !c->cfg.plan_ahead) {
+        c->dirty_rows.push_back(o.row);
+        return HPL_OK;
+    }
     CUDA_TRY(cudaMemcpyAsync(&c->d_dir[o.row].ready_chunks, &c->h_iota[chunks], sizeof(uint32_t), cudaMemcpyHostToDevice, s));
     return HPL_OK;
 }
@@ -755,6 +794,8 @@ int progress(hpl_ctx* c) {
     {
         int rc = order_main_after_control(c);
         if (rc != HPL_OK) return rc;
+        rc = flush_directory(c);
+        if (rc != HPL_OK) return rc;
     }
     if (c->copy_pending && !c->cfg.plan_ahead) {
         // host objects: their chunks become usable once the main stream is ordered after the copies
@@ -807,8 +848,7 @@ int sync_and_check(hpl_ctx* c) {
         for (auto& kv : c->objects)
             if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
-    if (!c->work_in_flight) {
-        CUDA_TRY(cudaStreamSynchronize(c->stream));
+    if (!c->work_in_flight) {   // nothing of the library's is running: nothing to wait for
         c->journal.clear();
         return HPL_OK;
     }
@@ -909,6 +949,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         bool ok = c->d_dir && c->d_status;
         ok = ok && cudaHostAlloc((void**)&c->h_dir, sizeof(DirRow) * kMaxRows, cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaHostAlloc((void**)&c->h_status, sizeof(DeviceStatus), cudaHostAllocDefault) == cudaSuccess;
+        ok = ok && cudaHostAlloc((void**)&c->h_stage, sizeof(DirRow) * kStageRows, cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaHostAlloc((void**)&c->h_iota, sizeof(uint32_t) * (kMaxChunks + 1), cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->ctl_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -920,6 +961,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         if (!ok) {
             if (c->h_dir) cudaFreeHost(c->h_dir);
             if (c->h_status) cudaFreeHost(c->h_status);
+            if (c->h_stage) cudaFreeHost(c->h_stage);
             if (c->h_iota) cudaFreeHost(c->h_iota);
             if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
             if (c->ctl_stream) cudaStreamDestroy(c->ctl_stream);
@@ -946,6 +988,7 @@ int hpl_shutdown(hpl_ctx* c) {
         for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
         cudaFreeHost(c->h_dir);
         cudaFreeHost(c->h_status);
+        cudaFreeHost(c->h_stage);
         cudaFreeHost(c->h_iota);
         cudaStreamDestroy(c->copy_stream);
         cudaStreamDestroy(c->ctl_stream);
@@ -1050,6 +1093,8 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
         }
         // the row (pointer) must be in the directory before any copy-stream counter update can matter
         cudaStream_t row_stream = c->cfg.plan_ahead ? c->ctl_stream : c->stream;
+        rc = flush_directory(c);
+        if (rc != HPL_OK) return rc;
         CUDA_TRY(cudaEventRecord(c->copy_ev, row_stream));
         CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
     }
