@@ -632,6 +632,7 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16);
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
             if (grid < 1) grid = 1;
+            if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
             {
                 LaunchTimer timer(c, 0);
                 if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
@@ -775,6 +776,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
+        if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
         {
             LaunchTimer timer(c, 1);
             if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
