@@ -116,6 +116,8 @@ class Context:
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
                      int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes)
         self._h = C.c_void_p()
+        self._p, self._n = C.c_void_p(), C.c_uint64()
+        self._pref, self._nref = C.byref(self._p), C.byref(self._n)
         self._check(self._lib.hpl_init(C.byref(cfg), C.c_void_p(stream or None), C.byref(self._h)), "hpl_init")
 
     def _check(self, rc: int, what: str) -> int:
@@ -134,14 +136,21 @@ class Context:
     def __exit__(self, *exc):
         self.shutdown()
 
+    # the per-object calls below are on every step's path: they pass plain integers straight to ctypes
     def advance(self, t_ns: int):
-        self._check(self._lib.hpl_advance(self._h, t_ns), "hpl_advance")
+        rc = self._lib.hpl_advance(self._h, t_ns)
+        if rc:
+            raise HplError(rc, "hpl_advance")
 
     def create(self, object_id: int, worker: int, total_bytes: int, dtype: int = HPL_F32):
-        self._check(self._lib.hpl_create(self._h, object_id, worker, total_bytes, dtype), "hpl_create")
+        rc = self._lib.hpl_create(self._h, object_id, worker, total_bytes, dtype)
+        if rc:
+            raise HplError(rc, "hpl_create")
 
     def put(self, object_id: int, dev_buf, nbytes: int):
-        self._check(self._lib.hpl_put(self._h, object_id, C.c_void_p(_addr(dev_buf)), nbytes), "hpl_put")
+        rc = self._lib.hpl_put(self._h, object_id, dev_buf if type(dev_buf) is int else _addr(dev_buf), nbytes)
+        if rc:
+            raise HplError(rc, "hpl_put")
 
     def put_host(self, object_id: int, host_buf, nbytes: int):
         self._check(self._lib.hpl_put_host(self._h, object_id, C.c_void_p(_addr(host_buf)), nbytes), "hpl_put_host")
@@ -155,12 +164,20 @@ class Context:
         self._check(self._lib.hpl_broadcast(self._h, src_id, arr, len(dst_ids)), "hpl_broadcast")
 
     def join(self, dst_id: int, dev_buf=0):
-        self._check(self._lib.hpl_join(self._h, dst_id, C.c_void_p(_addr(dev_buf) if dev_buf is not None else None)), "hpl_join")
+        if dev_buf is None:
+            ptr = None
+        else:
+            ptr = dev_buf if type(dev_buf) is int else _addr(dev_buf)
+        rc = self._lib.hpl_join(self._h, dst_id, ptr)
+        if rc:
+            raise HplError(rc, "hpl_join")
 
     def get(self, object_id: int):
         """Returns ``(device_pointer, nbytes)``."""
-        p, n = C.c_void_p(), C.c_uint64()
-        self._check(self._lib.hpl_get(self._h, object_id, C.byref(p), C.byref(n)), "hpl_get")
+        p, n = self._p, self._n
+        rc = self._lib.hpl_get(self._h, object_id, self._pref, self._nref)
+        if rc:
+            raise HplError(rc, "hpl_get")
         return p.value, n.value
 
     def try_get(self, object_id: int):
