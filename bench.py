@@ -279,6 +279,21 @@ def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
             "h2d": h2d, "d2h": d2h}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(step_bytes, steps, world, total_ms):
+    """Aggregate throughput: every rank moved ``step_bytes * steps``; the job took the slowest rank's time."""
+    return gbs(step_bytes * steps * world, total_ms)
+
+
 def gbs(nbytes, ms):
     return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
@@ -411,14 +426,8 @@ def main():
     del runner
     torch.cuda.empty_cache()
 
-    total_ms = float(np.sum(res["total_ms"]))
-    if dist is not None:
-        tmax = torch.tensor([total_ms, res["wall_ms"]], device=device, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        total_ms, wall_ms = float(tmax[0]), float(tmax[1])
-    else:
-        wall_ms = res["wall_ms"]
-    value = gbs(step_bytes * args.steps * world, total_ms)
+    total_ms, wall_ms = max_over_ranks([float(np.sum(res["total_ms"])), res["wall_ms"]], dist, device)
+    value = whole_job_value(step_bytes, args.steps, world, total_ms)
     peak, peak_kind = measured_peak()
     st = res["stats"]
 
@@ -476,12 +485,8 @@ def main():
         rr.close()
         del rr
         torch.cuda.empty_cache()
-        e_ms = float(np.sum(r3["total_ms"]))
-        if dist is not None:
-            tm = torch.tensor([e_ms], device=device, dtype=torch.float64)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            e_ms = float(tm[0])
-        line["e2e"] = {"value": gbs(step_bytes * e_steps * world, e_ms), "unit": "GB/s", "h2d_bytes_per_step": int(r3["h2d"]),
+        e_ms = max_over_ranks([float(np.sum(r3["total_ms"]))], dist, device)[0]
+        line["e2e"] = {"value": whole_job_value(step_bytes, e_steps, world, e_ms), "unit": "GB/s", "h2d_bytes_per_step": int(r3["h2d"]),
                        "d2h_bytes_per_step": int(r3["d2h"]), "ms_per_step": e_ms / e_steps,
                        "how": "hpl_put_host from pinned host memory, chunks consumed by polling kernels as they land; hpl_get_host of the result"}
 
