@@ -60,7 +60,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -116,7 +116,7 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
 class Runner:
     """Holds the device buffers of one workload and runs steps through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device, host_buffers: bool = False, plan_ahead: bool = False):
+    def __init__(self, w: wl.Workload, device, host_buffers: bool = False, plan_ahead: bool = False, ft_eager: bool = True):
         import torch
         import paper_2002_05814_b200 as hpl
 
@@ -124,6 +124,7 @@ class Runner:
         self.dt = hpl.HPL_BF16 if w.dtype == "bf16" else hpl.HPL_F32
         S = w.object_bytes
         self.host_buffers = host_buffers
+        self.ft_eager = ft_eager
         n_src = w.n_objects
         arena_bytes = 64 * MiB + 2 * w.elems * 4 + (n_src + 2) * S * (1 if host_buffers else 0)
         if w.kind == "ft_reduce":
@@ -223,7 +224,8 @@ class Runner:
                     ctx.put(ids[i], self.src[i].data_ptr(), nbytes)
             self.t += tmax
             if w.kind == "ft_reduce":
-                ctx.progress()                       # chunks delivered by every worker are reduced before the failure
+                if self.ft_eager:
+                    ctx.progress()                   # chunks delivered by every worker are reduced before the failure
                 self.t += 1
                 ctx.advance(self.t)
                 ctx.fail(w.extra["fail_worker"])
@@ -360,12 +362,15 @@ def oracle_sample(w: wl.Workload, budget_s: float = 12.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--size", type=int, default=64 * MiB, help="object bytes for cfg5")
     ap.add_argument("--shrink", type=int, default=1, help="divide the object size by this (profiling captures on a smaller case)")
+    ap.add_argument("--ft-mode", default="eager", choices=["eager", "lazy"],
+                    help="cfg5: 'eager' runs hpl_progress before the failure (chunks delivered by every worker are reduced, "
+                         "then partly redone); 'lazy' applies the compressed timeline and plans at the Get")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads measured briefly and reported under 'also'")
@@ -418,7 +423,7 @@ def main():
     device = torch.device("cuda", local)
 
     sampler = ClockSampler(local)
-    runner = Runner(w, device)
+    runner = Runner(w, device, ft_eager=args.ft_mode == "eager")
     sampler.start()
     res = time_steps(runner, args.steps, args.warmup, dist)
     clocks = sampler.stop()
@@ -452,6 +457,12 @@ def main():
             "roofline": r_red if r_red is not None else r_fan}
     if r_red is not None and r_fan is not None:
         line["roofline_fanout"] = r_fan
+    planned = (st["bytes_read_planned"] + st["bytes_written_planned"]) / args.steps
+    kern_ms = (st["reduce_kernel_ns"] + st["fanout_kernel_ns"]) / 1e6 / args.steps
+    line["planned_traffic"] = {"bytes_per_step": planned, "over_algorithmic": planned / step_bytes,
+                               "kernel_GBps_on_planned_bytes": gbs(planned, kern_ms), "kernel_ms_per_step": kern_ms}
+    if w.kind == "ft_reduce":
+        line["config"]["ft_mode"] = args.ft_mode
     if ab["reduce"]:
         line["reduce"] = {"GBps": gbs(ab["reduce"] * args.steps, float(np.sum(res["reduce_ms"]))), "ms": float(np.mean(res["reduce_ms"])),
                           "ms_std": float(np.std(res["reduce_ms"]))}

@@ -669,11 +669,17 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
     }
     std::vector<int64_t> pre(op.phys_have);  // what every copy holds before this pass
     pre[0] = src_avail;
-    auto usable = [&](int x) {
-        if (x == 0) return src->alive && src->ptr != nullptr;
+    std::vector<char> usable_v(locs.size(), 0);   // copies whose buffer may be read or written now
+    usable_v[0] = src->alive && src->ptr != nullptr;
+    bool any_pending = false;
+    for (size_t x = 1; x < locs.size(); ++x) {
+        if (!locs[x].alive) continue;
         Object* o = find(c, locs[x].obj);
-        return locs[x].alive && o && o->alive && o->ptr && o->row >= 0;
-    };
+        usable_v[x] = o && o->alive && o->ptr && o->row >= 0;
+        if (usable_v[x] && op.phys_have[x] < (int64_t)C) any_pending = true;
+    }
+    if (!any_pending) return HPL_OK;
+    auto usable = [&](int x) { return usable_v[x] != 0; };
     std::vector<uint32_t> bp = {0u, src_avail};
     for (size_t i = 1; i < locs.size(); ++i) bp.push_back((uint32_t)pre[i]);
     std::sort(bp.begin(), bp.end());
