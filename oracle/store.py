@@ -9,6 +9,11 @@ times: failures, then publications, then requests).
 
 "Arrival" of an object is its first publication, which Section 3.2 places at the moment Put is
 called, before the copy has finished.
+
+Composition (Sections 3.3, 3.4.2, 3.4.3): the output of a Reduce is an object like any other.  It is
+published (as partial) when the Reduce is called, so it may be a source of a later Reduce or the
+source of a broadcast (reduce followed by broadcast = allreduce); its chunk prefix is what its
+current tree can already produce -- the smallest prefix among its members once the tree is full.
 """
 from __future__ import annotations
 
@@ -38,6 +43,7 @@ class _Entry:
         self.data = None
         self.ready_bytes = 0
         self.alive = True
+        self.arrived = False
         self.t_arrival = -1
         self.chunk_bytes = chunk_bytes
 
@@ -87,16 +93,18 @@ class OracleStore:
             raise StoreError(ERR_INVALID, "produced by a collective")
         if nbytes < e.ready_bytes or nbytes > e.nbytes or data.nbytes != e.nbytes:
             raise StoreError(ERR_INVALID)
-        first = e.data is None
+        first = not e.arrived
         e.data = data
         e.ready_bytes = nbytes
         if first:
+            e.arrived = True
             e.t_arrival = self.now
             for r in self.reduces.values():
                 if oid in r["srcs"]:
                     r["sched"].on_arrival(oid)
         if oid in self.bcasts:
             self.bcasts[oid]["sched"].source_progress(self.now, e.ready_chunks)
+        self._refresh_composed()
 
     def reduce(self, target: int, srcs: list[int], k: int, op: int = OP_SUM, dtype: int = DT_F32) -> None:
         if target in self.objects:
@@ -105,7 +113,7 @@ class OracleStore:
         if not (1 <= k <= n) or len(set(srcs)) != n:
             raise StoreError(ERR_INVALID)
         ents = [self._entry(s) for s in srcs]
-        if any(e.dtype != dtype or e.nbytes != ents[0].nbytes for e in ents):
+        if any(e.dtype != dtype or e.nbytes != ents[0].nbytes or e.oid in self.dst_of for e in ents):
             raise StoreError(ERR_INVALID)
         live = [e for e in ents if e.alive]
         if len(live) < 1:
@@ -116,10 +124,14 @@ class OracleStore:
         for e in ents:                       # sources lost before the call never take part
             if not e.alive:
                 sched.on_fail(e.oid, 0, self._delivered)
-        arrived = sorted((e for e in live if e.data is not None), key=lambda e: (e.t_arrival, srcs.index(e.oid)))
+        arrived = sorted((e for e in live if e.arrived), key=lambda e: (e.t_arrival, srcs.index(e.oid)))
         for e in arrived:
             sched.on_arrival(e.oid)
         self.reduces[target] = {"sched": sched, "op": op, "srcs": list(srcs)}
+        t = self.objects[target]          # the output is published at once, as a partial object
+        t.arrived = True
+        t.t_arrival = self.now
+        self._refresh_composed()
 
     def broadcast(self, src: int, dsts: list[int]) -> None:
         e = self._entry(src)
@@ -127,15 +139,15 @@ class OracleStore:
             raise StoreError(ERR_EXISTS)
         for dd in dsts:
             de = self._entry(dd)
-            if de.nbytes != e.nbytes or de.dtype != e.dtype or dd in self.dst_of or de.data is not None:
+            if de.nbytes != e.nbytes or de.dtype != e.dtype or dd in self.dst_of or de.arrived or dd in self.reduces:
                 raise StoreError(ERR_INVALID)
         sched = BroadcastSchedule(src, e.C, self.d_bcast, self.tau)
         sched.advance(self.now)
         if not e.alive:
             raise StoreError(ERR_FAILED_WORKER)
-        if e.data is not None:
-            # chunks published before the broadcast existed count as available from t_arrival on
-            sched.source_progress(self.now, e.ready_chunks)
+        if e.arrived:
+            # chunks published before the broadcast existed count as available from now on
+            sched.source_progress(self.now, self._delivered(src))
         self.bcasts[src] = {"sched": sched, "dsts": list(dsts)}
         for dd in dsts:
             self.dst_of[dd] = src
@@ -159,6 +171,7 @@ class OracleStore:
             mine = [e.oid for e in lost if e.oid == src or self.dst_of.get(e.oid) == src]
             if mine:
                 b["sched"].fail(self.now, mine)
+        self._refresh_composed()
 
     def delete(self, oid: int) -> None:
         self._entry(oid)
@@ -180,12 +193,14 @@ class OracleStore:
             sched: ReduceSchedule = r["sched"]
             if sched.k == 0:
                 raise StoreError(ERR_INSUFFICIENT)
-            if not sched.full() or any(not self.objects[m].complete for m in sched.members()):
+            if not sched.full() or any(self._delivered(m) < self.objects[m].C for m in sched.members()):
                 raise StoreError(ERR_TIMEOUT)
-            if e.data is None:
-                objs = {m: self.objects[m].data for m in sched.members()}
+            key = self._membership(oid)
+            if e.data is None or r.get("evaluated") != key:
+                # a member that is itself the output of a Reduce is evaluated first (composed Reduce)
+                objs = {m: (self.get(m) if m in self.reduces else self.objects[m].data) for m in sched.members()}
                 e.data = tree_reduce(sched.obj_at, sched.d, objs, r["op"])
-                e.ready_bytes = e.nbytes
+                r["evaluated"] = key
             return e.data
         if oid in self.dst_of:
             if not e.alive:
@@ -203,8 +218,9 @@ class OracleStore:
             self.now = max(self.now, sched.now)
             for b in self.bcasts.values():
                 b["sched"].advance(self.now)
-            if e.data is None:
-                e.data = self.objects[src].data.copy() if src in self.objects else None
+            srcdata = self.get(src) if src in self.reduces else self.objects[src].data
+            if e.data is None or src in self.reduces:
+                e.data = srcdata.copy()
                 e.ready_bytes = e.nbytes
             return e.data
         if not e.alive:
@@ -228,4 +244,21 @@ class OracleStore:
         return self.objects[oid]
 
     def _delivered(self, oid: int) -> int:
+        """Published chunk prefix: of a Put object what was put; of a Reduce output what its tree can produce."""
+        if oid in self.reduces:
+            sched = self.reduces[oid]["sched"]
+            if not sched.full():
+                return 0
+            return min(self._delivered(m) for m in sched.members())
         return self.objects[oid].ready_chunks
+
+    def _membership(self, oid: int) -> tuple:
+        """Who is in the tree of ``oid``, and in the trees of the members that are Reduce outputs themselves."""
+        sched = self.reduces[oid]["sched"]
+        return tuple(sched.obj_at) + tuple(self._membership(m) for m in sched.members() if m in self.reduces)
+
+    def _refresh_composed(self) -> None:
+        """After every event: a broadcast whose source is a Reduce output learns how far that output has got."""
+        for src, b in self.bcasts.items():
+            if src in self.reduces:
+                b["sched"].source_progress(self.now, self._delivered(src))

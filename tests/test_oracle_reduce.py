@@ -281,3 +281,57 @@ def test_store_reduce_with_no_live_source_is_insufficient():
     with pytest.raises(StoreError) as ei:
         st.get(100)
     assert ei.value.code == ERR_INSUFFICIENT
+
+
+# ---------------------------------------------------------------- composition (Sections 3.3, 3.4.2, 3.4.3)
+def test_composed_reduce_and_allreduce_equal_the_plain_sums():
+    st, data = _store_with(6, 3, 2, elems=64)
+    st.reduce(100, [0, 1, 2], 3)                 # first Reduce: a future
+    st.reduce(200, [100, 3, 4], 3)               # its output id is an input of the next one
+    for j in (300, 301, 302):
+        st.create(j, 50 + j, 256, DT_F32)
+    st.broadcast(200, [300, 301, 302])           # reduce followed by broadcast = allreduce
+    st.join(300)
+    with pytest.raises(StoreError):
+        st.get(200)
+    st.advance(1)
+    for o in (0, 1):
+        st.put(o, data[o], 256)
+    st.put(2, data[2], 128)                      # object 2 is half there: so is the first output
+    assert st._delivered(100) == 2 and st._delivered(200) == 0
+    st.advance(2)
+    for o in (3, 4):
+        st.put(o, data[o], 256)
+    assert st._delivered(200) == 2               # the partial first output already feeds the second Reduce
+    st.join(301)
+    st.advance(3)
+    st.put(2, data[2], 256)
+    st.join(302)
+    total = sum(data[o] for o in range(5))       # integer-valued inputs: any association is exact
+    assert np.array_equal(st.get(100), data[0] + data[1] + data[2])
+    assert np.array_equal(st.get(200), total)
+    for j in (300, 301, 302):
+        assert st.get(j).tobytes() == total.astype(np.float32).tobytes()
+    # each input was reduced once and only once (Section 3.4.2)
+    ones = {o: np.ones(64, np.float32) for o in range(5)}
+    st2, _ = _store_with(6, 3, 2, elems=64)
+    st2.reduce(100, [0, 1, 2], 3)
+    st2.reduce(200, [100, 3, 4], 3)
+    for o in range(5):
+        st2.put(o, ones[o], 256)
+    assert np.array_equal(st2.get(200), np.full(64, 5, np.float32))
+
+
+def test_composed_reduce_redoes_the_downstream_after_an_upstream_failure():
+    st, data = _store_with(6, 3, 2, elems=64)
+    st.reduce(100, [0, 1, 2, 5], 3)
+    st.reduce(200, [100, 3], 2)
+    for o in (0, 1, 2, 3):
+        st.put(o, data[o], 256)
+    assert np.array_equal(st.get(200), data[0] + data[1] + data[2] + data[3])
+    st.advance(9)
+    st.fail(1)                                   # a member of the first Reduce is lost; object 5 is its spare
+    with pytest.raises(StoreError):
+        st.get(200)
+    st.put(5, data[5], 256)
+    assert np.array_equal(st.get(200), data[0] + data[5] + data[2] + data[3])
