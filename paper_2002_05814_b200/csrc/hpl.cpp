@@ -234,6 +234,32 @@ Object* find(hpl_ctx* c, int64_t id) {
     return it == c->objects.end() ? nullptr : &it->second;
 }
 
+// Chunk prefix an object has published, as the schedules see it: of a Put object what was put; of a Reduce
+// output (published when Reduce is called, Section 3.4.2) what its tree can already produce.
+int64_t logical_delivered(hpl_ctx* c, int64_t oid) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    if (o->kind == OBJ_TARGET) {
+        auto it = c->reduce_of_target.find(oid);
+        if (it == c->reduce_of_target.end()) return 0;
+        ReduceTreeSchedule& s = *c->reduces.at(it->second).sched;
+        if (!s.full()) return 0;
+        int64_t m = o->C;
+        for (int p = 0; p < s.k(); ++p) m = std::min(m, logical_delivered(c, s.object_at(p)));
+        return m;
+    }
+    return (int64_t)published_chunks(c, *o);
+}
+
+// Chunks of a Reduce output that earlier waves on the stream have produced (or will have, by stream order).
+uint32_t produced_prefix(hpl_ctx* c, const Object& o) {
+    auto it = c->reduce_of_target.find(o.id);
+    if (it == c->reduce_of_target.end()) return 0;
+    const ReduceOp& op = c->reduces.at(it->second);
+    if (op.computed.empty() || op.computed[0].iv.empty() || op.computed[0].iv[0].first != 0) return 0;
+    return op.computed[0].iv[0].second;
+}
+
 #define CUDA_TRY(x)                                  \
     do {                                             \
         if ((x) != cudaSuccess) return HPL_ERR_CUDA; \
@@ -515,9 +541,13 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         if (oid < 0) continue;
         Object* o = find(c, oid);
         if (!o || !o->alive || !o->ptr || o->row < 0) continue;
-        const uint32_t pub = published_chunks(c, *o);
-        landed[p] = std::min(pub, o->landed);
-        ready[p] = c->cfg.plan_ahead ? o->C : landed[p];
+        if (o->kind == OBJ_TARGET) {   // composed Reduce: the member is the output of an earlier Reduce
+            landed[p] = ready[p] = produced_prefix(c, *o);
+        } else {
+            const uint32_t pub = published_chunks(c, *o);
+            landed[p] = std::min(pub, o->landed);
+            ready[p] = c->cfg.plan_ahead ? o->C : landed[p];
+        }
         bp.push_back(ready[p]);
         bp.push_back(landed[p]);
     }
@@ -664,8 +694,12 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
     const uint32_t C = src->C;
     uint32_t src_landed = 0, src_avail = 0;
     if (src->alive && src->ptr && src->row >= 0) {
-        src_landed = std::min(published_chunks(c, *src), src->landed);
-        src_avail = c->cfg.plan_ahead ? C : src_landed;
+        if (src->kind == OBJ_TARGET) {   // reduce followed by broadcast: the source is a Reduce output
+            src_landed = src_avail = produced_prefix(c, *src);
+        } else {
+            src_landed = std::min(published_chunks(c, *src), src->landed);
+            src_avail = c->cfg.plan_ahead ? C : src_landed;
+        }
     }
     std::vector<int64_t> pre(op.phys_have);  // what every copy holds before this pass
     pre[0] = src_avail;
@@ -813,19 +847,27 @@ int progress(hpl_ctx* c) {
         for (auto& kv : c->objects)
             if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
-    for (auto& kv : c->bcasts) {
-        std::vector<PlannedFanout> tasks;
-        int rc = plan_bcast(c, kv.second, tasks);
-        if (rc != HPL_OK) return rc;
-        rc = launch_fanout_tasks(c, kv.second, tasks);
-        if (rc != HPL_OK) return rc;
-    }
-    for (auto& kv : c->reduces) {
-        std::vector<PlannedReduceTask> tasks;
-        int rc = plan_reduce(c, kv.second, tasks);
-        if (rc != HPL_OK) return rc;
-        rc = launch_reduce_tasks(c, kv.second, tasks);
-        if (rc != HPL_OK) return rc;
+    // collectives in creation order, so that one that consumes another's output (composed Reduce, reduce
+    // followed by broadcast) is planned after its producer and launched behind it on the stream
+    auto ri = c->reduces.begin();
+    auto bi = c->bcasts.begin();
+    while (ri != c->reduces.end() || bi != c->bcasts.end()) {
+        const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
+        if (take_reduce) {
+            std::vector<PlannedReduceTask> tasks;
+            int rc = plan_reduce(c, ri->second, tasks);
+            if (rc != HPL_OK) return rc;
+            rc = launch_reduce_tasks(c, ri->second, tasks);
+            if (rc != HPL_OK) return rc;
+            ++ri;
+        } else {
+            std::vector<PlannedFanout> tasks;
+            int rc = plan_bcast(c, bi->second, tasks);
+            if (rc != HPL_OK) return rc;
+            rc = launch_fanout_tasks(c, bi->second, tasks);
+            if (rc != HPL_OK) return rc;
+            ++bi;
+        }
     }
     return HPL_OK;
 }
@@ -877,9 +919,29 @@ int sync_and_check(hpl_ctx* c) {
 
 int after_event(hpl_ctx* c) { return c->cfg.eager ? progress(c) : HPL_OK; }
 
-int64_t delivered_of(hpl_ctx* c, int64_t oid) {
-    Object* o = find(c, oid);
-    return o ? (int64_t)published_chunks(c, *o) : 0;
+int64_t delivered_of(hpl_ctx* c, int64_t oid) { return logical_delivered(c, oid); }
+
+// After every event: a broadcast whose source is a Reduce output learns how far that output has got.
+void refresh_composed(hpl_ctx* c) {
+    for (auto& kv : c->bcasts) {
+        Object* src = find(c, kv.second.src);
+        if (src && src->kind == OBJ_TARGET) kv.second.sched->source_progress((int64_t)c->now, logical_delivered(c, src->id));
+    }
+}
+
+// The value of `target` changes (a member of its tree was replaced): whatever was computed from it is void.
+void invalidate_consumers(hpl_ctx* c, int64_t target) {
+    for (auto& kv : c->reduces) {
+        ReduceOp& op = kv.second;
+        if (!op.sched->has_source(target)) continue;
+        for (auto& cs : op.computed) cs.clear();
+        invalidate_consumers(c, op.target);
+    }
+    auto b = c->bcast_of_src.find(target);
+    if (b != c->bcast_of_src.end()) {
+        BcastOp& op = c->bcasts.at(b->second);
+        std::fill(op.phys_have.begin(), op.phys_have.end(), 0);
+    }
 }
 
 void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv) {
@@ -906,6 +968,7 @@ int do_put_common(hpl_ctx* c, Object& o, uint64_t bytes, bool first) {
     }
     auto b = c->bcast_of_src.find(o.id);
     if (b != c->bcast_of_src.end()) c->bcasts.at(b->second).sched->source_progress((int64_t)c->now, published_chunks(c, o));
+    refresh_composed(c);
     return HPL_OK;
 }
 
@@ -1141,7 +1204,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     for (int64_t s : srcs) {
         Object* o = find(c, s);
         if (!o) return HPL_ERR_NOT_FOUND;
-        if (o->dtype != dtype || (bytes && o->bytes != bytes)) return HPL_ERR_INVALID;
+        if (o->dtype != dtype || (bytes && o->bytes != bytes) || o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;
         bytes = o->bytes;
         if (o->alive) ++live;
     }
@@ -1156,6 +1219,9 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     t.C = find(c, srcs[0])->C;
     t.kind = OBJ_TARGET;
     t.lib_owned = true;
+    t.arrived = true;   // the output is published at once, as a partial object (Section 3.4.2)
+    t.t_arrival = (int64_t)c->now;
+    t.ready_bytes = 0;
     t.seq = c->seq++;
     if (c->device) {
         t.ptr = c->arena.alloc(t.bytes);
@@ -1193,6 +1259,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     const uint64_t key = r.seq;
     c->reduce_of_target[target] = key;
     c->reduces.emplace(key, std::move(r));
+    refresh_composed(c);
     return after_event(c);
 }
 
@@ -1213,7 +1280,7 @@ int hpl_broadcast(hpl_ctx* c, int64_t src_id, const int64_t* dst_ids, int32_t n)
     b.src = src_id;
     b.sched.reset(new BroadcastTreeSchedule(src_id, src->C, c->cfg.bcast_degree, (int64_t)c->tau));
     b.sched->advance((int64_t)c->now);
-    if (src->arrived) b.sched->source_progress((int64_t)c->now, published_chunks(c, *src));
+    if (src->arrived) b.sched->source_progress((int64_t)c->now, logical_delivered(c, src_id));
     b.dsts.assign(dst_ids, dst_ids + n);
     b.seq = c->seq++;
     for (int i = 0; i < n; ++i) {
@@ -1259,6 +1326,7 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
             if (!op.sched->has_source(o->id)) continue;
             ReduceInvalidation inv = op.sched->fail(o->id, (int64_t)published_chunks(c, *o), dl);
             apply_invalidation(op, inv);
+            if (!inv.positions.empty() || inv.shrank) invalidate_consumers(c, op.target);
         }
     }
     for (auto& kv : c->bcasts) {
@@ -1268,6 +1336,7 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
             if (o->id == op.src || (o->kind == OBJ_RECEIVER && o->op_key == op.src)) mine.push_back(o->id);
         if (!mine.empty()) op.sched->fail((int64_t)c->now, mine);
     }
+    refresh_composed(c);
     return after_event(c);
 }
 
@@ -1293,7 +1362,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (!op.sched->full()) return HPL_ERR_TIMEOUT;
         for (int p = 0; p < op.sched->k(); ++p) {
             Object* m = find(c, op.sched->object_at(p));
-            if (!m || m->ready_bytes < m->bytes) return HPL_ERR_TIMEOUT;
+            if (!m || logical_delivered(c, m->id) < (int64_t)m->C) return HPL_ERR_TIMEOUT;
         }
         if (!c->device) return HPL_ERR_CUDA;
         if (!op.computed[0].contains(0, op.C)) return HPL_ERR_TIMEOUT;
@@ -1307,6 +1376,15 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (!op.sched->run_until_complete(id)) return HPL_ERR_TIMEOUT;
         if ((uint64_t)op.sched->now() > c->now) c->now = (uint64_t)op.sched->now();
         for (auto& kv : c->bcasts) kv.second.sched->advance((int64_t)c->now);
+        {
+            // a copy of a Reduce output is only complete while that output is (a member may have been lost since)
+            Object* so = find(c, op.src);
+            if (so && so->kind == OBJ_TARGET) {
+                ReduceOp& up = c->reduces.at(c->reduce_of_target.at(op.src));
+                if (up.sched->k() == 0) return HPL_ERR_INSUFFICIENT;
+                if (logical_delivered(c, op.src) < (int64_t)so->C) return HPL_ERR_TIMEOUT;
+            }
+        }
         if (!c->device) return HPL_ERR_CUDA;
         if (li < (int)op.phys_have.size() && op.phys_have[li] >= (int64_t)o->C && !c->work_in_flight && !c->copy_pending) {
             if (dev_ptr) *dev_ptr = o->ptr;   // already copied and waited for

@@ -191,3 +191,61 @@ def _bcast_timeline(seed):
 def test_broadcast_schedules_match_on_random_timelines(block):
     for seed in range(block * 150, (block + 1) * 150):
         _bcast_timeline(seed)
+
+
+def _composed_timeline(seed):
+    """Reduce A, Reduce B that takes A's output as an input, and a broadcast of B's output (allreduce)."""
+    rng = np.random.default_rng(seed)
+    na, nb, R = int(rng.integers(1, 6)), int(rng.integers(1, 5)), int(rng.integers(1, 6))
+    ka = int(rng.integers(1, na + 1))
+    kb = int(rng.integers(1, nb + 2))
+    d = int(rng.integers(1, 4))
+    tau = int(rng.integers(1, 20))
+    nbytes = int(rng.integers(1, 6)) * 64
+    p = Pair(d, int(rng.integers(1, 3)), tau)
+    n = na + nb
+    n_workers = max(1, int(rng.integers(1, n + 1)))
+    for i in range(n):
+        p.create(i, int(rng.integers(0, n_workers)), nbytes)
+    for j in range(R):
+        p.create(500 + j, 100 + int(rng.integers(0, 3)), nbytes)
+    A, B = 1000, 2000
+    ops = []
+    if p.both("reduce", A, list(range(na)), ka, 0, 0) != OK:
+        p.close()
+        return
+    ops.append(A)
+    if p.both("reduce", B, [A] + list(range(na, n)), kb, 0, 0) == OK:
+        ops.append(B)
+        if p.both("broadcast", B, [500 + j for j in range(R)]) == OK:
+            ops.append("bcast")
+    prefix = {i: 0 for i in range(n)}
+    joiners = [500 + j for j in range(R)]
+    t = 0
+    for s in range(int(rng.integers(n, 5 * n + 6))):
+        t += int(rng.integers(0, 2 * tau))
+        p.both("advance", max(t, p.o.now))
+        t = max(t, p.o.now)
+        r = rng.random()
+        if r < 0.5:
+            i = int(rng.integers(0, n))
+            nb_ = nbytes if rng.random() < 0.5 else min(nbytes, prefix[i] + 64)
+            p.put(i, nb_)
+            if p.o.objects[i].alive:
+                prefix[i] = max(prefix[i], nb_)
+        elif r < 0.62:
+            p.both("fail", int(rng.integers(0, n_workers)))
+        elif r < 0.8 and joiners and "bcast" in ops:
+            p.join(joiners.pop(0))
+        else:
+            p.get(int(rng.choice([A, B] + [500 + j for j in range(R)])) if len(ops) > 1 else A)
+            t = max(t, p.o.now)
+        for o in ops:
+            p.compare(B if o == "bcast" else o)
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_composed_schedules_match_on_random_timelines(block):
+    for seed in range(block * 150, (block + 1) * 150):
+        _composed_timeline(seed)
