@@ -40,6 +40,8 @@ class _Entry:
     def __init__(self, oid, worker, nbytes, dtype, chunk_bytes):
         self.oid, self.worker, self.nbytes, self.dtype = oid, worker, nbytes, dtype
         self.C = (nbytes + chunk_bytes - 1) // chunk_bytes
+        self.elems = nbytes // _ELEM[dtype]
+        self.chunk_elems = max(1, min(chunk_bytes, nbytes) // _ELEM[dtype])   # elements per chunk of this object
         self.data = None
         self.ready_bytes = 0
         self.alive = True
@@ -121,13 +123,15 @@ class OracleStore:
         elems = ents[0].nbytes // _ELEM[dtype]
         self.create(target, -1, elems * 4, DT_F32)
         sched = ReduceSchedule(srcs, k, self.d_reduce)
+        self.reduces[target] = {"sched": sched, "op": op, "srcs": list(srcs), "chunk_elems": ents[0].chunk_elems,
+                                "C": ents[0].C}
+        delivered = lambda o: self._delivered_in(o, target)
         for e in ents:                       # sources lost before the call never take part
             if not e.alive:
-                sched.on_fail(e.oid, 0, self._delivered)
+                sched.on_fail(e.oid, 0, delivered)
         arrived = sorted((e for e in live if e.arrived), key=lambda e: (e.t_arrival, srcs.index(e.oid)))
         for e in arrived:
             sched.on_arrival(e.oid)
-        self.reduces[target] = {"sched": sched, "op": op, "srcs": list(srcs)}
         t = self.objects[target]          # the output is published at once, as a partial object
         t.arrived = True
         t.t_arrival = self.now
@@ -166,7 +170,8 @@ class OracleStore:
         for r in self.reduces.values():
             for e in lost:
                 if e.oid in r["srcs"]:
-                    r["sched"].on_fail(e.oid, e.ready_chunks, self._delivered)
+                    tgt = next(t for t, rr in self.reduces.items() if rr is r)
+                    r["sched"].on_fail(e.oid, self._delivered_in(e.oid, tgt), lambda o, tgt=tgt: self._delivered_in(o, tgt))
         for src, b in self.bcasts.items():
             mine = [e.oid for e in lost if e.oid == src or self.dst_of.get(e.oid) == src]
             if mine:
@@ -193,7 +198,7 @@ class OracleStore:
             sched: ReduceSchedule = r["sched"]
             if sched.k == 0:
                 raise StoreError(ERR_INSUFFICIENT)
-            if not sched.full() or any(self._delivered(m) < self.objects[m].C for m in sched.members()):
+            if not sched.full() or any(self._ready_elems(m) < self.objects[m].elems for m in sched.members()):
                 raise StoreError(ERR_TIMEOUT)
             key = self._membership(oid)
             if e.data is None or r.get("evaluated") != key:
@@ -243,14 +248,29 @@ class OracleStore:
             raise StoreError(ERR_NOT_FOUND)
         return self.objects[oid]
 
-    def _delivered(self, oid: int) -> int:
-        """Published chunk prefix: of a Put object what was put; of a Reduce output what its tree can produce."""
+    def _ready_elems(self, oid: int) -> int:
+        """Published element prefix: of a Put object what was put (whole chunks); of a Reduce output what its
+        tree can produce, i.e. the smallest prefix among its members once the tree is full."""
+        e = self.objects[oid]
         if oid in self.reduces:
             sched = self.reduces[oid]["sched"]
             if not sched.full():
                 return 0
-            return min(self._delivered(m) for m in sched.members())
-        return self.objects[oid].ready_chunks
+            return min(self._ready_elems(m) for m in sched.members())
+        return e.elems if e.complete else e.ready_chunks * e.chunk_elems
+
+    def _delivered(self, oid: int) -> int:
+        """The same prefix counted in the object's own chunks (chunk_bytes of its own dtype)."""
+        e = self.objects[oid]
+        n = self._ready_elems(oid)
+        return e.C if n >= e.elems else n // e.chunk_elems
+
+    def _delivered_in(self, oid: int, target: int) -> int:
+        """The same prefix counted in the chunks of the Reduce that produces ``target`` (chunk_bytes of its
+        input dtype: a bf16 Reduce works on twice as many elements per chunk as its fp32 output holds)."""
+        r = self.reduces[target]
+        n = self._ready_elems(oid)
+        return r["C"] if n >= self.objects[oid].elems else n // r["chunk_elems"]
 
     def _membership(self, oid: int) -> tuple:
         """Who is in the tree of ``oid``, and in the trees of the members that are Reduce outputs themselves."""

@@ -234,9 +234,15 @@ Object* find(hpl_ctx* c, int64_t id) {
     return it == c->objects.end() ? nullptr : &it->second;
 }
 
-// Chunk prefix an object has published, as the schedules see it: of a Put object what was put; of a Reduce
-// output (published when Reduce is called, Section 3.4.2) what its tree can already produce.
-int64_t logical_delivered(hpl_ctx* c, int64_t oid) {
+inline uint64_t object_elems(const Object& o) { return o.bytes / elem_size(o.dtype); }
+inline uint64_t object_chunk_elems(const hpl_ctx* c, const Object& o) {
+    return std::max<uint64_t>(1, std::min<uint64_t>(c->cfg.chunk_bytes, o.bytes) / elem_size(o.dtype));
+}
+
+// Element prefix an object has published, as the schedules see it: of a Put object what was put (whole
+// chunks); of a Reduce output (published when Reduce is called, Section 3.4.2) what its tree can already
+// produce, i.e. the smallest prefix among its members once the tree is full.
+uint64_t logical_ready_elems(hpl_ctx* c, int64_t oid) {
     Object* o = find(c, oid);
     if (!o) return 0;
     if (o->kind == OBJ_TARGET) {
@@ -244,20 +250,38 @@ int64_t logical_delivered(hpl_ctx* c, int64_t oid) {
         if (it == c->reduce_of_target.end()) return 0;
         ReduceTreeSchedule& s = *c->reduces.at(it->second).sched;
         if (!s.full()) return 0;
-        int64_t m = o->C;
-        for (int p = 0; p < s.k(); ++p) m = std::min(m, logical_delivered(c, s.object_at(p)));
+        uint64_t m = object_elems(*o);
+        for (int p = 0; p < s.k(); ++p) m = std::min(m, logical_ready_elems(c, s.object_at(p)));
         return m;
     }
-    return (int64_t)published_chunks(c, *o);
+    if (o->ready_bytes >= o->bytes) return object_elems(*o);
+    return (uint64_t)published_chunks(c, *o) * object_chunk_elems(c, *o);
 }
 
-// Chunks of a Reduce output that earlier waves on the stream have produced (or will have, by stream order).
-uint32_t produced_prefix(hpl_ctx* c, const Object& o) {
+// The same prefix counted in the object's own chunks (chunk_bytes of its own dtype) ...
+int64_t logical_delivered(hpl_ctx* c, int64_t oid) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    const uint64_t n = logical_ready_elems(c, oid);
+    return n >= object_elems(*o) ? (int64_t)o->C : (int64_t)(n / object_chunk_elems(c, *o));
+}
+
+// ... and in the chunks of a Reduce (chunk_bytes of its input dtype: a bf16 Reduce works on twice as many
+// elements per chunk as its fp32 output holds).
+int64_t logical_delivered_in(hpl_ctx* c, int64_t oid, const ReduceOp& op) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    const uint64_t n = logical_ready_elems(c, oid);
+    return n >= object_elems(*o) ? (int64_t)op.C : (int64_t)(n / op.chunk_elems);
+}
+
+// Elements of a Reduce output that earlier waves on the stream have produced (or will have, by stream order).
+uint64_t produced_elems(hpl_ctx* c, const Object& o) {
     auto it = c->reduce_of_target.find(o.id);
     if (it == c->reduce_of_target.end()) return 0;
     const ReduceOp& op = c->reduces.at(it->second);
     if (op.computed.empty() || op.computed[0].iv.empty() || op.computed[0].iv[0].first != 0) return 0;
-    return op.computed[0].iv[0].second;
+    return std::min<uint64_t>((uint64_t)op.computed[0].iv[0].second * op.chunk_elems, op.elems);
 }
 
 #define CUDA_TRY(x)                                  \
@@ -542,7 +566,8 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         Object* o = find(c, oid);
         if (!o || !o->alive || !o->ptr || o->row < 0) continue;
         if (o->kind == OBJ_TARGET) {   // composed Reduce: the member is the output of an earlier Reduce
-            landed[p] = ready[p] = produced_prefix(c, *o);
+            const uint64_t n = produced_elems(c, *o);
+            landed[p] = ready[p] = n >= op.elems ? op.C : (uint32_t)(n / op.chunk_elems);
         } else {
             const uint32_t pub = published_chunks(c, *o);
             landed[p] = std::min(pub, o->landed);
@@ -695,7 +720,8 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
     uint32_t src_landed = 0, src_avail = 0;
     if (src->alive && src->ptr && src->row >= 0) {
         if (src->kind == OBJ_TARGET) {   // reduce followed by broadcast: the source is a Reduce output
-            src_landed = src_avail = produced_prefix(c, *src);
+            const uint64_t n = produced_elems(c, *src);   // fp32 elements -> chunks of the broadcast (bytes of the object)
+            src_landed = src_avail = n * 4 >= src->bytes ? C : (uint32_t)(n * 4 / c->cfg.chunk_bytes);
         } else {
             src_landed = std::min(published_chunks(c, *src), src->landed);
             src_avail = c->cfg.plan_ahead ? C : src_landed;
@@ -918,8 +944,6 @@ int sync_and_check(hpl_ctx* c) {
 }
 
 int after_event(hpl_ctx* c) { return c->cfg.eager ? progress(c) : HPL_OK; }
-
-int64_t delivered_of(hpl_ctx* c, int64_t oid) { return logical_delivered(c, oid); }
 
 // After every event: a broadcast whose source is a Reduce output learns how far that output has got.
 void refresh_composed(hpl_ctx* c) {
@@ -1216,7 +1240,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     t.worker = -1;
     t.bytes = elems * 4;
     t.dtype = HPL_F32;
-    t.C = find(c, srcs[0])->C;
+    t.C = (uint32_t)((t.bytes + c->cfg.chunk_bytes - 1) / c->cfg.chunk_bytes);
     t.kind = OBJ_TARGET;
     t.lib_owned = true;
     t.arrived = true;   // the output is published at once, as a partial object (Section 3.4.2)
@@ -1240,11 +1264,12 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     r.red_op = op;
     r.in_dtype = dtype;
     r.elems = elems;
-    r.C = t.C;
+    r.C = find(c, srcs[0])->C;          // chunks of this Reduce follow its inputs (chunk_bytes of the input dtype)
     r.chunk_elems = (uint32_t)(std::min<uint64_t>(c->cfg.chunk_bytes, bytes) / elem_size(dtype));
     if (r.chunk_elems == 0) r.chunk_elems = 1;
     r.seq = c->seq++;
-    auto dl = [c](int64_t o) { return delivered_of(c, o); };
+    ReduceOp* rp = &r;
+    auto dl = [c, rp](int64_t o) { return logical_delivered_in(c, o, *rp); };
     for (int64_t s : srcs)
         if (!find(c, s)->alive) r.sched->fail(s, 0, dl);  // sources lost before the call never take part
     std::vector<std::pair<std::pair<int64_t, int>, int64_t>> arrived;
@@ -1319,12 +1344,13 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
         if (kv.second.worker == worker && kv.second.alive) lost.push_back(&kv.second);
     std::sort(lost.begin(), lost.end(), [](Object* a, Object* b) { return a->seq < b->seq; });
     for (Object* o : lost) o->alive = false;
-    auto dl = [c](int64_t o) { return delivered_of(c, o); };
     for (auto& kv : c->reduces) {
         ReduceOp& op = kv.second;
+        ReduceOp* rp = &op;
+        auto dl = [c, rp](int64_t o) { return logical_delivered_in(c, o, *rp); };
         for (Object* o : lost) {
             if (!op.sched->has_source(o->id)) continue;
-            ReduceInvalidation inv = op.sched->fail(o->id, (int64_t)published_chunks(c, *o), dl);
+            ReduceInvalidation inv = op.sched->fail(o->id, logical_delivered_in(c, o->id, op), dl);
             apply_invalidation(op, inv);
             if (!inv.positions.empty() || inv.shrank) invalidate_consumers(c, op.target);
         }
@@ -1362,7 +1388,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (!op.sched->full()) return HPL_ERR_TIMEOUT;
         for (int p = 0; p < op.sched->k(); ++p) {
             Object* m = find(c, op.sched->object_at(p));
-            if (!m || logical_delivered(c, m->id) < (int64_t)m->C) return HPL_ERR_TIMEOUT;
+            if (!m || logical_ready_elems(c, m->id) < object_elems(*m)) return HPL_ERR_TIMEOUT;
         }
         if (!c->device) return HPL_ERR_CUDA;
         if (!op.computed[0].contains(0, op.C)) return HPL_ERR_TIMEOUT;
