@@ -105,7 +105,7 @@ def test_upstream_failure_voids_what_was_derived_from_the_output():
     p.join(60)
     p.check_target_bits(200)
     p.check_receiver_bytes(60)
-    p.advance(100)
+    p.advance(p.o.now + 100)                           # the Get let virtual time run
     p.fail(1)                                          # a member of the first Reduce; object 5 is the spare
     rc, _, _ = p.c.try_get(60)
     assert rc == hpl.HPL_ERR_TIMEOUT
