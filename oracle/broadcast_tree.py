@@ -156,8 +156,9 @@ class BroadcastSchedule:
     # ---- events
     def join(self, t: int, dst_obj: int) -> None:
         self.advance(t)
-        if dst_obj in self.by_obj:
+        if dst_obj in self.by_obj and self.by_obj[dst_obj].alive:
             return    # a request for this copy is already in flight: just wait for it
+        # (a receiver whose worker failed and was rebuilt simply asks again, Section 3.5.1: a new location)
         r = Location(dst_obj, len(self.locs), slots=self.d, t_join=t)
         self.locs.append(r)
         self.by_obj[dst_obj] = r

@@ -43,6 +43,23 @@ def ancestors(p: int, d: int) -> list[int]:
     return out
 
 
+def choose_degree(n: int, size_bytes: float, latency: float, bandwidth: float) -> int:
+    """Eq. 1 and Section 4: among d = 1, 2 and n, the degree with the smallest estimated reduce time
+    ``T(1) = n L + S/B``, ``T(d) = L log_d n + d S/B``.  Ties go to the smaller degree."""
+    import math
+    if n <= 1:
+        return 1
+    t1 = n * latency + size_bytes / bandwidth
+    t2 = latency * math.log2(n) + 2.0 * size_bytes / bandwidth
+    tn = latency + n * size_bytes / bandwidth          # log_n n = 1
+    best, d = t1, 1
+    if t2 < best:
+        best, d = t2, 2
+    if tn < best:
+        best, d = tn, n
+    return d
+
+
 def inorder(k: int, d: int) -> list[int]:
     """Positions of the complete d-ary tree on k nodes in generalised in-order."""
     out: list[int] = []
@@ -135,6 +152,15 @@ class ReduceSchedule:
             self.spares.append(obj)
         else:
             self._assign(obj, p)
+
+    def on_rejoin(self, obj: int) -> None:
+        """A failed source was reconstructed (Section 3.5): it is a future again and will count as a new
+        arrival when it is put again ("R7 can also be the rejoined R2", Section 3.5.2).  A tree that has
+        shrunk in the meantime does not grow back."""
+        if obj in self.alive and not self.alive[obj]:
+            self.alive[obj] = True
+            if obj in self.arrived:
+                self.arrived.remove(obj)
 
     def on_fail(self, obj: int, delivered_chunks: int, delivered_of=None) -> None:
         """``obj`` is lost.  ``delivered_chunks`` is its published chunk prefix; ``delivered_of(o)``

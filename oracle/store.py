@@ -178,6 +178,20 @@ class OracleStore:
                 b["sched"].fail(self.now, mine)
         self._refresh_composed()
 
+    def rejoin(self, worker: int) -> None:
+        """The task framework has reconstructed a failed worker (Section 3.5): its objects are futures again.
+        A Reduce counts each as a new arrival once it is put again; a receiver may Get (join) again."""
+        for e in self.objects.values():
+            if e.worker == worker and not e.alive and e.oid not in self.bcasts:
+                e.alive = True
+                e.arrived = False
+                e.data = None
+                e.ready_bytes = 0
+                e.t_arrival = -1
+                for r in self.reduces.values():
+                    if e.oid in r["srcs"]:
+                        r["sched"].on_rejoin(e.oid)
+
     def delete(self, oid: int) -> None:
         self._entry(oid)
         if oid in self.dst_of or any(oid in r["srcs"] for r in self.reduces.values()):

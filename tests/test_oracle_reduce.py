@@ -335,3 +335,51 @@ def test_composed_reduce_redoes_the_downstream_after_an_upstream_failure():
         st.get(200)
     st.put(5, data[5], 256)
     assert np.array_equal(st.get(200), data[0] + data[5] + data[2] + data[3])
+
+
+# ---------------------------------------------------------------- rejoin (Section 3.5) and degree choice (Eq. 1)
+def test_rejoined_source_counts_as_a_new_arrival():
+    # "R7 can also be the rejoined R2": reduce 6 of 6, R2 fails, is rebuilt and put again
+    s = rt.ReduceSchedule(list(range(6)), 6, 2)
+    for o in range(6):
+        s.on_arrival(o)
+    pos = s.pos_of[1]
+    s.on_fail(1, 2, lambda o: 4)
+    assert s.k == 5                                   # no spare: the tree shrank (build-defined)
+    s.on_rejoin(1)
+    s.on_arrival(1)
+    assert s.spares == [1] and s.live_count() == 6    # it does not grow back; the source waits as a spare
+    s2 = rt.ReduceSchedule(list(range(7)), 6, 2)      # with a seventh source still to come the position stays open
+    for o in range(6):
+        s2.on_arrival(o)
+    s2.on_fail(1, 2, lambda o: 4)
+    assert not s2.full() and s2.k == 6
+    s2.on_rejoin(1)
+    s2.on_arrival(1)
+    assert s2.full() and s2.pos_of[1] == pos          # the rebuilt R2 takes its old position back
+    st, data = _store_with(4, 3, 2)
+    st.reduce(100, [0, 1, 2, 3], 4)
+    for o in range(4):
+        st.put(o, data[o], 256)
+    st.fail(2)
+    assert np.array_equal(st.get(100), data[0] + data[1] + data[3])
+    st.rejoin(2)
+    with pytest.raises(StoreError) as ei:
+        st.get(2)
+    assert ei.value.code == ERR_TIMEOUT               # a future again
+    st.put(2, data[2], 256)
+    assert np.array_equal(st.get(100), data[0] + data[1] + data[3])   # the shrunk tree is complete without it
+
+
+def test_degree_choice_follows_eq_1():
+    L, B = 100e-6, 1.25e9                             # 100 us, 10 Gbit/s
+    # the three closed forms of Section 3.4.2
+    for n in (2, 4, 8, 16):
+        for S in (1e3, 1e6, 1e9):
+            t = {1: n * L + S / B, 2: L * math.log2(n) + 2 * S / B, n: L + n * S / B}
+            want = min(sorted(t), key=lambda d: (t[d], d))
+            assert rt.choose_degree(n, S, L, B) == want
+    assert rt.choose_degree(16, 1e3, L, B) == 16      # small objects: latency dominates, d = n
+    assert rt.choose_degree(16, 1e9, L, B) == 1       # large objects: bandwidth dominates, the chain
+    assert rt.choose_degree(16, 4e5, L, B) == 2       # in between
+    assert rt.choose_degree(1, 1e6, L, B) == 1
