@@ -57,7 +57,8 @@ typedef struct hpl_ctx hpl_ctx;
 typedef struct hpl_config {
     uint64_t chunk_bytes;     /* pipelining block (Section 3.3; 4 MB in the paper).  Multiple of 16.  An object
                                  smaller than this is one chunk. */
-    int32_t  reduce_degree;   /* d of the reduce tree, >= 1 (Section 3.4.2, Eq. 1) */
+    int32_t  reduce_degree;   /* d of the reduce tree, >= 1 (Section 3.4.2, Eq. 1); 0 = chosen per Reduce among 1, 2 and
+                                 k by Eq. 1 from model_latency_ns and model_bandwidth_bps (Section 4) */
     int32_t  bcast_degree;    /* concurrent sends per location, >= 1 (1 = the rule of Section 3.4.1) */
     uint64_t virt_chunk_ns;   /* virtual time for one chunk to cross one broadcast edge; 0 = chunk_bytes at 64 GiB/s */
     uint64_t poll_budget_ns;  /* bound on any device-side wait; 0 = 2 s */
@@ -72,6 +73,8 @@ typedef struct hpl_config {
                                  targets and copies of host objects; owned by the caller, must outlive the
                                  context.  NULL = schedule-only context (no device work; hpl_get fails). */
     uint64_t arena_bytes;
+    uint64_t model_latency_ns;     /* L of Eq. 1: latency of one hop; used only when reduce_degree == 0 */
+    uint64_t model_bandwidth_bps;  /* B of Eq. 1: bytes per second into one node; used only when reduce_degree == 0 */
 } hpl_config;
 
 /* Creates a context.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Nothing is
@@ -133,6 +136,18 @@ int hpl_get_host(hpl_ctx* ctx, int64_t object_id, void* dst, uint64_t cap);
  * position, ancestors' partial results are cleared; with no spare left the tree shrinks.  Broadcast: the
  * receivers it was sending to ask again and resume from what they hold. */
 int hpl_fail(hpl_ctx* ctx, int32_t worker);
+
+/* The task framework has reconstructed failed worker `worker` (Section 3.5: "we want to allow a recovered
+ * task to rejoin"): the objects it owns are futures again -- not arrived, empty, to be Put again -- and the
+ * receivers it owns may hpl_join again (a new location).  A Reduce counts a re-Put source as a new arrival:
+ * it takes an open position or waits as a spare; a tree that shrank does not grow back.  A broadcast whose
+ * SOURCE was lost is not revived.  Waits for enqueued work (directory rows are recycled). */
+int hpl_rejoin(hpl_ctx* ctx, int32_t worker);
+
+/* Eq. 1 / Section 4: the degree among 1, 2 and n with the smallest estimated reduce time
+ * T(1) = n L + S/B, T(d) = L log_d n + d S/B (ties: the smaller degree).  Returns the degree (>= 1), or
+ * HPL_ERR_INVALID.  Pure function: needs no context. */
+int32_t hpl_choose_degree(int32_t n, uint64_t object_bytes, double latency_s, double bandwidth_bytes_per_s);
 
 /* Delete (Table 1): drops the directory entry (and the collective it names, if it is a reduce target or a
  * broadcast source).  Library-owned memory returns to the arena; caller buffers may then be freed. */

@@ -20,7 +20,7 @@ from __future__ import annotations
 import numpy as np
 
 from .broadcast_tree import BroadcastSchedule
-from .reduce_tree import ReduceSchedule
+from .reduce_tree import ReduceSchedule, choose_degree
 from .values import OP_SUM, tree_reduce
 
 OK = 0
@@ -59,9 +59,12 @@ class _Entry:
 
 
 class OracleStore:
-    def __init__(self, chunk_bytes: int, reduce_degree: int, bcast_degree: int, virt_chunk_ns: int = 0):
+    def __init__(self, chunk_bytes: int, reduce_degree: int, bcast_degree: int, virt_chunk_ns: int = 0,
+                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0):
         self.chunk_bytes = chunk_bytes
-        self.d_reduce = reduce_degree
+        self.d_reduce = reduce_degree      # 0: chosen per Reduce by Eq. 1 from the two model parameters
+        self.model_latency_ns = model_latency_ns
+        self.model_bandwidth_bps = model_bandwidth_bps
         self.d_bcast = bcast_degree
         # default virtual chunk time: chunk_bytes at 64 GiB/s, in whole nanoseconds
         self.tau = virt_chunk_ns if virt_chunk_ns > 0 else max(1, chunk_bytes * 1_000_000_000 // (64 << 30))
@@ -122,7 +125,10 @@ class OracleStore:
             raise StoreError(ERR_INSUFFICIENT)
         elems = ents[0].nbytes // _ELEM[dtype]
         self.create(target, -1, elems * 4, DT_F32)
-        sched = ReduceSchedule(srcs, k, self.d_reduce)
+        d = self.d_reduce
+        if d == 0:
+            d = choose_degree(k, float(ents[0].nbytes), self.model_latency_ns * 1e-9, float(self.model_bandwidth_bps))
+        sched = ReduceSchedule(srcs, k, d)
         self.reduces[target] = {"sched": sched, "op": op, "srcs": list(srcs), "chunk_elems": ents[0].chunk_elems,
                                 "C": ents[0].C}
         delivered = lambda o: self._delivered_in(o, target)

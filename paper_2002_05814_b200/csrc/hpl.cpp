@@ -1018,7 +1018,8 @@ const char* hpl_strerror(int code) {
 
 int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
     if (!cfg || !out) return HPL_ERR_INVALID;
-    if (cfg->chunk_bytes == 0 || cfg->chunk_bytes % 16 || cfg->reduce_degree < 1 || cfg->bcast_degree < 1) return HPL_ERR_INVALID;
+    if (cfg->chunk_bytes == 0 || cfg->chunk_bytes % 16 || cfg->reduce_degree < 0 || cfg->bcast_degree < 1) return HPL_ERR_INVALID;
+    if (cfg->reduce_degree == 0 && (cfg->model_latency_ns == 0 || cfg->model_bandwidth_bps == 0)) return HPL_ERR_INVALID;
     hpl_ctx* c = new (std::nothrow) hpl_ctx();
     if (!c) return HPL_ERR_NOMEM;
     c->cfg = *cfg;
@@ -1260,7 +1261,10 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
 
     ReduceOp r;
     r.target = target;
-    r.sched.reset(new ReduceTreeSchedule(srcs, k, c->cfg.reduce_degree));
+    int degree = c->cfg.reduce_degree;
+    if (degree == 0)   // Section 4: picked per Reduce from the latency / bandwidth model and the object size
+        degree = choose_reduce_degree(k, (double)bytes, (double)c->cfg.model_latency_ns * 1e-9, (double)c->cfg.model_bandwidth_bps);
+    r.sched.reset(new ReduceTreeSchedule(srcs, k, degree));
     r.red_op = op;
     r.in_dtype = dtype;
     r.elems = elems;
@@ -1327,7 +1331,8 @@ int hpl_join(hpl_ctx* c, int64_t dst_id, void* dst_buf) {
     if (!d->alive) return HPL_ERR_FAILED_WORKER;
     if (c->device && (!dst_buf || (uintptr_t)dst_buf % 16)) return HPL_ERR_INVALID;
     BcastOp& b = c->bcasts.at(c->bcast_of_src.at(d->op_key));
-    if (b.sched->index_of(dst_id) < 0) {
+    const int li = b.sched->index_of(dst_id);
+    if (li < 0 || !b.sched->locations()[li].alive) {   // first join, or again after its worker was rebuilt
         d->ptr = dst_buf;
         d->ready_bytes = 0;
         int rc = alloc_row(c, *d);
@@ -1364,6 +1369,42 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
     }
     refresh_composed(c);
     return after_event(c);
+}
+
+int hpl_rejoin(hpl_ctx* c, int32_t worker) {
+    if (!c || worker < 0) return HPL_ERR_INVALID;
+    bool any = false;
+    for (auto& kv : c->objects) {
+        Object& o = kv.second;
+        if (o.worker == worker && !o.alive && !c->bcast_of_src.count(o.id)) any = true;
+    }
+    if (!any) return HPL_OK;
+    if (c->device) {   // rows and store copies of the revived objects are recycled: nothing may still read them
+        cudaStreamSynchronize(c->ctl_stream);
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamSynchronize(c->stream);
+    }
+    for (auto& kv : c->objects) {
+        Object& o = kv.second;
+        if (o.worker != worker || o.alive || c->bcast_of_src.count(o.id)) continue;
+        release_object_memory(c, o);
+        o.alive = true;
+        o.arrived = false;
+        o.ready_bytes = 0;
+        o.landed = 0;
+        o.t_arrival = -1;
+        o.lib_owned = false;
+        o.from_host = false;
+        o.async_counter = false;
+        for (auto& rk : c->reduces)
+            if (rk.second.sched->has_source(o.id)) rk.second.sched->rejoin(o.id);
+    }
+    return after_event(c);
+}
+
+int32_t hpl_choose_degree(int32_t n, uint64_t object_bytes, double latency_s, double bandwidth_bytes_per_s) {
+    if (n < 1 || !(latency_s >= 0.0) || !(bandwidth_bytes_per_s > 0.0)) return HPL_ERR_INVALID;
+    return choose_reduce_degree(n, (double)object_bytes, latency_s, bandwidth_bytes_per_s);
 }
 
 int hpl_progress(hpl_ctx* c) {

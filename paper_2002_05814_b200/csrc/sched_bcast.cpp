@@ -128,7 +128,11 @@ void BroadcastTreeSchedule::serve_waiting(int64_t t) {
 
 void BroadcastTreeSchedule::join(int64_t t, int64_t dst_obj) {
     advance(t);
-    if (index_.count(dst_obj)) return;  // a request for this copy is already in flight
+    {
+        auto it = index_.find(dst_obj);
+        if (it != index_.end() && locs_[it->second].alive) return;  // a request for this copy is already in flight
+        // (a receiver whose worker failed and was rebuilt asks again: a new location)
+    }
     BcastLocation r;
     r.obj = dst_obj;
     r.slots = d_;

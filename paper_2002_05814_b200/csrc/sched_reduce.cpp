@@ -1,6 +1,7 @@
 #include "sched_reduce.h"
 
 #include <algorithm>
+#include <cmath>
 
 namespace hpl {
 
@@ -27,6 +28,21 @@ std::vector<int> generalised_inorder(int k, int d) {
     }
     inorder_rec(0, k, d, out);
     return out;
+}
+
+int choose_reduce_degree(int n, double size_bytes, double latency_s, double bandwidth_bytes_per_s) {
+    if (n <= 1) return 1;
+    const double chain = n * latency_s + size_bytes / bandwidth_bytes_per_s;
+    const double binary = latency_s * std::log2((double)n) + 2.0 * size_bytes / bandwidth_bytes_per_s;
+    const double star = latency_s + n * size_bytes / bandwidth_bytes_per_s;   // log_n n = 1
+    double best = chain;
+    int d = 1;
+    if (binary < best) {
+        best = binary;
+        d = 2;
+    }
+    if (star < best) d = n;
+    return d;
 }
 
 ReduceTreeSchedule::ReduceTreeSchedule(const std::vector<int64_t>& srcs, int k, int d)
@@ -89,6 +105,13 @@ void ReduceTreeSchedule::arrive(int64_t obj) {
         spares_.push_back(obj);
     else
         assign(obj, p);
+}
+
+void ReduceTreeSchedule::rejoin(int64_t obj) {
+    auto it = alive_.find(obj);
+    if (it == alive_.end() || it->second) return;
+    it->second = true;
+    arrived_.erase(obj);
 }
 
 ReduceInvalidation ReduceTreeSchedule::fail(int64_t obj, int64_t delivered,

@@ -50,6 +50,7 @@ public:
 
     // events; each returns the positions whose materialised results are no longer valid
     void arrive(int64_t obj);
+    void rejoin(int64_t obj);   // a failed source was reconstructed: a future again, a new arrival when put again
     ReduceInvalidation fail(int64_t obj, int64_t delivered_chunks, const std::function<int64_t(int64_t)>& delivered_of);
 
     void dump(int64_t target, std::vector<int64_t>& w) const;
@@ -72,6 +73,9 @@ private:
     std::vector<std::pair<int64_t, int>> placements_;
     std::vector<ReduceEdit> edits_;
 };
+
+// Eq. 1 / Section 4: the degree among 1, 2 and n with the smallest estimated reduce time (ties: the smaller).
+int choose_reduce_degree(int n, double size_bytes, double latency_s, double bandwidth_bytes_per_s);
 
 // Positions of the complete d-ary tree on k nodes in generalised in-order.
 std::vector<int> generalised_inorder(int k, int d);

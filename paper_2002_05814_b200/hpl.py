@@ -28,7 +28,8 @@ class Config(C.Structure):
     _fields_ = [("chunk_bytes", C.c_uint64), ("reduce_degree", C.c_int32), ("bcast_degree", C.c_int32),
                 ("virt_chunk_ns", C.c_uint64), ("poll_budget_ns", C.c_uint64), ("eager", C.c_int32),
                 ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
-                ("arena", C.c_void_p), ("arena_bytes", C.c_uint64)]
+                ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
+                ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64)]
 
 
 class Stats(C.Structure):
@@ -77,6 +78,7 @@ def load_library():
         "hpl_get": [VP, I64, P(VP), P(U64)],
         "hpl_get_host": [VP, I64, VP, U64],
         "hpl_fail": [VP, I32],
+        "hpl_rejoin": [VP, I32],
         "hpl_delete": [VP, I64],
         "hpl_progress": [VP],
         "hpl_sync": [VP],
@@ -89,6 +91,8 @@ def load_library():
         fn.restype = C.c_int
     lib.hpl_reduce_noalloc.argtypes = [P(VP), I32, I32, I32, I32, U64, VP, VP]
     lib.hpl_reduce_noalloc.restype = C.c_int
+    lib.hpl_choose_degree.argtypes = [I32, U64, C.c_double, C.c_double]
+    lib.hpl_choose_degree.restype = I32
     lib.hpl_strerror.argtypes = [C.c_int]
     lib.hpl_strerror.restype = C.c_char_p
     _LIB = lib
@@ -111,10 +115,12 @@ class Context:
 
     def __init__(self, chunk_bytes: int, reduce_degree: int = 2, bcast_degree: int = 2, *, arena=0,
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
-                 eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False):
+                 eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False,
+                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
-                     int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes)
+                     int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes,
+                     model_latency_ns, model_bandwidth_bps)
         self._h = C.c_void_p()
         self._p, self._n = C.c_void_p(), C.c_uint64()
         self._pref, self._nref = C.byref(self._p), C.byref(self._n)
@@ -192,6 +198,9 @@ class Context:
     def fail(self, worker: int):
         self._check(self._lib.hpl_fail(self._h, worker), "hpl_fail")
 
+    def rejoin(self, worker: int):
+        self._check(self._lib.hpl_rejoin(self._h, worker), "hpl_rejoin")
+
     def delete(self, object_id: int):
         self._check(self._lib.hpl_delete(self._h, object_id), "hpl_delete")
 
@@ -227,3 +236,8 @@ def reduce_noalloc(src_ptrs, degree: int, op: int, dtype: int, elems: int, out_p
     lib = load_library()
     arr = (C.c_void_p * len(src_ptrs))(*src_ptrs)
     return lib.hpl_reduce_noalloc(arr, len(src_ptrs), degree, op, dtype, elems, C.c_void_p(out_ptr), C.c_void_p(stream or None))
+
+
+def choose_degree(n: int, object_bytes: int, latency_s: float, bandwidth_bytes_per_s: float) -> int:
+    """``hpl_choose_degree``: Eq. 1's best degree among 1, 2 and n."""
+    return load_library().hpl_choose_degree(n, object_bytes, latency_s, bandwidth_bytes_per_s)

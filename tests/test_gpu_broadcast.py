@@ -125,3 +125,31 @@ def test_get_before_join_and_before_source_times_out():
     p.put(0)
     p.check_receiver_bytes(1)
     p.close()
+
+
+def test_rebuilt_receiver_asks_again():
+    nbytes, chunk = 32 * 4096, 4096
+    p = Pair(chunk, 2, 1, tau=100)
+    p.create(0, 99, gen(("uniform",), 8, 0, nbytes // 4))
+    for j in range(1, 5):
+        p.create(j, j, nbytes=nbytes, dtype=DT_F32)
+    p.put(0)
+    p.broadcast(0, [1, 2, 3, 4])
+    for j in (1, 2, 3):
+        p.advance(j * 120)
+        p.join(j)
+    p.progress()
+    p.advance(1000)
+    p.fail(2)
+    p.advance(1500)
+    p.c.rejoin(2)
+    p.o.rejoin(2)
+    p.dev[2] = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    p.advance(1600)
+    p.join(2)
+    p.join(4)
+    p.check_schedule(0)
+    for j in (1, 2, 3, 4):
+        p.check_receiver_bytes(j)
+    p.check_schedule(0)
+    p.close()

@@ -268,3 +268,30 @@ def test_deep_and_wide_trees():
         p.reduce(1000, list(range(k)), k)
         p.check_target_bits(1000)
         p.close()
+
+
+def test_rebuilt_worker_rejoins_as_a_new_arrival():
+    elems = 20_000
+    p = Pair(16 << 10, 2)
+    for i in range(7):
+        p.create(i, i, gen(("uniform",), 33, i, elems))
+    p.reduce(100, list(range(7)), 6)
+    for i in range(6):
+        p.advance(i + 1)
+        p.put(i)
+    p.progress()
+    p.advance(10)
+    p.fail(1)                                  # the position stays open: a seventh source may still come
+    rc, _, _ = p.c.try_get(100)
+    assert rc == hpl.HPL_ERR_TIMEOUT
+    p.advance(20)
+    p.c.rejoin(1)
+    p.o.rejoin(1)
+    fresh = torch.from_numpy(p.host[1]).cuda()  # the rebuilt task puts its object again, from a new buffer
+    p.dev[1] = fresh
+    p.advance(30)
+    p.put(1)
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert _norm_err(got, ov.naive_sum_f64([0, 1, 2, 3, 4, 5], p.host)) <= 1e-5 * 3
+    p.close()

@@ -126,8 +126,16 @@ def _reduce_timeline(seed):
             prefix[i] = nb
             if nb == nbytes:
                 order.pop(0)
-        elif r < 0.85:
+        elif r < 0.82:
             p.both("fail", int(rng.integers(0, n_workers)))
+        elif r < 0.88:
+            wk = int(rng.integers(0, n_workers))
+            p.both("rejoin", wk)
+            for i in range(n):                      # a rebuilt worker's objects are futures again
+                if p.o.objects[i].worker == wk and p.o.objects[i].alive and not p.o.objects[i].arrived:
+                    prefix[i] = 0
+                    if i not in order:
+                        order.append(i)
         elif called:
             p.get(1000)
         if called:
@@ -173,8 +181,14 @@ def _bcast_timeline(seed):
         elif r < 0.6 and src_pref < nbytes:
             src_pref = nbytes if rng.random() < 0.5 else min(nbytes, src_pref + 64)
             p.put(0, src_pref)
-        elif r < 0.75:
+        elif r < 0.72:
             p.both("fail", int(rng.integers(0, n_workers)))
+        elif r < 0.8:
+            wk = int(rng.integers(0, n_workers))
+            p.both("rejoin", wk)
+            for j in range(1, R + 1):               # rebuilt receivers ask again
+                if p.o.objects[j].worker == wk and j not in joiners and rng.random() < 0.7:
+                    joiners.append(j)
         else:
             p.get(int(rng.integers(1, R + 1)))
             t = max(t, p.o.now)
@@ -249,3 +263,25 @@ def _composed_timeline(seed):
 def test_composed_schedules_match_on_random_timelines(block):
     for seed in range(block * 150, (block + 1) * 150):
         _composed_timeline(seed)
+
+
+def test_degree_choice_matches_the_oracle():
+    from oracle.reduce_tree import choose_degree
+    rng = np.random.default_rng(9)
+    for _ in range(3000):
+        n = int(rng.integers(1, 200))
+        S = int(10 ** rng.uniform(1, 10))
+        L = float(10 ** rng.uniform(-7, -2))
+        B = float(10 ** rng.uniform(8, 12))
+        assert hpl.choose_degree(n, S, L, B) == choose_degree(n, float(S), L, B)
+    # through the store: degree 0 means "choose per Reduce"
+    for nbytes, want in ((64, 4), (64 * 4096, 1)):
+        o = OracleStore(64, 0, 1, 0, model_latency_ns=1000, model_bandwidth_bps=10**9)
+        c = hpl.Context(64, 0, 1, model_latency_ns=1000, model_bandwidth_bps=10**9)
+        for i in range(4):
+            o.create(i, i, nbytes, 0)
+            c.create(i, i, nbytes)
+        o.reduce(100, [0, 1, 2, 3], 4)
+        c.reduce(100, [0, 1, 2, 3], 4)
+        assert c.schedule_dump(100) == o.dump(100) and o.dump(100)[5] == want
+        c.shutdown()
