@@ -148,6 +148,14 @@ class Runner:
                 self.host_recv = torch.empty(S, dtype=torch.uint8).pin_memory()
             if n_src:
                 self.host_out = torch.empty(w.elems, dtype=torch.float32).pin_memory()
+        # argument arrays of the batch calls (events that share one time are submitted together)
+        C = self.ctx
+        self.a_dst_ids = C.ids_array([6000 + j for j in range(w.n_receivers)])
+        self.a_dst_workers = [1000 + j for j in range(w.n_receivers)]
+        self.a_dst_ptrs = C.ptr_array([t.data_ptr() for t in self.recv])
+        self.a_src_ids = C.ids_array(list(range(n_src)))
+        self.a_src_workers = list(range(n_src))
+        self.a_src_ptrs = C.ptr_array([t.data_ptr() for t in self.src])
         self.round = 0
         self.t = 0
         torch.cuda.synchronize()
@@ -173,8 +181,7 @@ class Runner:
                 h2d += S
             else:
                 ctx.put(src_id, self.policy.data_ptr(), S)
-            for j, dd in enumerate(dsts):
-                ctx.create(dd, 1000 + j, S, self.dt)
+            ctx.create_batch(self.a_dst_ids, self.a_dst_workers, S, self.dt)
             ctx.broadcast(src_id, dsts)
             if w.kind == "broadcast":
                 offs = wl.uniform_offsets_ns(w.seed + r, w.n_receivers, w.extra["join_window_ns"])
@@ -184,8 +191,7 @@ class Runner:
                     ctx.join(dsts[j], self.recv[j].data_ptr())
                 self.t += w.extra["join_window_ns"]
             else:
-                for j, dd in enumerate(dsts):
-                    ctx.join(dd, self.recv[j].data_ptr())
+                ctx.join_batch(self.a_dst_ids, self.a_dst_ptrs)
             for dd in dsts:
                 ctx.get(dd)
             if self.host_buffers:
@@ -199,8 +205,7 @@ class Runner:
             n = w.n_objects
             ids = [base + i for i in range(n)]
             tgt = base + 9000
-            for i in ids:
-                ctx.create(i, i, S, self.dt)
+            ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
             if w.kind == "reduce" and "mean_arrival_ns" in w.extra:
                 arr = wl.exponential_arrivals_ns(w.seed + r, n, w.extra["mean_arrival_ns"])
             else:
@@ -208,6 +213,9 @@ class Runner:
             order = sorted(range(n), key=lambda i: (arr[i], i))
             ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
             tmax = 0
+            if w.kind == "round" and not self.host_buffers:      # all returned objects are ready at once
+                ctx.put_batch(self.a_src_ids, self.a_src_ptrs, S)
+                order = []
             for i in order:
                 ctx.advance(max(self.t + arr[i], self.t + tmax))
                 tmax = max(tmax, arr[i])

@@ -106,6 +106,17 @@ int hpl_put(hpl_ctx* ctx, int64_t object_id, const void* buf, uint64_t bytes);
  * the copy overlap. */
 int hpl_put_host(hpl_ctx* ctx, int64_t object_id, const void* buf, uint64_t bytes);
 
+/* Many hpl_create / hpl_put / hpl_join calls at the current time, applied in array order exactly as the
+ * single calls would be (so: ascending ids for equal-time events).  Stops at the first failure and returns
+ * its code; *n_done (may be NULL) receives how many were applied.  They exist because a harness that stands
+ * for many workers otherwise pays a foreign-call round trip per object. */
+int hpl_create_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const int32_t* workers, uint64_t total_bytes,
+                     int32_t dtype, int32_t* n_done);
+int hpl_put_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const void* const* bufs /* host array of DEVICE
+                  pointers */, const uint64_t* bytes, int32_t* n_done);
+int hpl_join_batch(hpl_ctx* ctx, int32_t n, const int64_t* dst_ids, void* const* dst_bufs /* host array of DEVICE
+                   pointers */, int32_t* n_done);
+
 /* Reduce (Table 1, Section 3.4.2).  Non-blocking.  Creates `target_id` (fp32, library-owned, in the arena)
  * from `k_first_ready` of the `n` objects `src_ids` -- those that arrive first; ties by index in src_ids --
  * combined with `op` in the association order of the degree-d tree.  All sources have dtype `dtype` and one

@@ -1407,6 +1407,31 @@ int32_t hpl_choose_degree(int32_t n, uint64_t object_bytes, double latency_s, do
     return choose_reduce_degree(n, (double)object_bytes, latency_s, bandwidth_bytes_per_s);
 }
 
+int hpl_create_batch(hpl_ctx* c, int32_t n, const int64_t* ids, const int32_t* workers, uint64_t total_bytes, int32_t dtype,
+                     int32_t* n_done) {
+    if (!c || n < 0 || (n && (!ids || !workers))) return HPL_ERR_INVALID;
+    int rc = HPL_OK, i = 0;
+    for (; i < n && rc == HPL_OK; ++i) rc = hpl_create(c, ids[i], workers[i], total_bytes, dtype);
+    if (n_done) *n_done = rc == HPL_OK ? i : i - 1;
+    return rc;
+}
+
+int hpl_put_batch(hpl_ctx* c, int32_t n, const int64_t* ids, const void* const* bufs, const uint64_t* bytes, int32_t* n_done) {
+    if (!c || n < 0 || (n && (!ids || !bufs || !bytes))) return HPL_ERR_INVALID;
+    int rc = HPL_OK, i = 0;
+    for (; i < n && rc == HPL_OK; ++i) rc = hpl_put(c, ids[i], bufs[i], bytes[i]);
+    if (n_done) *n_done = rc == HPL_OK ? i : i - 1;
+    return rc;
+}
+
+int hpl_join_batch(hpl_ctx* c, int32_t n, const int64_t* ids, void* const* bufs, int32_t* n_done) {
+    if (!c || n < 0 || (n && (!ids || !bufs))) return HPL_ERR_INVALID;
+    int rc = HPL_OK, i = 0;
+    for (; i < n && rc == HPL_OK; ++i) rc = hpl_join(c, ids[i], bufs[i]);
+    if (n_done) *n_done = rc == HPL_OK ? i : i - 1;
+    return rc;
+}
+
 int hpl_progress(hpl_ctx* c) {
     if (!c) return HPL_ERR_INVALID;
     return progress(c);

@@ -72,6 +72,9 @@ def load_library():
         "hpl_create": [VP, I64, I32, U64, I32],
         "hpl_put": [VP, I64, VP, U64],
         "hpl_put_host": [VP, I64, VP, U64],
+        "hpl_create_batch": [VP, I32, P(I64), P(I32), U64, I32, P(I32)],
+        "hpl_put_batch": [VP, I32, P(I64), P(VP), P(U64), P(I32)],
+        "hpl_join_batch": [VP, I32, P(I64), P(VP), P(I32)],
         "hpl_reduce": [VP, I64, P(I64), I32, I32, I32, I32],
         "hpl_broadcast": [VP, I64, P(I64), I32],
         "hpl_join": [VP, I64, VP],
@@ -157,6 +160,31 @@ class Context:
         rc = self._lib.hpl_put(self._h, object_id, dev_buf if type(dev_buf) is int else _addr(dev_buf), nbytes)
         if rc:
             raise HplError(rc, "hpl_put")
+
+    # batch forms: the arrays may be prepared once (``ids_array`` etc.) and reused
+    @staticmethod
+    def ids_array(ids):
+        return (C.c_int64 * len(ids))(*ids)
+
+    @staticmethod
+    def ptr_array(ptrs):
+        return (C.c_void_p * len(ptrs))(*ptrs)
+
+    def create_batch(self, ids, workers, total_bytes: int, dtype: int = HPL_F32):
+        ids = ids if isinstance(ids, C.Array) else self.ids_array(ids)
+        wk = workers if isinstance(workers, C.Array) else (C.c_int32 * len(workers))(*workers)
+        self._check(self._lib.hpl_create_batch(self._h, len(ids), ids, wk, total_bytes, dtype, None), "hpl_create_batch")
+
+    def put_batch(self, ids, dev_ptrs, nbytes):
+        ids = ids if isinstance(ids, C.Array) else self.ids_array(ids)
+        ptrs = dev_ptrs if isinstance(dev_ptrs, C.Array) else self.ptr_array(dev_ptrs)
+        nb = nbytes if isinstance(nbytes, C.Array) else (C.c_uint64 * len(ids))(*([nbytes] * len(ids) if isinstance(nbytes, int) else nbytes))
+        self._check(self._lib.hpl_put_batch(self._h, len(ids), ids, ptrs, nb, None), "hpl_put_batch")
+
+    def join_batch(self, ids, dev_ptrs):
+        ids = ids if isinstance(ids, C.Array) else self.ids_array(ids)
+        ptrs = dev_ptrs if isinstance(dev_ptrs, C.Array) else self.ptr_array(dev_ptrs)
+        self._check(self._lib.hpl_join_batch(self._h, len(ids), ids, ptrs, None), "hpl_join_batch")
 
     def put_host(self, object_id: int, host_buf, nbytes: int):
         self._check(self._lib.hpl_put_host(self._h, object_id, C.c_void_p(_addr(host_buf)), nbytes), "hpl_put_host")

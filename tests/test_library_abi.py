@@ -69,3 +69,30 @@ def test_error_strings_and_argument_checks():
         with pytest.raises(hpl.HplError) as ei:
             c.put_host(1, bytearray(256), 256)
         assert ei.value.code in (hpl.HPL_ERR_CUDA, hpl.HPL_ERR_INVALID)
+
+
+def test_batch_calls_are_the_single_calls_in_array_order():
+    with hpl.Context(chunk_bytes=64) as a, hpl.Context(chunk_bytes=64) as b:
+        ids, workers, ptrs = [5, 3, 9, 4], [0, 1, 2, 3], [4096, 8192, 12288, 16384]
+        a.create_batch(ids, workers, 256)
+        for i, w in zip(ids, workers):
+            b.create(i, w, 256)
+        a.reduce(100, ids, 3)
+        b.reduce(100, ids, 3)
+        a.put_batch(ids, ptrs, [256, 128, 256, 64])
+        for i, p, n in zip(ids, ptrs, [256, 128, 256, 64]):
+            b.put(i, p, n)
+        assert a.schedule_dump(100) == b.schedule_dump(100)
+        for ctx in (a, b):
+            ctx.create(50, 7, 256)
+            ctx.create(51, 8, 256)
+            ctx.broadcast(5, [50, 51])
+        a.join_batch([50, 51], [20480, 24576])
+        b.join(50, 20480)
+        b.join(51, 24576)
+        assert a.schedule_dump(5) == b.schedule_dump(5)
+        with pytest.raises(hpl.HplError) as ei:
+            a.create_batch([60, 5], [0, 0], 256)        # the second id exists: the first was still created
+        assert ei.value.code == hpl.HPL_ERR_EXISTS
+        with pytest.raises(hpl.HplError):
+            a.create(60, 0, 256)
