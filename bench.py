@@ -35,6 +35,11 @@ import workloads as wl  # noqa: E402
 MiB = 1 << 20
 FALLBACK_HBM_GBS = 6650.0
 
+# dram__bytes_read.sum + dram__bytes_write.sum per full-size launch, from the ncu captures summarised in
+# profiles/ (taken on objects shrunk 4x and scaled by the elements processed; traffic is proportional).
+# Valid only for the kernels as captured: set an entry to None when its kernel changes.
+NCU_TRAFFIC = {"cfg4": {"reduce": 4.4227e9, "fanout": 4.1236e9}}
+
 
 # ----------------------------------------------------------------------------------------- helpers
 def measured_peak():
@@ -304,6 +309,62 @@ def whole_job_value(step_bytes, steps, world, total_ms):
     return gbs(step_bytes * steps * world, total_ms)
 
 
+def realtime_rounds(device, rounds: int = 8):
+    """The asynchrony view of the paper's Fig. 8 on the async-SGD shape (cfg3): objects are put at their real
+    arrival offsets (the host waits), every event lets the library run what has become runnable, and the
+    figure is the time from the k-th arrival -- the last one the Reduce needs -- until the caller holds the
+    result.  Early arrivals are reduced while the later ones are still on their way."""
+    import torch
+    import paper_2002_05814_b200 as hpl
+
+    w = wl.workload("cfg3")
+    S = w.object_bytes
+    arena = torch.empty(64 * MiB + 10 * w.elems * 4, dtype=torch.uint8, device=device)
+    out = {}
+    for eager in (True, False):
+        ctx = hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=arena.data_ptr(), arena_bytes=arena.numel(),
+                          stream=torch.cuda.current_stream().cuda_stream, eager=eager)
+        src = [wl.values_torch(w.dist, w.seed + i, i, 0, w.elems, "f32", device=device) for i in range(w.n_objects)] if eager else src_keep
+        src_keep = src
+        torch.cuda.synchronize()
+        lat, tail_bytes = [], []
+        t_base = 0
+        for r in range(rounds + 1):
+            arr = wl.exponential_arrivals_ns(w.seed + r, w.n_objects, w.extra["mean_arrival_ns"])
+            order = sorted(range(w.n_objects), key=lambda i: (arr[i], i))
+            t_base += 1_000_000_000
+            ctx.advance(t_base)
+            ids = list(range(w.n_objects))
+            ctx.create_batch(ids, ids, S)
+            ctx.reduce(9000, ids, w.k)
+            t0 = time.perf_counter_ns()
+            b0 = 0
+            for n, i in enumerate(order[:w.k]):            # the spares arrive later and are not needed
+                while time.perf_counter_ns() - t0 < arr[i]:
+                    pass
+                ctx.advance(t_base + arr[i])
+                if n == w.k - 1:
+                    st = ctx.stats()
+                    b0 = st["bytes_read_planned"] + st["bytes_written_planned"]
+                    t_last = time.perf_counter_ns()
+                ctx.put(i, src[i].data_ptr(), S)
+            ctx.get(9000)
+            t_done = time.perf_counter_ns()
+            st = ctx.stats()
+            if r > 0:                                      # the first round warms up
+                lat.append((t_done - t_last) / 1e3)
+                tail_bytes.append(st["bytes_read_planned"] + st["bytes_written_planned"] - b0)
+            for i in [9000] + ids:
+                ctx.delete(i)
+        ctx.shutdown()
+        out["eager" if eager else "lazy"] = {"latency_after_last_needed_arrival_us": float(np.mean(lat)),
+                                             "std_us": float(np.std(lat)), "bytes_moved_in_that_tail": float(np.mean(tail_bytes)),
+                                             "rounds": rounds}
+    out["note"] = ("eager: every Put also runs what became runnable (partial results of complete subtrees); lazy: everything "
+                   "is planned at the Get, one fused pass over the 8 members")
+    return out
+
+
 def gbs(nbytes, ms):
     return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
@@ -379,6 +440,7 @@ def main():
     ap.add_argument("--ft-mode", default="eager", choices=["eager", "lazy"],
                     help="cfg5: 'eager' runs hpl_progress before the failure (chunks delivered by every worker are reduced, "
                          "then partly redone); 'lazy' applies the compressed timeline and plans at the Get")
+    ap.add_argument("--realtime", action="store_true", help="also measure cfg3 with puts at their real arrival offsets")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads measured briefly and reported under 'also'")
@@ -444,17 +506,18 @@ def main():
     peak, peak_kind = measured_peak()
     st = res["stats"]
 
-    def roof(kind_ns, kind_launches, per_launch_bytes):
+    def roof(kind_ns, kind_launches, per_launch_bytes, traffic=None):
         if st[kind_launches] == 0:
             return None
         avg_ms = st[kind_ns] / st[kind_launches] / 1e6
         ach = gbs(per_launch_bytes, avg_ms)
-        return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": None,
+        return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": traffic,
                 "peak_kind": f"of {peak_kind} (copy bandwidth)", "avg_launch_ms": avg_ms, "launches": st[kind_launches],
                 "algorithmic_bytes_per_launch": per_launch_bytes, "frac_of_8TBs_nominal": ach / 8000.0}
 
-    r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * args.steps / max(1, st["reduce_launches"])) if ab["reduce"] else None
-    r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * args.steps / max(1, st["fanout_launches"])) if ab["broadcast"] else None
+    traf = NCU_TRAFFIC.get(w.name, {}) if args.shrink == 1 else {}
+    r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * args.steps / max(1, st["reduce_launches"]), traf.get("reduce")) if ab["reduce"] else None
+    r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * args.steps / max(1, st["fanout_launches"]), traf.get("fanout")) if ab["broadcast"] else None
     line = {"metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value, "unit": "GB/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -496,6 +559,9 @@ def main():
             also[nm] = {"GBps": g, "ms_per_step": float(np.mean(r2["total_ms"])), "kernel_GBps": kern,
                         "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / 5}
         line["also"] = also
+
+    if rank == 0 and world == 1 and args.realtime:
+        line["realtime_cfg3"] = realtime_rounds(device)
 
     if not args.no_e2e:
         e_steps = max(1, min(args.steps, 3))
