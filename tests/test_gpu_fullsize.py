@@ -181,7 +181,7 @@ def test_cfg4_policy_round_bf16():
     c.shutdown()
 
 
-@pytest.mark.parametrize("size", [64 << 20, 4 << 20])
+@pytest.mark.parametrize("size", [64 << 20, 4 << 20, 1 << 30])
 def test_cfg5_fault_tolerant_reduce(size):
     w = wl.cfg5_at(size)
     S = w.object_bytes

@@ -259,9 +259,11 @@ def test_reduce_with_missing_source_times_out_then_completes():
     p.close()
 
 
-def test_deep_and_wide_trees():
+@pytest.mark.parametrize("fuse", [True, False])
+def test_deep_and_wide_trees(fuse):
+    # unfused, 200 members give ~100 tasks on some levels: more than one wave holds, so launches are split
     for k, d in ((64, 1), (64, 64), (200, 2), (100, 3)):
-        p = Pair(8 << 10, d, arena_bytes=64 << 20)
+        p = Pair(8 << 10, d, arena_bytes=64 << 20, fuse=fuse)
         for i in range(k):
             p.create(i, i, gen(("uniform",), 6, i, 6000))
             p.put(i)
