@@ -38,7 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per full-size launch, from the ncu captures summarised in
 # profiles/ (taken on objects shrunk 4x and scaled by the elements processed; traffic is proportional).
 # Valid only for the kernels as captured: set an entry to None when its kernel changes.
-NCU_TRAFFIC = {"cfg4": {"reduce": 4.4227e9, "fanout": 4.1236e9}}
+NCU_TRAFFIC = {"cfg4": {"reduce": 4.4227e9, "fanout": 4.1236e9},     # shrunk 4x, scaled
+               "cfg2": {"fanout": 1.0780e9}, "cfg3": {"reduce": 0.9077e9}}          # captured at full size
 
 
 # ----------------------------------------------------------------------------------------- helpers
