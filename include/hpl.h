@@ -202,7 +202,7 @@ typedef struct hpl_stats_t {
     uint64_t fanout_launches;      /* launches of the fan-out kernel */
     uint64_t reduce_kernel_ns;     /* summed device time of reduce launches (time_kernels = 1; updated by waits) */
     uint64_t fanout_kernel_ns;
-    uint64_t reserved[1];
+    uint64_t device_waits;         /* polls of a progress counter that did not succeed at the first look (updated by waits) */
 } hpl_stats_t;
 
 int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);

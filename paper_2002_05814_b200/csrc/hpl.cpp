@@ -11,7 +11,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
-#include <cstdio>
+#include <cstddef>
 #include <cstring>
 #include <map>
 #include <memory>
@@ -932,10 +932,12 @@ int sync_and_check(hpl_ctx* c) {
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->work_in_flight = false;
     collect_kernel_times(c);
+    c->stats.device_waits = c->h_status->waits;
     if (c->h_status->error) {
         c->stats.device_timeouts++;
         undo_journal(c);
-        CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus), c->stream));
+        // clear the error record but keep the running count of waits
+        CUDA_TRY(cudaMemsetAsync(c->d_status, 0, offsetof(DeviceStatus, waits), c->stream));
         CUDA_TRY(cudaStreamSynchronize(c->stream));
         return HPL_ERR_TIMEOUT;
     }

@@ -91,9 +91,6 @@ __device__ __forceinline__ unsigned int meta_code(unsigned int m) { return m & 3
 __device__ __forceinline__ unsigned int meta_acc(unsigned int m) { return (m >> 2) & 7u; }
 __device__ __forceinline__ bool meta_is_bf16(unsigned int m) { return (m & 32u) != 0; }
 
-__device__ __forceinline__ void cp_async16(unsigned int smem_addr, unsigned long long gaddr) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gaddr) : "memory");
-}
 __device__ __forceinline__ void cp_async16_partial(unsigned int smem_addr, unsigned long long gaddr, unsigned int src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gaddr), "r"(src_bytes) : "memory");
 }

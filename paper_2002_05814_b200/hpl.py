@@ -38,8 +38,7 @@ class Stats(C.Structure):
                                           "bytes_read_planned", "bytes_written_planned", "device_timeouts",
                                           "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
                                           "reduce_launches", "fanout_launches", "reduce_kernel_ns",
-                                          "fanout_kernel_ns")] + \
-               [("reserved", C.c_uint64 * 1)]
+                                          "fanout_kernel_ns", "device_waits")]
 
 
 class HplError(RuntimeError):
@@ -254,7 +253,7 @@ class Context:
     def stats(self) -> dict:
         st = Stats()
         self._check(self._lib.hpl_stats(self._h, C.byref(st)), "hpl_stats")
-        return {name: getattr(st, name) for name, _ in Stats._fields_ if name != "reserved"}
+        return {name: getattr(st, name) for name, _ in Stats._fields_}
 
 
 def reduce_noalloc(src_ptrs, degree: int, op: int, dtype: int, elems: int, out_ptr: int, stream: int = 0) -> int:

@@ -119,3 +119,63 @@ def test_a_wait_nothing_ends_runs_out_and_the_context_stays_usable():
     p.check_target_bits(100)
     assert p.c.sync() == hpl.HPL_OK
     p.close()
+
+
+def test_eager_mode_runs_what_became_runnable_at_every_event():
+    k, elems = 8, 30_000
+    p = Pair(32 << 10, 2, 2, eager=True)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 74, i, elems))
+    for j in range(3):
+        p.create(50 + j, 20 + j, nbytes=elems * 4, dtype=DT_F32)
+    p.reduce(100, list(range(k)), k)
+    p.broadcast(100, [50, 51, 52])
+    p.join(50)
+    launches = []
+    for t, i in enumerate([2, 5, 0, 7, 1, 3, 6, 4]):
+        p.advance(t + 1)
+        p.put(i)                                   # no explicit hpl_progress anywhere
+        launches.append(p.c.stats()["kernel_launches"])
+    assert launches[1] == 0 and launches[-1] > launches[2] >= 1      # subtrees were reduced as they completed
+    p.join(51)
+    p.join(52)
+    p.check_target_bits(100)
+    for j in range(3):
+        p.check_receiver_bytes(50 + j)
+    p.close()
+
+
+def test_delete_returns_memory_and_rows_for_the_next_round():
+    p = Pair(16 << 10, 2, 2, arena_bytes=8 << 20)       # room for one round only: every round must give it back
+    base = p.c.stats()["arena_used"]
+    for rnd in range(6):
+        ids = [10 * rnd + i for i in range(4)]
+        for i in ids:
+            p.create(i, i % 4, gen(("uniform",), 75 + rnd, i, 300_000))
+        p.reduce(1000 + rnd, ids, 4)
+        for i in ids:
+            p.put(i)
+            p.progress()
+        p.check_target_bits(1000 + rnd)
+        assert p.c.stats()["arena_used"] > base
+        for i in [1000 + rnd] + ids:
+            p.c.delete(i)
+            p.o.delete(i)
+        assert p.c.stats()["arena_used"] == base
+    p.close()
+
+
+def test_waits_are_counted():
+    p = Pair(16 << 10, 2, plan_ahead=True, poll_budget_ns=5_000_000_000)
+    for i in range(2):
+        p.create(i, i, gen(("uniform",), 76, i, 8 * 4096))
+    p.reduce(100, [0, 1], 2)
+    p.put(0)
+    p.put(1, 16 << 10)
+    p.progress()
+    import time
+    time.sleep(0.05)                                # the kernel is polling for chunk 1 of object 1
+    p.put(1)
+    p.check_target_bits(100)
+    assert p.c.stats()["device_waits"] >= 1 and p.c.stats()["device_timeouts"] == 0
+    p.close()
