@@ -136,7 +136,7 @@ def test_eager_mode_runs_what_became_runnable_at_every_event():
         p.advance(t + 1)
         p.put(i)                                   # no explicit hpl_progress anywhere
         launches.append(p.c.stats()["kernel_launches"])
-    assert launches[1] == 0 and launches[-1] > launches[2] >= 1      # subtrees were reduced as they completed
+    assert launches[0] == 0 and launches[1] >= 1 and launches[-1] > launches[1]   # subtrees are reduced as they complete
     p.join(51)
     p.join(52)
     p.check_target_bits(100)
