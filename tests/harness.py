@@ -25,9 +25,21 @@ class Pair:
         self.o = OracleStore(chunk_bytes, d_reduce, d_bcast, tau)
         self.host: dict[int, np.ndarray] = {}
         self.dev: dict[int, torch.Tensor] = {}
+        self.guarded: dict[int, torch.Tensor] = {}
+
+    GUARD = 256   # bytes of canary before and after every receiver buffer
 
     def close(self):
+        """Shuts the context down and checks what no test may violate: objects are immutable (the bytes of every
+        put object are unchanged) and nothing was written outside a receiver's buffer."""
         self.c.shutdown()
+        torch.cuda.synchronize()
+        for oid, a in self.host.items():
+            got = self.dev[oid].view(torch.uint8).cpu().numpy().tobytes() if oid in self.dev else None
+            assert got is None or got == a.tobytes(), f"object {oid} was modified"
+        for oid, (whole, nbytes) in self.guarded.items():
+            g = self.GUARD
+            assert bool((whole[:g] == 0x5C).all()) and bool((whole[g + nbytes:] == 0x5C).all()), f"write outside receiver {oid}"
 
     def advance(self, t):
         self.c.advance(t)
@@ -42,7 +54,11 @@ class Pair:
             nbytes = data.nbytes
         else:
             dt = dtype
-            self.dev[oid] = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")
+            pad = (-nbytes) % 16                       # keep the trailing canary 16-byte aligned after the buffer
+            whole = torch.full((nbytes + pad + 2 * self.GUARD,), 0x5C, dtype=torch.uint8, device="cuda")
+            whole[self.GUARD:self.GUARD + nbytes] = 0xA5
+            self.guarded[oid] = (whole, nbytes)
+            self.dev[oid] = whole[self.GUARD:self.GUARD + nbytes]
         self.c.create(oid, worker, nbytes, dt)
         self.o.create(oid, worker, nbytes, dt)
 
