@@ -481,9 +481,24 @@ void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial
     task.steps.push_back(st);
 }
 
-void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& dep_level) {
+// Nodes in the subtree of position q of the complete d-ary tree on k positions.
+int64_t subtree_size(const ReduceTreeSchedule& s, int q) {
+    int64_t total = 0, lo = q, hi = q;
+    const int64_t k = s.k(), d = s.d();
+    while (lo < k) {
+        total += std::min(hi, k - 1) - lo + 1;
+        lo = d * lo + 1;
+        hi = d * hi + d;
+    }
+    return total;
+}
+
+// `budget`: steps this subtree may still add to the task (a task must fit one wave's step table).  A child
+// subtree that does not fit beside its siblings is materialised by a task of its own first.
+void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& dep_level, int64_t budget) {
     ReduceTreeSchedule& s = *p.op->sched;
     auto is_materialised = [&](int q) { return !s.is_leaf(q) && (p.done[q] || p.level_of[q] >= 0); };
+    const int64_t begin = (int64_t)task.steps.size();
     task.n_acc = std::max(task.n_acc, acc + 1);
     if (s.is_leaf(u)) {
         emit_operand(p, task, u, false, OPC_LOAD, acc);
@@ -497,13 +512,18 @@ void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& d
         if (s.is_leaf(cj)) {
             emit_operand(p, task, cj, false, code, acc);
         } else {
-            if (!is_materialised(cj) && (!p.c->cfg.fuse || acc_j >= kMaxAcc)) ensure_result(p, cj);
+            // what the rest of this node still needs at least: its own object and one load per remaining child
+            const int64_t used = (int64_t)task.steps.size() - begin;
+            const int64_t reserve = (j == 0 ? 1 : 0) + 2 * (int64_t)(nc - 1 - j);
+            const int64_t avail = budget - used - reserve - 1;
+            const bool fits = 2 * subtree_size(s, cj) <= avail;
+            if (!is_materialised(cj) && (!p.c->cfg.fuse || acc_j >= kMaxAcc || !fits)) ensure_result(p, cj);
             if (p.err != HPL_OK) return;
             if (is_materialised(cj)) {
                 if (p.level_of[cj] > dep_level) dep_level = p.level_of[cj];
                 emit_operand(p, task, cj, true, code, acc);
             } else {
-                gen_steps(p, cj, acc_j, task, dep_level);
+                gen_steps(p, cj, acc_j, task, dep_level, avail);
                 if (j > 0) {
                     ReduceStep st{};
                     st.code = OPC_ADD_ACC;
@@ -535,7 +555,8 @@ int ensure_result(ReducePlanCtx& p, int v) {
     task.n_acc = 1;
     task.poll = false;
     int dep = 0;
-    gen_steps(p, v, 0, task, dep);
+    gen_steps(p, v, 0, task, dep, kMaxStepsPerWave);
+    if (p.err == HPL_OK && task.steps.size() > (size_t)kMaxStepsPerWave) p.err = HPL_ERR_INVALID;   // a node with more children than a task holds
     task.level = dep + 1;
     p.level_of[v] = task.level;
     p.out->push_back(std::move(task));
@@ -1270,6 +1291,12 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     int degree = c->cfg.reduce_degree;
     if (degree == 0)   // Section 4: picked per Reduce from the latency / bandwidth model and the object size
         degree = choose_reduce_degree(k, (double)bytes, (double)c->cfg.model_latency_ns * 1e-9, (double)c->cfg.model_bandwidth_bps);
+    if (std::min<int64_t>(degree, k - 1) + 2 > (int64_t)kMaxStepsPerWave) {   // one node's operands must fit one task
+        if (t.ptr) c->arena.release(t.ptr);
+        if (t.row >= 0) c->free_rows.push_back(t.row);
+        c->objects.erase(target);
+        return HPL_ERR_INVALID;
+    }
     r.sched.reset(new ReduceTreeSchedule(srcs, k, degree));
     r.red_op = op;
     r.in_dtype = dtype;

@@ -297,3 +297,24 @@ def test_rebuilt_worker_rejoins_as_a_new_arrival():
     got = p.check_target_bits(100).cpu().numpy()
     assert _norm_err(got, ov.naive_sum_f64([0, 1, 2, 3, 4, 5], p.host)) <= 1e-5 * 3
     p.close()
+
+
+def test_more_members_than_one_task_holds_are_cut_into_subtree_tasks():
+    for k, d in ((1000, 1), (700, 2), (500, 499)):
+        p = Pair(8 << 10, d, arena_bytes=64 << 20)
+        for i in range(k):
+            p.create(i, i % 7, gen(("smallint", 20), 44, i, 2500))
+            p.put(i)
+        p.reduce(5000, list(range(k)), k)
+        got = p.check_target_bits(5000).cpu().numpy()
+        assert np.array_equal(got.astype(np.float64), ov.naive_sum_f64(list(range(k)), p.host))
+        if k > 640:
+            assert p.c.stats()["reduce_tasks"] > 1
+        p.close()
+    p = Pair(8 << 10, 1000)
+    for i in range(800):
+        p.c.create(i, 0, 64)
+    with pytest.raises(hpl.HplError) as ei:
+        p.c.reduce(5000, list(range(800)), 800)       # a star with more operands than one task holds
+    assert ei.value.code == hpl.HPL_ERR_INVALID
+    p.c.shutdown()
