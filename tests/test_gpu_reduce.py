@@ -300,6 +300,8 @@ def test_rebuilt_worker_rejoins_as_a_new_arrival():
 
 
 def test_more_members_than_one_task_holds_are_cut_into_subtree_tasks():
+    import sys
+    sys.setrecursionlimit(10_000)          # the oracle evaluates a chain of 1000 recursively
     for k, d in ((1000, 1), (700, 2), (500, 499)):
         p = Pair(8 << 10, d, arena_bytes=64 << 20)
         for i in range(k):
