@@ -75,6 +75,70 @@ struct IntervalSet {  // disjoint, sorted [a, b) chunk ranges
     }
 };
 
+// Per tree position: for which chunks how many leading operands of the node (first child, own object, second
+// child, ...) have been merged into its result buffer.  All operands merged = the node's result is complete.
+struct IntervalMap {  // disjoint, sorted [a, b) -> value > 0
+    struct E { uint32_t a, b; int v; };
+    std::vector<E> iv;
+    void clear() { iv.clear(); }
+    int value_at(uint32_t c) const {
+        for (auto& x : iv)
+            if (x.a <= c && c < x.b) return x.v;
+        return 0;
+    }
+    void set(uint32_t a, uint32_t b, int v) {   // v == 0 erases
+        if (a >= b) return;
+        std::vector<E> out;
+        for (auto& x : iv) {
+            if (x.b <= a || b <= x.a) {
+                out.push_back(x);
+                continue;
+            }
+            if (x.a < a) out.push_back({x.a, a, x.v});
+            if (b < x.b) out.push_back({b, x.b, x.v});
+        }
+        if (v > 0) out.push_back({a, b, v});
+        std::sort(out.begin(), out.end(), [](const E& l, const E& r) { return l.a < r.a; });
+        iv.clear();
+        for (auto& x : out) {   // join neighbours with the same value
+            if (!iv.empty() && iv.back().b == x.a && iv.back().v == x.v)
+                iv.back().b = x.b;
+            else
+                iv.push_back(x);
+        }
+    }
+    void truncate_above(int j) {   // forget everything that has more than j operands merged
+        std::vector<E> out;
+        for (auto& x : iv)
+            if (x.v <= j) out.push_back(x);
+        iv.swap(out);
+    }
+    void breakpoints(std::vector<uint32_t>& bp) const {
+        for (auto& x : iv) {
+            bp.push_back(x.a);
+            bp.push_back(x.b);
+        }
+    }
+    uint32_t full_prefix(int full) const {   // end of the run of complete chunks that starts at chunk 0
+        uint32_t end = 0;
+        for (auto& x : iv) {
+            if (x.a != end || x.v != full) break;
+            end = x.b;
+        }
+        return end;
+    }
+    bool covers(uint32_t a, uint32_t b, int full) const {
+        uint32_t at = a;
+        for (auto& x : iv) {
+            if (x.b <= at) continue;
+            if (x.a > at || x.v != full) return false;
+            at = x.b;
+            if (at >= b) return true;
+        }
+        return at >= b;
+    }
+};
+
 struct Arena {
     uint8_t* base = nullptr;
     uint64_t size = 0, used = 0;
@@ -149,7 +213,7 @@ struct Object {
 };
 
 struct Journal {  // what was planned since the last successful sync (undone if a device wait expires)
-    struct R { int64_t target; int pos; uint32_t a, b; };
+    struct R { int64_t target; int pos; uint32_t a, b; int old_v; };
     struct B { int64_t src; int loc; int64_t old_have; };
     std::vector<R> r;
     std::vector<B> b;
@@ -158,6 +222,7 @@ struct Journal {  // what was planned since the last successful sync (undone if 
 
 struct PlannedReduceTask {
     int pos;
+    int end;      // operands of the position merged once this task has run
     int level;
     uint32_t a, b;
     int n_acc;
@@ -172,7 +237,8 @@ struct ReduceOp {
     uint64_t elems;
     uint32_t C, chunk_elems;
     uint64_t seq;
-    std::vector<IntervalSet> computed;      // per position: chunks of its result that are materialised and valid
+    std::vector<IntervalMap> merged;        // per position: chunks -> leading operands merged into its buffer (valid ones only)
+    int n_ops(int pos) const { return sched->n_children(pos) + 1; }
     std::vector<int64_t> partial_key;       // per position: internal object id of its partial buffer (0 none)
 };
 
@@ -280,8 +346,8 @@ uint64_t produced_elems(hpl_ctx* c, const Object& o) {
     auto it = c->reduce_of_target.find(o.id);
     if (it == c->reduce_of_target.end()) return 0;
     const ReduceOp& op = c->reduces.at(it->second);
-    if (op.computed.empty() || op.computed[0].iv.empty() || op.computed[0].iv[0].first != 0) return 0;
-    return std::min<uint64_t>((uint64_t)op.computed[0].iv[0].second * op.chunk_elems, op.elems);
+    if (op.merged.empty()) return 0;
+    return std::min<uint64_t>((uint64_t)op.merged[0].full_prefix(op.n_ops(0)) * op.chunk_elems, op.elems);
 }
 
 #define CUDA_TRY(x)                                  \
@@ -423,8 +489,10 @@ struct ReducePlanCtx {
     uint32_t a, b;                 // chunk interval being planned
     std::vector<uint32_t> ready;   // per position: chunks that may be consumed
     std::vector<uint32_t> landed;  // per position: chunks known to be visible without polling
-    std::vector<char> done, avail;
-    std::vector<int> level_of;     // level at which the position's result becomes available in this pass
+    std::vector<int> m0;           // per position: operands already merged into its buffer over [a, b)
+    std::vector<int> prefix;       // per position: operands that could be merged now (>= m0)
+    std::vector<char> full, avail; // result complete already / could be completed now
+    std::vector<int> level_of;     // level at which the position's complete result becomes available in this pass
     std::vector<PlannedReduceTask>* out;
     int err = HPL_OK;
 };
@@ -460,11 +528,9 @@ int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out) {
     return HPL_OK;
 }
 
-// Emits the steps that leave the result of subtree `u` in accumulator `acc`.  Children that cannot be
-// fused (fusion switched off, or no accumulator left) are materialised first by tasks of a lower level.
-int ensure_result(ReducePlanCtx& p, int v);
+int ensure_result(ReducePlanCtx& p, int v, int end);
 
-// One load step: the position's own object (partial == false) or its materialised partial result.
+// One load step: the position's own object (partial == false) or the buffer that holds its (partial) result.
 void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial, uint8_t code, int acc) {
     ReduceOp& op = *p.op;
     ReduceStep st{};
@@ -472,7 +538,7 @@ void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial
     st.a = (uint8_t)acc;
     if (partial) {
         st.kind = SRC_F32;
-        st.row = (uint32_t)find(p.c, op.partial_key[q])->row;
+        st.row = (uint32_t)find(p.c, q == 0 ? op.target : op.partial_key[q])->row;
     } else {
         st.kind = op.in_dtype == HPL_BF16 ? SRC_BF16 : SRC_F32;
         st.row = (uint32_t)find(p.c, op.sched->object_at(q))->row;
@@ -493,38 +559,52 @@ int64_t subtree_size(const ReduceTreeSchedule& s, int q) {
     return total;
 }
 
-// `budget`: steps this subtree may still add to the task (a task must fit one wave's step table).  A child
-// subtree that does not fit beside its siblings is materialised by a task of its own first.
-void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& dep_level, int64_t budget) {
+// Operand i of an internal node u, in the association order of the tree: 0 = first child, 1 = the node's own
+// object, i >= 2 = child i-1.  Returns the child's position, or -1 for the own object.
+inline int operand_child(const ReduceTreeSchedule& s, int u, int i) { return i == 1 ? -1 : s.first_child(u) + (i == 0 ? 0 : i - 1); }
+inline int operand_index_of_child(const ReduceTreeSchedule& s, int u, int child) {
+    const int j = child - s.first_child(u);
+    return j == 0 ? 0 : j + 1;
+}
+
+// Emits the steps that merge operands [m0[u], end) of node u into accumulator `acc`, starting from the buffer
+// of u when some operands are merged already.  `budget`: steps this subtree may still add (a task must fit one
+// wave's step table).  A child subtree that cannot be fused (fusion off, no accumulator left, no room) is
+// completed by a task of its own first.
+void gen_steps(ReducePlanCtx& p, int u, int acc, int end, PlannedReduceTask& task, int& dep_level, int64_t budget) {
     ReduceTreeSchedule& s = *p.op->sched;
-    auto is_materialised = [&](int q) { return !s.is_leaf(q) && (p.done[q] || p.level_of[q] >= 0); };
+    auto is_complete = [&](int q) { return !s.is_leaf(q) && (p.full[q] || p.level_of[q] >= 0); };
     const int64_t begin = (int64_t)task.steps.size();
     task.n_acc = std::max(task.n_acc, acc + 1);
     if (s.is_leaf(u)) {
         emit_operand(p, task, u, false, OPC_LOAD, acc);
         return;
     }
-    const int c0 = s.first_child(u), nc = s.n_children(u);
-    for (int j = 0; j < nc; ++j) {
-        const int cj = c0 + j;
-        const int acc_j = j == 0 ? acc : acc + 1;            // where a fused subtree of this child would live
-        const uint8_t code = j == 0 ? OPC_LOAD : OPC_ADD_LOAD;
-        if (s.is_leaf(cj)) {
+    bool first = true;
+    if (p.m0[u] > 0) {   // continue from what the node's buffer already holds
+        emit_operand(p, task, u, true, OPC_LOAD, acc);
+        first = false;
+    }
+    for (int i = p.m0[u]; i < end; ++i) {
+        const uint8_t code = first ? OPC_LOAD : OPC_ADD_LOAD;
+        const int cj = operand_child(s, u, i);
+        if (cj < 0) {
+            emit_operand(p, task, u, false, code, acc);
+        } else if (s.is_leaf(cj)) {
             emit_operand(p, task, cj, false, code, acc);
         } else {
-            // what the rest of this node still needs at least: its own object and one load per remaining child
+            const int acc_j = first ? acc : acc + 1;   // where a fused subtree of this child would live
             const int64_t used = (int64_t)task.steps.size() - begin;
-            const int64_t reserve = (j == 0 ? 1 : 0) + 2 * (int64_t)(nc - 1 - j);
-            const int64_t avail = budget - used - reserve - 1;
-            const bool fits = 2 * subtree_size(s, cj) <= avail;
-            if (!is_materialised(cj) && (!p.c->cfg.fuse || acc_j >= kMaxAcc || !fits)) ensure_result(p, cj);
+            const int64_t avail = budget - used - 2 * (int64_t)(end - 1 - i) - 1;
+            const bool fits = 2 * subtree_size(s, cj) + 1 <= avail;
+            if (!is_complete(cj) && (!p.c->cfg.fuse || acc_j >= kMaxAcc || !fits)) ensure_result(p, cj, p.op->n_ops(cj));
             if (p.err != HPL_OK) return;
-            if (is_materialised(cj)) {
+            if (is_complete(cj)) {
                 if (p.level_of[cj] > dep_level) dep_level = p.level_of[cj];
                 emit_operand(p, task, cj, true, code, acc);
             } else {
-                gen_steps(p, cj, acc_j, task, dep_level, avail);
-                if (j > 0) {
+                gen_steps(p, cj, acc_j, p.op->n_ops(cj), task, dep_level, avail);
+                if (!first) {
                     ReduceStep st{};
                     st.code = OPC_ADD_ACC;
                     st.a = (uint8_t)acc;
@@ -533,14 +613,16 @@ void gen_steps(ReducePlanCtx& p, int u, int acc, PlannedReduceTask& task, int& d
                 }
             }
         }
-        if (j == 0) emit_operand(p, task, u, false, OPC_ADD_LOAD, acc);  // first child, then the node itself
+        first = false;
     }
 }
 
-// Plans the task that materialises the result of position v over [a, b); returns its level (>= 1).
-int ensure_result(ReducePlanCtx& p, int v) {
+// Plans the task that merges operands up to `end` into the buffer of position v over [a, b); returns the level
+// (>= 1) at which that buffer is ready.
+int ensure_result(ReducePlanCtx& p, int v, int end) {
     if (p.err != HPL_OK) return 0;
-    if (p.done[v]) return 0;
+    const bool complete = end == p.op->n_ops(v);
+    if (p.full[v]) return 0;
     if (p.level_of[v] >= 0) return p.level_of[v];
     Object* outbuf = nullptr;
     int rc = ensure_partial_buffer(p.c, *p.op, v, &outbuf);
@@ -550,28 +632,40 @@ int ensure_result(ReducePlanCtx& p, int v) {
     }
     PlannedReduceTask task;
     task.pos = v;
+    task.end = end;
     task.a = p.a;
     task.b = p.b;
     task.n_acc = 1;
     task.poll = false;
     int dep = 0;
-    gen_steps(p, v, 0, task, dep, kMaxStepsPerWave);
+    gen_steps(p, v, 0, end, task, dep, kMaxStepsPerWave);
     if (p.err == HPL_OK && task.steps.size() > (size_t)kMaxStepsPerWave) p.err = HPL_ERR_INVALID;   // a node with more children than a task holds
     task.level = dep + 1;
-    p.level_of[v] = task.level;
+    if (complete) p.level_of[v] = task.level;
     p.out->push_back(std::move(task));
-    return p.level_of[v];
+    return task.level;
 }
 
+// Whatever can run now: a node whose remaining operands are all available is completed (its whole ready
+// subtree fused into one task); otherwise the operands that are available, in order, are merged into its
+// buffer (each arriving part is reduced into the parent's partial result), and the search goes on below.
 void visit_for_progress(ReducePlanCtx& p, int v) {
     ReduceTreeSchedule& s = *p.op->sched;
-    if (s.is_leaf(v) || p.done[v]) return;
+    if (s.is_leaf(v) || p.full[v]) return;
     if (p.avail[v]) {
-        ensure_result(p, v);
+        ensure_result(p, v, p.op->n_ops(v));
         return;
     }
-    const int c0 = s.first_child(v), nc = s.n_children(v);
-    for (int j = 0; j < nc; ++j) visit_for_progress(p, c0 + j);
+    int merged = p.m0[v];
+    if (p.prefix[v] > p.m0[v] && p.prefix[v] >= 2) {
+        ensure_result(p, v, p.prefix[v]);
+        merged = p.prefix[v];
+    }
+    const int nops = p.op->n_ops(v);
+    for (int i = merged; i < nops; ++i) {
+        const int cj = operand_child(s, v, i);
+        if (cj >= 0) visit_for_progress(p, cj);
+    }
 }
 
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
@@ -581,7 +675,7 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
     std::vector<uint32_t> ready(k, 0), landed(k, 0);
     std::vector<uint32_t> bp = {0u, op.C};
     for (int p = 0; p < k; ++p) {
-        op.computed[p].breakpoints(bp);
+        op.merged[p].breakpoints(bp);
         const int64_t oid = s.object_at(p);
         if (oid < 0) continue;
         Object* o = find(c, oid);
@@ -609,34 +703,46 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         if (p.b > op.C) break;
         p.ready = ready;
         p.landed = landed;
-        p.done.assign(k, 0);
+        p.m0.assign(k, 0);
+        p.prefix.assign(k, 0);
+        p.full.assign(k, 0);
         p.avail.assign(k, 0);
         p.level_of.assign(k, -1);
         std::vector<PlannedReduceTask> local;
         p.out = &local;
-        for (int q = k - 1; q >= 0; --q) {
-            p.done[q] = op.computed[q].contains(p.a, p.b) ? 1 : 0;
-            bool av = ready[q] >= p.b;
-            if (!s.is_leaf(q)) {
-                const int c0 = s.first_child(q), nc = s.n_children(q);
-                for (int j = 0; j < nc && av; ++j) av = s.is_leaf(c0 + j) ? (ready[c0 + j] >= p.b) : (p.done[c0 + j] || p.avail[c0 + j]);
+        for (int q = k - 1; q >= 0; --q) {   // children have larger indices than their parent
+            const int nops = op.n_ops(q);
+            p.m0[q] = op.merged[q].value_at(p.a);
+            p.full[q] = p.m0[q] == nops ? 1 : 0;
+            if (s.is_leaf(q)) {
+                p.avail[q] = ready[q] >= p.b ? 1 : 0;
+                p.prefix[q] = p.avail[q] ? 1 : 0;
+                continue;
             }
-            p.avail[q] = av ? 1 : 0;
+            int m1 = p.m0[q];
+            while (m1 < nops) {
+                const int cj = operand_child(s, q, m1);
+                const bool ok = cj < 0 ? ready[q] >= p.b : (s.is_leaf(cj) ? ready[cj] >= p.b : (p.full[cj] || p.avail[cj]));
+                if (!ok) break;
+                ++m1;
+            }
+            p.prefix[q] = m1;
+            p.avail[q] = m1 == nops ? 1 : 0;
         }
         if (s.is_leaf(0)) {
             // k == 1: the target is a copy of the only member
-            if (!p.done[0] && p.avail[0]) ensure_result(p, 0);
+            if (!p.full[0] && p.avail[0]) ensure_result(p, 0, 1);
         } else {
             visit_for_progress(p, 0);
         }
         if (p.err != HPL_OK) return p.err;
         for (auto& t : local) {
-            op.computed[t.pos].add(t.a, t.b);
-            c->journal.r.push_back({op.target, t.pos, t.a, t.b});
+            c->journal.r.push_back({op.target, t.pos, t.a, t.b, p.m0[t.pos]});
+            op.merged[t.pos].set(t.a, t.b, t.end);
             // merge with the previous interval's task for the same position when the program is the same
             bool merged = false;
             for (auto& prev : tasks) {
-                if (prev.pos == t.pos && prev.b == t.a && prev.level == t.level && prev.poll == t.poll &&
+                if (prev.pos == t.pos && prev.end == t.end && prev.b == t.a && prev.level == t.level && prev.poll == t.poll &&
                     prev.steps.size() == t.steps.size() &&
                     std::memcmp(prev.steps.data(), t.steps.data(), t.steps.size() * sizeof(ReduceStep)) == 0) {
                     prev.b = t.b;
@@ -924,7 +1030,7 @@ void undo_journal(hpl_ctx* c) {
         auto it = c->reduce_of_target.find(e.target);
         if (it == c->reduce_of_target.end()) continue;
         ReduceOp& op = c->reduces.at(it->second);
-        if (e.pos < (int)op.computed.size()) op.computed[e.pos].remove(e.a, e.b);
+        if (e.pos < (int)op.merged.size()) op.merged[e.pos].set(e.a, e.b, e.old_v);
     }
     for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
         auto f = c->bcast_of_src.find(it->src);
@@ -981,7 +1087,7 @@ void invalidate_consumers(hpl_ctx* c, int64_t target) {
     for (auto& kv : c->reduces) {
         ReduceOp& op = kv.second;
         if (!op.sched->has_source(target)) continue;
-        for (auto& cs : op.computed) cs.clear();
+        for (auto& cs : op.merged) cs.clear();
         invalidate_consumers(c, op.target);
     }
     auto b = c->bcast_of_src.find(target);
@@ -991,14 +1097,22 @@ void invalidate_consumers(hpl_ctx* c, int64_t target) {
     }
 }
 
+// A position's own object changed, or the position disappeared: its buffer is void, and so is, in every
+// ancestor, whatever was merged from the child on that path onwards.  What an ancestor had merged BEFORE that
+// child (its earlier operands) is untouched and kept -- healthy chunks are not redone.
 void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv) {
     const int k = op.sched->k();
+    ReduceTreeSchedule& s = *op.sched;
     if (inv.shrank) {
-        op.computed.resize(k);
+        op.merged.resize(k);
         op.partial_key.resize(k, 0);
     }
-    for (int p : inv.positions)
-        if (p >= 0 && p < k) op.computed[p].clear();
+    for (int x : inv.touched) {
+        if (x < 0) continue;
+        if (x < k) op.merged[x].clear();
+        for (int child = x, u = s.parent(x); u >= 0; child = u, u = s.parent(u))
+            if (u < k) op.merged[u].truncate_above(operand_index_of_child(s, u, child));
+    }
 }
 
 void notify_arrival(hpl_ctx* c, Object& o) {
@@ -1316,7 +1430,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     }
     std::sort(arrived.begin(), arrived.end());
     for (auto& a : arrived) r.sched->arrive(a.second);
-    r.computed.assign(r.sched->k(), IntervalSet());
+    r.merged.assign(r.sched->k(), IntervalMap());
     r.partial_key.assign(r.sched->k(), 0);
     const uint64_t key = r.seq;
     c->reduce_of_target[target] = key;
@@ -1490,7 +1604,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
             if (!m || logical_ready_elems(c, m->id) < object_elems(*m)) return HPL_ERR_TIMEOUT;
         }
         if (!c->device) return HPL_ERR_CUDA;
-        if (!op.computed[0].contains(0, op.C)) return HPL_ERR_TIMEOUT;
+        if (!op.merged[0].covers(0, op.C, op.n_ops(0))) return HPL_ERR_TIMEOUT;
         rc = sync_and_check(c);
         if (rc != HPL_OK) return rc;
     } else if (o->kind == OBJ_RECEIVER) {

@@ -129,6 +129,7 @@ ReduceInvalidation ReduceTreeSchedule::fail(int64_t obj, int64_t delivered,
         at_[p] = -1;
         ++epoch_;
         inv.positions.push_back(p);
+        inv.touched.push_back(p);
         if (!spares_.empty()) {
             const int64_t s = spares_.front();
             spares_.erase(spares_.begin());
@@ -159,6 +160,7 @@ void ReduceTreeSchedule::shrink(int p, int64_t old_obj, int64_t hi_failed,
     --k_;
     at_.pop_back();
     inv.shrank = true;
+    inv.touched.push_back(q);
     int64_t dest = -1, hi_moved = 0, moved_from = -1, new_obj = -1;
     if (q != p && moved >= 0) {
         pos_.erase(moved);
@@ -169,6 +171,7 @@ void ReduceTreeSchedule::shrink(int p, int64_t old_obj, int64_t hi_failed,
             if (std::find(cleared.begin(), cleared.end(), a) == cleared.end()) cleared.push_back(a);
         assign(moved, (int)dest);
         new_obj = moved;
+        inv.touched.push_back((int)dest);
         if (std::find(inv.positions.begin(), inv.positions.end(), (int)dest) == inv.positions.end())
             inv.positions.push_back((int)dest);
     } else {

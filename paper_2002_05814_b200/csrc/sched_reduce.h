@@ -26,6 +26,7 @@ struct ReduceEdit {
 // What an edit means for materialised results: positions whose own partial must be recomputed.
 struct ReduceInvalidation {
     std::vector<int> positions;   // includes the vacated position itself and all cleared ancestors
+    std::vector<int> touched;     // positions whose own object changed or that disappeared (old numbering)
     bool shrank = false;          // the last position disappeared
 };
 

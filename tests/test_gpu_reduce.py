@@ -320,3 +320,58 @@ def test_more_members_than_one_task_holds_are_cut_into_subtree_tasks():
         p.c.reduce(5000, list(range(800)), 800)       # a star with more operands than one task holds
     assert ei.value.code == hpl.HPL_ERR_INVALID
     p.c.shutdown()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+@pytest.mark.parametrize("d", [2, 3, 4])
+def test_each_arrival_is_merged_into_its_parents_partial_result(d, fuse):
+    """Progress after every single arrival, degree up to 4: a node's buffer receives its operands in order
+    (first child, own object, the other children) as they become available, and the final pass only adds
+    what is still missing.  The bits must not depend on when the merging happened."""
+    k, elems, chunk = 13, 3 * 4096 + 5, 16 << 10
+    for order_seed in (0, 1):
+        p = Pair(chunk, d, fuse=fuse)
+        for i in range(k):
+            p.create(i, i, gen(("normal", 1e-3), 50 + order_seed, i, elems))
+        p.reduce(100, list(range(k)), k)
+        order = list(np.random.default_rng(order_seed).permutation(k))
+        reads = []
+        for t, i in enumerate(order):
+            p.advance(t + 1)
+            p.put(int(i))
+            p.progress()
+            reads.append(p.c.stats()["bytes_read_planned"])
+        p.check_schedule(100)
+        p.check_target_bits(100)
+        st = p.c.stats()
+        if fuse:
+            last_pass = st["bytes_read_planned"] - reads[-2]
+            assert last_pass < k * elems * 4 / 2          # most of the tree had been merged before the last arrival
+        p.close()
+
+
+def test_failure_keeps_what_ancestors_had_merged_before_the_lost_subtree():
+    """The root of a binary tree has merged (first child's result + own object) when a member of its SECOND
+    child's subtree fails: that partial result does not contain the lost object and must survive."""
+    k, elems = 7, 5 * 4096
+    p = Pair(16 << 10, 2)
+    for i in range(k + 1):
+        p.create(i, i, gen(("smallint", 100), 60, i, elems))
+    p.reduce(100, list(range(k + 1)), k)              # 7 of 8: object 7 is the spare
+    for t, i in enumerate(range(5)):                  # arrivals 0..4 fill the first child's subtree, the root and one more
+        p.advance(t + 1)
+        p.put(i)
+        p.progress()
+    before = p.c.stats()["bytes_read_planned"]
+    p.advance(10)
+    p.fail(4)                                         # sits below the root's second child
+    for t, i in enumerate((5, 6, 7)):
+        p.advance(20 + t)
+        p.put(i)
+        p.progress()
+    p.check_schedule(100)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert np.array_equal(got.astype(np.float64), ov.naive_sum_f64([0, 1, 2, 3, 5, 6, 7], p.host))
+    after = p.c.stats()["bytes_read_planned"]
+    assert after - before <= 5 * elems * 4            # the root's partial was read back, not rebuilt from objects 0..3
+    p.close()
