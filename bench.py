@@ -361,8 +361,8 @@ def realtime_rounds(device, rounds: int = 8):
         out["eager" if eager else "lazy"] = {"latency_after_last_needed_arrival_us": float(np.mean(lat)),
                                              "std_us": float(np.std(lat)), "bytes_moved_in_that_tail": float(np.mean(tail_bytes)),
                                              "rounds": rounds}
-    out["note"] = ("eager: every Put also runs what became runnable (partial results of complete subtrees); lazy: everything "
-                   "is planned at the Get, one fused pass over the 8 members")
+    out["note"] = ("eager: every Put also runs what became runnable (arrived operands are merged into their parents' partial "
+                   "results); lazy: everything is planned at the Get, one fused pass over the 8 members")
     return out
 
 
