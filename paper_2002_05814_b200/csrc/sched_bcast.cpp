@@ -36,8 +36,7 @@ void BroadcastTreeSchedule::source_progress(int64_t t, int64_t have) {
         s.complete = true;
         s.t_complete = t;
     }
-    const std::vector<int> rs = s.receivers;
-    for (int r : rs) try_start(r, t);
+    for (size_t i = 0; i < locs_[0].receivers.size(); ++i) try_start(locs_[0].receivers[i], t);
 }
 
 void BroadcastTreeSchedule::advance(int64_t t) {
@@ -77,8 +76,8 @@ void BroadcastTreeSchedule::land(int ri, int64_t t) {
     } else {
         try_start(ri, t);
     }
-    const std::vector<int> rs = locs_[ri].receivers;
-    for (int c : rs) try_start(c, t);
+    // (try_start never changes a receiver list, so no copy is needed)
+    for (size_t i = 0; i < locs_[ri].receivers.size(); ++i) try_start(locs_[ri].receivers[i], t);
 }
 
 bool BroadcastTreeSchedule::depends_on(int cand, int root) const {
