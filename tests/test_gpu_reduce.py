@@ -197,6 +197,10 @@ def test_cfg5_shape_worker_7_fails_after_40_percent(size, fuse):
         redo = after["bytes_read_planned"] - before["bytes_read_planned"]
         if not fuse:   # healthy partial results are kept: only the two root paths are recomputed below chunk h
             assert redo < 31 * size
+            # Section 3.5.2: at most log_d n nodes clear per touched position (two here: the vacated one and the
+            # one the last leaf moved away from), for each of the two chunk ranges (below / above the failure point)
+            redone_tasks = after["reduce_tasks"] - before["reduce_tasks"]
+            assert redone_tasks <= 2 * 2 * (math.ceil(math.log2(32)) + 1)
     p.close()
 
 
