@@ -198,6 +198,12 @@ class Runner:
                 self.t += w.extra["join_window_ns"]
             else:
                 ctx.join_batch(self.a_dst_ids, self.a_dst_ptrs)
+            if w.kind == "round" and not self.host_buffers:
+                # the Reduce of the objects the workers will return is requested with futures while the
+                # broadcast is still running (the pattern of the paper's Fig. 1)
+                ctx.progress()
+                ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
+                ctx.reduce(base + 9000, [base + i for i in range(w.n_objects)], w.k, self.hpl.HPL_SUM, self.dt)
             for dd in dsts:
                 ctx.get(dd)
             if self.host_buffers:
@@ -211,13 +217,16 @@ class Runner:
             n = w.n_objects
             ids = [base + i for i in range(n)]
             tgt = base + 9000
-            ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
+            early = w.kind == "round" and not self.host_buffers      # created and requested above
+            if not early:
+                ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
             if w.kind == "reduce" and "mean_arrival_ns" in w.extra:
                 arr = wl.exponential_arrivals_ns(w.seed + r, n, w.extra["mean_arrival_ns"])
             else:
                 arr = [0] * n
             order = sorted(range(n), key=lambda i: (arr[i], i))
-            ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
+            if not early:
+                ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
             tmax = 0
             if w.kind == "round" and not self.host_buffers:      # all returned objects are ready at once
                 ctx.put_batch(self.a_src_ids, self.a_src_ptrs, S)

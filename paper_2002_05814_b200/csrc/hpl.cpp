@@ -1612,6 +1612,11 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
         const int li = op.sched->index_of(id);
         if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
+        if (c->device && (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C)) {
+            // start the copies first: the GPU works while the host lets the virtual clock run below
+            int rc = progress(c);
+            if (rc != HPL_OK) return rc;
+        }
         if (!op.sched->run_until_complete(id)) return HPL_ERR_TIMEOUT;
         if ((uint64_t)op.sched->now() > c->now) c->now = (uint64_t)op.sched->now();
         for (auto& kv : c->bcasts) kv.second.sched->advance((int64_t)c->now);
