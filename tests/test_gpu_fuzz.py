@@ -1,0 +1,113 @@
+"""Random timelines on the GPU: puts in instalments, failures, rejoins, joins, composed collectives and
+explicit progress calls in random order, under random library flags.  Whenever the oracle can deliver an
+object the library must deliver the same bits; whenever it cannot, the library must say the same."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_05814_b200 as hpl
+from oracle.store import StoreError, OK, DT_F32
+from tests.harness import Pair, gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2002_05814_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _get_both(p: Pair, oid, plan_ahead):
+    ro, want = OK, None
+    try:
+        want = p.o.get(oid)
+    except StoreError as e:
+        ro = e.code
+    rl, ptr, n = p.c.try_get(oid)
+    if plan_ahead and ro == OK and rl == hpl.HPL_ERR_TIMEOUT:
+        p.c.sync()                                   # a polling kernel gave up earlier; its work is planned again
+        rl, ptr, n = p.c.try_get(oid)
+    assert rl == ro, (oid, ro, rl)
+    if ro == OK:
+        got = p.view(ptr, n).cpu().numpy().tobytes()
+        assert got == want.tobytes(), f"object {oid} differs"
+    if plan_ahead:
+        p.c.sync()
+
+
+def _timeline(seed):
+    rng = np.random.default_rng(seed)
+    na, nb, R = int(rng.integers(2, 9)), int(rng.integers(1, 5)), int(rng.integers(1, 5))
+    ka, kb = int(rng.integers(1, na + 1)), int(rng.integers(1, nb + 2))
+    d = int(rng.integers(1, 5))
+    chunk = int(rng.choice([4096, 16384]))
+    elems = int(rng.integers(1, 6)) * (chunk // 4) + int(rng.choice([0, 0, 3, 1000]))
+    plan_ahead = bool(rng.random() < 0.3)
+    flags = dict(fuse=bool(rng.random() < 0.6), eager=bool(rng.random() < 0.4), plan_ahead=plan_ahead,
+                 poll_budget_ns=3_000_000 if plan_ahead else 0)
+    p = Pair(chunk, d, int(rng.integers(1, 3)), tau=int(rng.integers(1, 50)), arena_bytes=32 << 20, **flags)
+    n = na + nb
+    nbytes = elems * 4
+    n_workers = max(1, int(rng.integers(1, n + 1)))
+    for i in range(n):
+        p.create(i, int(rng.integers(0, n_workers)), gen(("smallint", 30) if seed % 2 else ("uniform",), 1000 + seed, i, elems))
+    for j in range(R):
+        p.create(500 + j, 100 + int(rng.integers(0, 2)), nbytes=nbytes, dtype=DT_F32)
+    A, B = 1000, 2000
+    p.reduce(A, list(range(na)), ka)
+    p.reduce(B, [A] + list(range(na, n)), kb)
+    p.broadcast(B, [500 + j for j in range(R)])
+    prefix = {i: 0 for i in range(n)}
+    joiners = [500 + j for j in range(R)]
+    t = 0
+    for _ in range(int(rng.integers(2 * n, 6 * n + 8))):
+        t = max(t + int(rng.integers(0, 40)), p.o.now)
+        p.advance(t)
+        r = rng.random()
+        if r < 0.5:
+            i = int(rng.integers(0, n))
+            e = p.o.objects[i]
+            if e.alive:
+                nb_ = nbytes if rng.random() < 0.5 else min(nbytes, prefix[i] + chunk)
+                p.put(i, nb_)
+                prefix[i] = nb_
+        elif r < 0.6:
+            p.fail(int(rng.integers(0, n_workers)))
+        elif r < 0.66:
+            wk = int(rng.integers(0, n_workers))
+            p.c.rejoin(wk)
+            p.o.rejoin(wk)
+            for i in range(n):
+                if p.o.objects[i].worker == wk and p.o.objects[i].alive and not p.o.objects[i].arrived:
+                    prefix[i] = 0
+        elif r < 0.76 and joiners:
+            j = joiners.pop(0)
+            if p.o.objects[j].alive:
+                p.join(j)
+        elif r < 0.86:
+            p.progress()
+        else:
+            _get_both(p, int(rng.choice([A, B] + [500 + j for j in range(R)])), plan_ahead)
+            t = max(t, p.o.now)
+        for op in (A, B):
+            p.check_schedule(op)
+    for i in range(n):                                # let everything that is still alive complete
+        if p.o.objects[i].alive:
+            t = max(t + 5, p.o.now)
+            p.advance(t)
+            p.put(i, nbytes)
+    for oid in [A, B] + [500 + j for j in range(R)]:
+        _get_both(p, oid, plan_ahead)
+    p.check_schedule(A)
+    p.check_schedule(B)
+    if plan_ahead:
+        p.c.sync()
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(6))
+def test_random_timelines_match_the_oracle(block):
+    for seed in range(block * 25, (block + 1) * 25):
+        _timeline(seed)
