@@ -1030,7 +1030,9 @@ void undo_journal(hpl_ctx* c) {
         auto it = c->reduce_of_target.find(e.target);
         if (it == c->reduce_of_target.end()) continue;
         ReduceOp& op = c->reduces.at(it->second);
-        if (e.pos < (int)op.merged.size()) op.merged[e.pos].set(e.a, e.b, e.old_v);
+        // back to nothing, not to the earlier value: a task that gave up half way may have updated part of the
+        // buffer in place, so what it held before is gone as well
+        if (e.pos < (int)op.merged.size()) op.merged[e.pos].set(e.a, e.b, 0);
     }
     for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
         auto f = c->bcast_of_src.find(it->src);
