@@ -28,6 +28,7 @@ using namespace hpl;
 namespace {
 
 constexpr uint32_t kMaxRows = 4096;
+constexpr uint32_t kStatusSlots = 256;   // one error record per wave in flight; beyond that the last one is shared
 constexpr uint32_t kMaxChunks = 1u << 20;
 constexpr uint64_t kAlign = 256;
 
@@ -212,9 +213,10 @@ struct Object {
     int row = -1;
 };
 
-struct Journal {  // what was planned since the last successful sync (undone if a device wait expires)
-    struct R { int64_t target; int pos; uint32_t a, b; int old_v; };
-    struct B { int64_t src; int loc; int64_t old_have; };
+struct Journal {  // what was planned since the last successful wait (undone if a device wait expires)
+    // tag: number of waves launched before the planning pass that made the entry (its waves have seq >= tag)
+    struct R { int64_t target; int pos; uint32_t a, b; int old_v; uint64_t tag; };
+    struct B { int64_t src; int loc; int64_t old_have; uint64_t tag; };
     std::vector<R> r;
     std::vector<B> b;
     void clear() { r.clear(); b.clear(); }
@@ -278,6 +280,10 @@ struct hpl_ctx {
     std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
     Journal journal;
     bool work_in_flight = false;
+    uint64_t launch_seq = 0;       // waves launched so far
+    uint64_t first_unchecked = 0;  // the first wave whose error record has not been read back
+    uint64_t batch_tag = 0;        // launch_seq when the current planning pass began
+    std::vector<uint64_t> wave_tag;  // for the waves in flight (seq - first_unchecked): the tag of their planning pass
     hpl_stats_t stats{};
     int occ_reduce[2][3] = {{0, 0, 0}, {0, 0, 0}};
     int occ_fanout = 0;
@@ -430,6 +436,14 @@ int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
 
 int sync_and_check(hpl_ctx* c);
 int progress(hpl_ctx* c);
+
+// The error record of the wave that is about to be launched.
+DeviceStatus* next_wave_status(hpl_ctx* c) {
+    const uint64_t idx = c->launch_seq - c->first_unchecked;
+    c->wave_tag.push_back(c->batch_tag);
+    ++c->launch_seq;
+    return c->d_status + std::min<uint64_t>(idx, kStatusSlots - 1);
+}
 
 cudaEvent_t take_event(hpl_ctx* c) {
     if (!c->event_pool.empty()) {
@@ -737,7 +751,7 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         }
         if (p.err != HPL_OK) return p.err;
         for (auto& t : local) {
-            c->journal.r.push_back({op.target, t.pos, t.a, t.b, p.m0[t.pos]});
+            c->journal.r.push_back({op.target, t.pos, t.a, t.b, p.m0[t.pos], c->batch_tag});
             op.merged[t.pos].set(t.a, t.b, t.end);
             // merge with the previous interval's task for the same position when the program is the same
             bool merged = false;
@@ -772,7 +786,7 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
         while (i < lv.size()) {
             static thread_local ReduceWave w;
             w.dir = c->d_dir;
-            w.status = c->d_status;
+            w.status = nullptr;
             w.budget_ns = c->cfg.poll_budget_ns;
             w.n_tasks = 0;
             w.total_tiles = 0;
@@ -815,6 +829,7 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
             if (grid < 1) grid = 1;
             if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
+            w.status = next_wave_status(c);
             {
                 LaunchTimer timer(c, 0);
                 if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
@@ -899,7 +914,7 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
                 continue;
             }
             groups[loc].push_back(r);
-            c->journal.b.push_back({op.src, r, op.phys_have[r]});
+            c->journal.b.push_back({op.src, r, op.phys_have[r], c->batch_tag});
             op.phys_have[r] = b;
         }
         for (auto& g : groups) {
@@ -928,7 +943,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
     while (i < tasks.size()) {
         static thread_local FanoutWave w;
         w.dir = c->d_dir;
-        w.status = c->d_status;
+        w.status = nullptr;
         w.budget_ns = c->cfg.poll_budget_ns;
         w.n_tasks = 0;
         w.total_tiles = 0;
@@ -970,6 +985,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
         if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
+        w.status = next_wave_status(c);
         {
             LaunchTimer timer(c, 1);
             if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
@@ -1006,6 +1022,7 @@ int progress(hpl_ctx* c) {
     auto bi = c->bcasts.begin();
     while (ri != c->reduces.end() || bi != c->bcasts.end()) {
         const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
+        c->batch_tag = c->launch_seq;
         if (take_reduce) {
             std::vector<PlannedReduceTask> tasks;
             int rc = plan_reduce(c, ri->second, tasks);
@@ -1025,8 +1042,11 @@ int progress(hpl_ctx* c) {
     return HPL_OK;
 }
 
-void undo_journal(hpl_ctx* c) {
+// Voids what was planned by the passes whose waves have seq >= from_tag (a wave of that pass gave up, and
+// later passes may have built on it); earlier passes ran to completion and are kept.
+void undo_journal(hpl_ctx* c, uint64_t from_tag) {
     for (auto& e : c->journal.r) {
+        if (e.tag < from_tag) continue;
         auto it = c->reduce_of_target.find(e.target);
         if (it == c->reduce_of_target.end()) continue;
         ReduceOp& op = c->reduces.at(it->second);
@@ -1035,6 +1055,7 @@ void undo_journal(hpl_ctx* c) {
         if (e.pos < (int)op.merged.size()) op.merged[e.pos].set(e.a, e.b, 0);
     }
     for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
+        if (it->tag < from_tag) continue;
         auto f = c->bcast_of_src.find(it->src);
         if (f == c->bcast_of_src.end()) continue;
         BcastOp& op = c->bcasts.at(f->second);
@@ -1057,17 +1078,28 @@ int sync_and_check(hpl_ctx* c) {
         c->journal.clear();
         return HPL_OK;
     }
-    CUDA_TRY(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, c->stream));
+    const uint32_t used = (uint32_t)std::min<uint64_t>(c->launch_seq - c->first_unchecked, kStatusSlots);
+    CUDA_TRY(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(DeviceStatus) * used, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->work_in_flight = false;
     collect_kernel_times(c);
-    c->stats.device_waits = c->h_status->waits;
-    if (c->h_status->error) {
+    bool failed = false;
+    uint64_t from_tag = ~0ull;
+    for (uint32_t i = 0; i < used; ++i) {
+        c->stats.device_waits += c->h_status[i].waits;
+        if (!c->h_status[i].error) continue;
+        failed = true;
+        // the record in the last slot may stand for several waves: the earliest of them decides
+        const uint64_t tag = c->wave_tag[i];
+        from_tag = std::min(from_tag, tag);
+    }
+    c->first_unchecked = c->launch_seq;
+    c->wave_tag.clear();
+    // the records are cleared behind everything launched so far; later launches are ordered after that
+    CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus) * used, c->stream));
+    if (failed) {
         c->stats.device_timeouts++;
-        undo_journal(c);
-        // clear the error record but keep the running count of waits
-        CUDA_TRY(cudaMemsetAsync(c->d_status, 0, offsetof(DeviceStatus, waits), c->stream));
-        CUDA_TRY(cudaStreamSynchronize(c->stream));
+        undo_journal(c, from_tag);
         return HPL_ERR_TIMEOUT;
     }
     c->journal.clear();
@@ -1166,7 +1198,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
     c->tau = cfg->virt_chunk_ns ? cfg->virt_chunk_ns : std::max<uint64_t>(1, cfg->chunk_bytes * 1000000000ull / (64ull << 30));
     c->stream = (cudaStream_t)cuda_stream;
     if (cfg->arena) {
-        const uint64_t need = sizeof(DirRow) * kMaxRows + sizeof(DeviceStatus) + 2 * kAlign;
+        const uint64_t need = sizeof(DirRow) * kMaxRows + sizeof(DeviceStatus) * kStatusSlots + 2 * kAlign;
         if (cfg->arena_bytes < need) {
             delete c;
             return HPL_ERR_NOMEM;
@@ -1180,10 +1212,10 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         c->n_sm = prop.multiProcessorCount;
         c->arena.init(cfg->arena, cfg->arena_bytes);
         c->d_dir = (DirRow*)c->arena.alloc(sizeof(DirRow) * kMaxRows);
-        c->d_status = (DeviceStatus*)c->arena.alloc(sizeof(DeviceStatus));
+        c->d_status = (DeviceStatus*)c->arena.alloc(sizeof(DeviceStatus) * kStatusSlots);
         bool ok = c->d_dir && c->d_status;
         ok = ok && cudaHostAlloc((void**)&c->h_dir, sizeof(DirRow) * kMaxRows, cudaHostAllocDefault) == cudaSuccess;
-        ok = ok && cudaHostAlloc((void**)&c->h_status, sizeof(DeviceStatus), cudaHostAllocDefault) == cudaSuccess;
+        ok = ok && cudaHostAlloc((void**)&c->h_status, sizeof(DeviceStatus) * kStatusSlots, cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaHostAlloc((void**)&c->h_stage, sizeof(DirRow) * kStageRows, cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaHostAlloc((void**)&c->h_iota, sizeof(uint32_t) * (kMaxChunks + 1), cudaHostAllocDefault) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -1191,7 +1223,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         ok = ok && cudaEventCreateWithFlags(&c->copy_ev, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->ctl_ev, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaMemsetAsync(c->d_dir, 0, sizeof(DirRow) * kMaxRows, c->stream) == cudaSuccess;
-        ok = ok && cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus), c->stream) == cudaSuccess;
+        ok = ok && cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus) * kStatusSlots, c->stream) == cudaSuccess;
         ok = ok && cudaStreamSynchronize(c->stream) == cudaSuccess;   // side streams must not overtake the clearing
         if (!ok) {
             if (c->h_dir) cudaFreeHost(c->h_dir);
@@ -1608,6 +1640,8 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (!c->device) return HPL_ERR_CUDA;
         if (!op.merged[0].covers(0, op.C, op.n_ops(0))) return HPL_ERR_TIMEOUT;
         rc = sync_and_check(c);
+        // a wait that expired in some other collective's wave does not concern this target if its own work stands
+        if (rc == HPL_ERR_TIMEOUT && op.merged[0].covers(0, op.C, op.n_ops(0))) rc = HPL_OK;
         if (rc != HPL_OK) return rc;
     } else if (o->kind == OBJ_RECEIVER) {
         if (!o->alive) return HPL_ERR_FAILED_WORKER;
@@ -1641,6 +1675,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (rc != HPL_OK) return rc;
         if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) return HPL_ERR_TIMEOUT;
         rc = sync_and_check(c);
+        if (rc == HPL_ERR_TIMEOUT && op.phys_have[li] >= (int64_t)o->C) rc = HPL_OK;   // the expired wait was elsewhere
         if (rc != HPL_OK) return rc;
     } else {
         if (!o->alive) return HPL_ERR_FAILED_WORKER;

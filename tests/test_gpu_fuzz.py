@@ -110,4 +110,7 @@ def _timeline(seed):
 @pytest.mark.parametrize("block", range(6))
 def test_random_timelines_match_the_oracle(block):
     for seed in range(block * 25, (block + 1) * 25):
-        _timeline(seed)
+        try:
+            _timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
