@@ -12,6 +12,7 @@
 
 #include <algorithm>
 #include <cstddef>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <memory>
@@ -362,7 +363,6 @@ uint64_t produced_elems(hpl_ctx* c, const Object& o) {
     } while (0)
 
 int alloc_row(hpl_ctx* c, Object& o) {
-    if (!c->device) return HPL_OK;
     if (o.row >= 0) return HPL_OK;
     if (c->free_rows.empty()) return HPL_ERR_NOMEM;
     o.row = c->free_rows.back();
@@ -377,7 +377,9 @@ int alloc_row(hpl_ctx* c, Object& o) {
     r.owner = (unsigned)o.worker;
     // With plan-ahead a kernel that polls may occupy the main stream for a while, so directory rows travel
     // on the control stream (tiny copies only) and the main stream is ordered after it before each launch.
-    if (c->cfg.plan_ahead) {
+    if (!c->device) {
+        // schedule-only context: the mirror is all there is (the planners run, nothing is launched)
+    } else if (c->cfg.plan_ahead) {
         CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->ctl_stream));
         c->ctl_pending = true;
     } else {
@@ -392,6 +394,7 @@ constexpr uint32_t kStageRows = 4 * kMaxRows;
 // consecutive rows, from an immutable pinned snapshot, ordered on the main stream before whatever is
 // launched next.  A Put is then a few stores on the host; its cost on the device is amortised over the batch.
 int flush_directory(hpl_ctx* c) {
+    if (!c->device) c->dirty_rows.clear();
     if (c->dirty_rows.empty()) return HPL_OK;
     std::sort(c->dirty_rows.begin(), c->dirty_rows.end());
     c->dirty_rows.erase(std::unique(c->dirty_rows.begin(), c->dirty_rows.end()), c->dirty_rows.end());
@@ -424,8 +427,9 @@ int order_main_after_control(hpl_ctx* c) {
 
 // Publishes the chunk prefix of a put object in the device directory, ordered on `s`.
 int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
-    if (!c->device || o.row < 0) return HPL_OK;
+    if (o.row < 0) return HPL_OK;
     c->h_dir[o.row].ready_chunks = chunks;   // the host mirror always holds the published value
+    if (!c->device) return HPL_OK;
     if (s == c->stream && !c->cfg.plan_ahead) {
         c->dirty_rows.push_back(o.row);
         return HPL_OK;
@@ -824,6 +828,12 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 ++i;
             }
             if (w.n_tasks == 0) return HPL_ERR_INVALID;  // a single task larger than a wave: tree too wide
+            if (!c->device) {   // schedule-only context: the wave is planned and counted, not run
+                c->stats.kernel_launches++;
+                c->stats.reduce_launches++;
+                c->stats.tiles += w.total_tiles;
+                continue;
+            }
             int& occ = c->occ_reduce[bf16 ? 1 : 0][occ_index(n_acc)];
             if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16);
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
@@ -981,6 +991,12 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
             ++i;
         }
         if (w.n_tasks == 0) return HPL_ERR_INVALID;
+        if (!c->device) {   // schedule-only context: planned and counted, not run
+            c->stats.kernel_launches++;
+            c->stats.fanout_launches++;
+            c->stats.tiles += w.total_tiles;
+            continue;
+        }
         if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
@@ -1001,7 +1017,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
 
 // ------------------------------------------------------------------------------------------ progress / sync
 int progress(hpl_ctx* c) {
-    if (!c->device) return HPL_OK;
+    // (a schedule-only context plans as well -- its planned tasks are counted, nothing is launched)
     {
         int rc = order_main_after_control(c);
         if (rc != HPL_OK) return rc;
@@ -1065,7 +1081,10 @@ void undo_journal(hpl_ctx* c, uint64_t from_tag) {
 }
 
 int sync_and_check(hpl_ctx* c) {
-    if (!c->device) return HPL_OK;
+    if (!c->device) {
+        c->journal.clear();
+        return HPL_OK;
+    }
     if (c->copy_pending || c->ctl_pending) {
         CUDA_TRY(cudaStreamSynchronize(c->ctl_stream));
         CUDA_TRY(cudaStreamSynchronize(c->copy_stream));
@@ -1240,6 +1259,17 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         for (uint32_t i = 0; i <= kMaxChunks; ++i) c->h_iota[i] = i;
         for (int r = (int)kMaxRows - 1; r >= 0; --r) c->free_rows.push_back(r);
         c->device = true;
+    } else {
+        // schedule-only context: no device memory.  Addresses are handed out from a range that is never
+        // dereferenced, so that the planners run exactly as they would with an arena.
+        c->arena.init((void*)(uintptr_t)(1ull << 44), 1ull << 44);
+        c->h_dir = (DirRow*)std::calloc(kMaxRows, sizeof(DirRow));
+        if (!c->h_dir) {
+            delete c;
+            return HPL_ERR_NOMEM;
+        }
+        for (int r = (int)kMaxRows - 1; r >= 0; --r) c->free_rows.push_back(r);
+        c->n_sm = 148;
     }
     *out = c;
     return HPL_OK;
@@ -1262,6 +1292,7 @@ int hpl_shutdown(hpl_ctx* c) {
         cudaEventDestroy(c->copy_ev);
         cudaEventDestroy(c->ctl_ev);
     }
+    if (!c->device) std::free(c->h_dir);
     delete c;
     return HPL_OK;
 }
@@ -1423,7 +1454,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     t.t_arrival = (int64_t)c->now;
     t.ready_bytes = 0;
     t.seq = c->seq++;
-    if (c->device) {
+    {
         t.ptr = c->arena.alloc(t.bytes);
         if (!t.ptr) return HPL_ERR_NOMEM;
         int rc = alloc_row(c, t);
@@ -1648,7 +1679,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
         const int li = op.sched->index_of(id);
         if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
-        if (c->device && (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C)) {
+        if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) {
             // start the copies first: the GPU works while the host lets the virtual clock run below
             int rc = progress(c);
             if (rc != HPL_OK) return rc;

@@ -1,0 +1,127 @@
+"""The planners (host logic) on a machine without a GPU.  A context created without an arena plans exactly
+as it would with one -- its tasks are counted in the statistics -- but launches nothing."""
+import math
+
+import pytest
+
+import paper_2002_05814_b200 as hpl
+import workloads as wl
+from paper_2002_05814_b200 import build as hpl_build
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    hpl_build.build()
+
+
+def _addr(i):
+    return 1 << 20 | (i + 1) << 24          # distinct, 16-byte aligned, never dereferenced
+
+
+def _plan_get(c, oid):
+    rc, _, _ = c.try_get(oid)
+    assert rc == hpl.HPL_ERR_CUDA            # planned to completion; only the device is missing
+    return c.stats()
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3", "cfg4"])
+def test_everything_ready_is_one_fused_pass_with_exactly_the_algorithmic_bytes(name):
+    w = wl.workload(name)
+    dt = hpl.HPL_BF16 if w.dtype == "bf16" else hpl.HPL_F32
+    with hpl.Context(w.chunk_bytes, w.degree, w.degree) as c:
+        S = w.object_bytes
+        for i in range(w.n_objects):
+            c.create(i, i, S, dt)
+        c.reduce(900, list(range(w.n_objects)), w.k, hpl.HPL_SUM, dt)
+        for i in range(w.n_objects):
+            c.advance(i)
+            c.put(i, _addr(i), S)
+        st = _plan_get(c, 900)
+        assert st["reduce_tasks"] == 1 and st["kernel_launches"] == 1
+        assert st["bytes_read_planned"] == w.k * S and st["bytes_written_planned"] == w.elems * 4
+
+
+def test_broadcast_to_all_joined_receivers_reads_the_source_once():
+    w = wl.workload("cfg4")
+    S = w.object_bytes
+    with hpl.Context(w.chunk_bytes, w.degree, w.degree) as c:
+        c.create(0, 99, S, hpl.HPL_BF16)
+        c.put(0, _addr(0), S)
+        ids = list(range(1, 65))
+        c.create_batch(ids, ids, S, hpl.HPL_BF16)
+        c.broadcast(0, ids)
+        c.join_batch(ids, [_addr(i) for i in ids])
+        st = _plan_get(c, 64)
+        assert st["fanout_tasks"] == 1 and st["bytes_read_planned"] == S and st["bytes_written_planned"] == 64 * S
+        # a receiver that joins later is served from its sender's copy, not from the source again
+        c.create(70, 70, S, hpl.HPL_BF16)
+
+
+@pytest.mark.parametrize("d", [2, 4])
+def test_progress_after_every_arrival_leaves_little_for_the_last_pass(d):
+    k, S = 16, 1 << 20
+    with hpl.Context(64 << 10, d, 2) as c:
+        for i in range(k):
+            c.create(i, i, S)
+        c.reduce(900, list(range(k)), k)
+        reads = []
+        for i in range(k):
+            c.advance(i + 1)
+            c.put(i, _addr(i), S)
+            c.progress()
+            reads.append(c.stats()["bytes_read_planned"])
+        st = _plan_get(c, 900)
+        assert reads[-1] - reads[-2] <= (math.ceil(math.log(k, d)) + d) * S     # only the root path was left
+        assert st["bytes_read_planned"] < 3 * k * S                             # merging early costs re-reads, boundedly
+
+
+def test_failure_without_fusion_recomputes_only_the_root_paths():
+    k, S, chunk = 32, 1 << 20, 64 << 10
+    with hpl.Context(chunk, 2, 2, fuse=False) as c:
+        for i in range(k):
+            c.create(i, i, S)
+        c.reduce(900, list(range(k)), k)
+        for i in range(k):
+            c.put(i, _addr(i), S if i != 7 else 6 * chunk)
+        c.progress()
+        before = c.stats()
+        c.advance(5)
+        c.fail(7)
+        st = _plan_get(c, 900)
+        redone = st["reduce_tasks"] - before["reduce_tasks"]
+        assert redone <= 2 * 2 * (math.ceil(math.log2(k)) + 1)
+        assert st["bytes_read_planned"] - before["bytes_read_planned"] < (k - 1) * S
+
+
+def test_a_tree_larger_than_one_task_is_cut_and_launched_in_levels():
+    k, S = 1000, 8192
+    with hpl.Context(4096, 2, 2) as c:
+        for i in range(k):
+            c.create(i, i % 5, S)
+            c.put(i, _addr(i), S)
+        c.reduce(5000, list(range(k)), k)
+        st = _plan_get(c, 5000)
+        assert st["reduce_tasks"] > 1 and st["kernel_launches"] >= 2
+        assert st["bytes_read_planned"] >= k * S
+    with hpl.Context(4096, 1000, 2) as c:
+        for i in range(800):
+            c.create(i, 0, 64)
+        with pytest.raises(hpl.HplError) as ei:
+            c.reduce(5000, list(range(800)), 800)
+        assert ei.value.code == hpl.HPL_ERR_INVALID
+
+
+def test_composed_collectives_are_planned_in_creation_order():
+    S = 1 << 18
+    with hpl.Context(64 << 10, 2, 2) as c:
+        for i in range(6):
+            c.create(i, i, S)
+            c.put(i, _addr(i), S)
+        c.reduce(100, [0, 1, 2], 3)
+        c.reduce(200, [100, 3, 4, 5], 4)
+        c.create(300, 50, S)
+        c.broadcast(200, [300])
+        c.join(300, _addr(30))
+        st = _plan_get(c, 300)
+        assert st["reduce_tasks"] == 2 and st["fanout_tasks"] == 1
+        assert st["bytes_read_planned"] == 3 * S + 4 * S + S      # inputs of each stage, then the output once
