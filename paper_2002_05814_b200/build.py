@@ -8,8 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhpl.so")
-SOURCES = ["hpl.cpp", "sched_reduce.cpp", "sched_bcast.cpp", "kernels.cu", "noalloc.cu"]
-HEADERS = ["device_types.h", "sched_reduce.h", "sched_bcast.h", os.path.join("..", "..", "include", "hpl.h")]
+SOURCES = ["hpl.cpp", "directory.cpp", "plan_reduce.cpp", "plan_bcast.cpp", "sched_reduce.cpp", "sched_bcast.cpp",
+           "kernels.cu", "noalloc.cu"]
+HEADERS = ["context.h", "device_types.h", "sched_reduce.h", "sched_bcast.h", os.path.join("..", "..", "include", "hpl.h")]
 
 
 def _stale() -> bool:

@@ -1,0 +1,171 @@
+// The object table and the device-resident directory: rows, progress counters, published prefixes as the
+// schedules see them, and the small per-launch resources (error records, timing events).
+#include "context.h"
+
+namespace hpl {
+
+Object* find(hpl_ctx* c, int64_t id) {
+    auto it = c->objects.find(id);
+    return it == c->objects.end() ? nullptr : &it->second;
+}
+
+// Element prefix an object has published, as the schedules see it: of a Put object what was put (whole
+// chunks); of a Reduce output (published when Reduce is called, Section 3.4.2) what its tree can already
+// produce, i.e. the smallest prefix among its members once the tree is full.
+uint64_t logical_ready_elems(hpl_ctx* c, int64_t oid) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    if (o->kind == OBJ_TARGET) {
+        auto it = c->reduce_of_target.find(oid);
+        if (it == c->reduce_of_target.end()) return 0;
+        ReduceTreeSchedule& s = *c->reduces.at(it->second).sched;
+        if (!s.full()) return 0;
+        uint64_t m = object_elems(*o);
+        for (int p = 0; p < s.k(); ++p) m = std::min(m, logical_ready_elems(c, s.object_at(p)));
+        return m;
+    }
+    if (o->ready_bytes >= o->bytes) return object_elems(*o);
+    return (uint64_t)published_chunks(c, *o) * object_chunk_elems(c, *o);
+}
+
+// The same prefix counted in the object's own chunks (chunk_bytes of its own dtype) ...
+int64_t logical_delivered(hpl_ctx* c, int64_t oid) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    const uint64_t n = logical_ready_elems(c, oid);
+    return n >= object_elems(*o) ? (int64_t)o->C : (int64_t)(n / object_chunk_elems(c, *o));
+}
+
+// ... and in the chunks of a Reduce (chunk_bytes of its input dtype: a bf16 Reduce works on twice as many
+// elements per chunk as its fp32 output holds).
+int64_t logical_delivered_in(hpl_ctx* c, int64_t oid, const ReduceOp& op) {
+    Object* o = find(c, oid);
+    if (!o) return 0;
+    const uint64_t n = logical_ready_elems(c, oid);
+    return n >= object_elems(*o) ? (int64_t)op.C : (int64_t)(n / op.chunk_elems);
+}
+
+// Elements of a Reduce output that earlier waves on the stream have produced (or will have, by stream order).
+uint64_t produced_elems(hpl_ctx* c, const Object& o) {
+    auto it = c->reduce_of_target.find(o.id);
+    if (it == c->reduce_of_target.end()) return 0;
+    const ReduceOp& op = c->reduces.at(it->second);
+    if (op.merged.empty()) return 0;
+    return std::min<uint64_t>((uint64_t)op.merged[0].full_prefix(op.n_ops(0)) * op.chunk_elems, op.elems);
+}
+
+int alloc_row(hpl_ctx* c, Object& o) {
+    if (o.row >= 0) return HPL_OK;
+    if (c->free_rows.empty()) return HPL_ERR_NOMEM;
+    o.row = c->free_rows.back();
+    c->free_rows.pop_back();
+    DirRow& r = c->h_dir[o.row];
+    r.ptr = (unsigned long long)(uintptr_t)o.ptr;
+    r.bytes = o.bytes;
+    r.n_chunks = o.C;
+    // rows of library-produced copies are never polled: validity of their bytes is stream order
+    r.ready_chunks = (o.kind == OBJ_PLAIN) ? 0u : o.C;
+    r.dtype = (unsigned)o.dtype;
+    r.owner = (unsigned)o.worker;
+    // With plan-ahead a kernel that polls may occupy the main stream for a while, so directory rows travel
+    // on the control stream (tiny copies only) and the main stream is ordered after it before each launch.
+    if (!c->device) {
+        // schedule-only context: the mirror is all there is (the planners run, nothing is launched)
+    } else if (c->cfg.plan_ahead) {
+        CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->ctl_stream));
+        c->ctl_pending = true;
+    } else {
+        c->dirty_rows.push_back(o.row);   // travels with the next flush, before the next launch
+    }
+    return HPL_OK;
+}
+
+
+// Batched mode (no plan-ahead): all rows changed since the last flush go to the device in one copy per run of
+// consecutive rows, from an immutable pinned snapshot, ordered on the main stream before whatever is
+// launched next.  A Put is then a few stores on the host; its cost on the device is amortised over the batch.
+int flush_directory(hpl_ctx* c) {
+    if (!c->device) c->dirty_rows.clear();
+    if (c->dirty_rows.empty()) return HPL_OK;
+    std::sort(c->dirty_rows.begin(), c->dirty_rows.end());
+    c->dirty_rows.erase(std::unique(c->dirty_rows.begin(), c->dirty_rows.end()), c->dirty_rows.end());
+    size_t i = 0;
+    while (i < c->dirty_rows.size()) {
+        size_t j = i + 1;
+        while (j < c->dirty_rows.size() && c->dirty_rows[j] == c->dirty_rows[j - 1] + 1) ++j;
+        const uint32_t n = (uint32_t)(j - i);
+        if (c->stage_cursor + n > kStageRows) {
+            CUDA_TRY(cudaStreamSynchronize(c->stream));   // every earlier snapshot has been consumed
+            c->stage_cursor = 0;
+        }
+        DirRow* snap = c->h_stage + c->stage_cursor;
+        std::memcpy(snap, c->h_dir + c->dirty_rows[i], n * sizeof(DirRow));
+        CUDA_TRY(cudaMemcpyAsync(c->d_dir + c->dirty_rows[i], snap, n * sizeof(DirRow), cudaMemcpyHostToDevice, c->stream));
+        c->stage_cursor += n;
+        i = j;
+    }
+    c->dirty_rows.clear();
+    return HPL_OK;
+}
+
+int order_main_after_control(hpl_ctx* c) {
+    if (!c->ctl_pending) return HPL_OK;
+    CUDA_TRY(cudaEventRecord(c->ctl_ev, c->ctl_stream));
+    CUDA_TRY(cudaStreamWaitEvent(c->stream, c->ctl_ev, 0));
+    c->ctl_pending = false;
+    return HPL_OK;
+}
+
+// Publishes the chunk prefix of a put object in the device directory, ordered on `s`.
+int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
+    if (o.row < 0) return HPL_OK;
+    c->h_dir[o.row].ready_chunks = chunks;   // the host mirror always holds the published value
+    if (!c->device) return HPL_OK;
+    if (s == c->stream && !c->cfg.plan_ahead) {
+        c->dirty_rows.push_back(o.row);
+        return HPL_OK;
+    }
+    CUDA_TRY(cudaMemcpyAsync(&c->d_dir[o.row].ready_chunks, &c->h_iota[chunks], sizeof(uint32_t), cudaMemcpyHostToDevice, s));
+    return HPL_OK;
+}
+
+// The error record of the wave that is about to be launched.
+DeviceStatus* next_wave_status(hpl_ctx* c) {
+    const uint64_t idx = c->launch_seq - c->first_unchecked;
+    c->wave_tag.push_back(c->batch_tag);
+    ++c->launch_seq;
+    return c->d_status + std::min<uint64_t>(idx, kStatusSlots - 1);
+}
+
+cudaEvent_t take_event(hpl_ctx* c) {
+    if (!c->event_pool.empty()) {
+        cudaEvent_t e = c->event_pool.back();
+        c->event_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+void collect_kernel_times(hpl_ctx* c) {   // call only after the stream has been waited for
+    for (auto& t : c->timed) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) {
+            const uint64_t ns = (uint64_t)((double)ms * 1e6);
+            if (t.kind == 0) c->stats.reduce_kernel_ns += ns; else c->stats.fanout_kernel_ns += ns;
+        }
+        c->event_pool.push_back(t.a);
+        c->event_pool.push_back(t.b);
+    }
+    c->timed.clear();
+}
+
+void release_object_memory(hpl_ctx* c, Object& o) {
+    if (o.lib_owned && o.ptr) c->arena.release(o.ptr);
+    o.ptr = nullptr;
+    if (o.row >= 0) c->free_rows.push_back(o.row);
+    o.row = -1;
+}
+
+}  // namespace hpl

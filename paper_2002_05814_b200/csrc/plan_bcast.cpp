@@ -1,0 +1,159 @@
+// Broadcast planner: which receivers can be served now, from which copy, as fan-out tasks.
+#include "context.h"
+
+namespace hpl {
+
+int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+    BroadcastTreeSchedule& s = *op.sched;
+    const auto& locs = s.locations();
+    op.phys_have.resize(locs.size(), 0);
+    Object* src = find(c, op.src);
+    if (!src) return HPL_OK;
+    const uint32_t C = src->C;
+    uint32_t src_landed = 0, src_avail = 0;
+    if (src->alive && src->ptr && src->row >= 0) {
+        if (src->kind == OBJ_TARGET) {   // reduce followed by broadcast: the source is a Reduce output
+            const uint64_t n = produced_elems(c, *src);   // fp32 elements -> chunks of the broadcast (bytes of the object)
+            src_landed = src_avail = n * 4 >= src->bytes ? C : (uint32_t)(n * 4 / c->cfg.chunk_bytes);
+        } else {
+            src_landed = std::min(published_chunks(c, *src), src->landed);
+            src_avail = c->cfg.plan_ahead ? C : src_landed;
+        }
+    }
+    std::vector<int64_t> pre(op.phys_have);  // what every copy holds before this pass
+    pre[0] = src_avail;
+    std::vector<char> usable_v(locs.size(), 0);   // copies whose buffer may be read or written now
+    usable_v[0] = src->alive && src->ptr != nullptr;
+    bool any_pending = false;
+    for (size_t x = 1; x < locs.size(); ++x) {
+        if (!locs[x].alive) continue;
+        Object* o = find(c, locs[x].obj);
+        usable_v[x] = o && o->alive && o->ptr && o->row >= 0;
+        if (usable_v[x] && op.phys_have[x] < (int64_t)C) any_pending = true;
+    }
+    if (!any_pending) return HPL_OK;
+    auto usable = [&](int x) { return usable_v[x] != 0; };
+    std::vector<uint32_t> bp = {0u, src_avail};
+    for (size_t i = 1; i < locs.size(); ++i) bp.push_back((uint32_t)pre[i]);
+    std::sort(bp.begin(), bp.end());
+    bp.erase(std::unique(bp.begin(), bp.end()), bp.end());
+
+    std::vector<char> stuck(locs.size(), 0);
+    for (size_t bi = 0; bi + 1 < bp.size(); ++bi) {
+        const uint32_t a = bp[bi], b = bp[bi + 1];
+        std::map<int, std::vector<int>> groups;  // read location -> receivers
+        for (int r = 1; r < (int)locs.size(); ++r) {
+            if (stuck[r] || !usable(r) || locs[r].last_sender < 0) continue;
+            if (op.phys_have[r] != (int64_t)a) continue;  // needs this interval next
+            int loc = -1;
+            for (int x = locs[r].last_sender, hops = 0; x >= 0 && hops <= (int)locs.size(); x = locs[x].last_sender, ++hops) {
+                if (usable(x) && pre[x] >= (int64_t)b) {
+                    loc = x;
+                    break;
+                }
+                if (x == 0) break;
+            }
+            if (loc < 0) {
+                for (int x = 0; x < (int)locs.size(); ++x)
+                    if (x != r && usable(x) && pre[x] >= (int64_t)b) {
+                        loc = x;
+                        break;
+                    }
+            }
+            if (loc < 0) {
+                stuck[r] = 1;
+                continue;
+            }
+            groups[loc].push_back(r);
+            c->journal.b.push_back({op.src, r, op.phys_have[r], c->batch_tag});
+            op.phys_have[r] = b;
+        }
+        for (auto& g : groups) {
+            const bool poll = (g.first == 0) && (src_landed < b);
+            bool merged = false;
+            for (auto& prev : tasks) {
+                if (prev.loc == g.first && prev.b == a && prev.poll == poll && prev.dst == g.second) {
+                    prev.b = b;
+                    merged = true;
+                    break;
+                }
+            }
+            if (!merged) tasks.push_back(PlannedFanout{g.first, a, b, poll, g.second});
+        }
+    }
+    return HPL_OK;
+}
+
+int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+    if (tasks.empty()) return HPL_OK;
+    Object* src = find(c, op.src);
+    const auto& locs = op.sched->locations();
+    const uint64_t chunk_bytes = c->cfg.chunk_bytes;
+    const uint32_t tpc = (uint32_t)((std::min<uint64_t>(chunk_bytes, src->bytes) + kFanoutTileBytes - 1) / kFanoutTileBytes);
+    size_t i = 0;
+    while (i < tasks.size()) {
+        static thread_local FanoutWave w;
+        w.dir = c->d_dir;
+        w.status = nullptr;
+        w.budget_ns = c->cfg.poll_budget_ns;
+        w.n_tasks = 0;
+        w.total_tiles = 0;
+        uint32_t n_dst = 0;
+        while (i < tasks.size() && w.n_tasks < (uint32_t)kMaxFanoutTasks) {
+            PlannedFanout& t = tasks[i];
+            if (t.dst.size() > (size_t)kMaxFanoutDst) {
+                // more receivers than one task holds: split the receiver list
+                PlannedFanout rest = t;
+                rest.dst.assign(t.dst.begin() + kMaxFanoutDst, t.dst.end());
+                t.dst.resize(kMaxFanoutDst);
+                tasks.insert(tasks.begin() + i + 1, rest);
+                continue;
+            }
+            if (n_dst + tasks[i].dst.size() > (size_t)kMaxFanoutDst) break;
+            PlannedFanout& tt = tasks[i];
+            FanoutTask& d = w.tasks[w.n_tasks++];
+            Object* lo = tt.loc == 0 ? src : find(c, locs[tt.loc].obj);
+            d.src_row = (uint32_t)lo->row;
+            d.c_begin = tt.a;
+            d.c_end = tt.b;
+            d.tiles_per_chunk = tpc;
+            d.tile_begin = w.total_tiles;
+            d.dst_begin = n_dst;
+            d.n_dst = (uint32_t)tt.dst.size();
+            d.poll = tt.poll ? 1u : 0u;
+            d.bytes = src->bytes;
+            d.chunk_bytes = chunk_bytes;
+            for (int r : tt.dst) w.dst_rows[n_dst++] = (uint32_t)find(c, locs[r].obj)->row;
+            w.total_tiles += (tt.b - tt.a) * tpc;
+            const uint64_t b_lo = (uint64_t)tt.a * chunk_bytes, b_hi = std::min<uint64_t>((uint64_t)tt.b * chunk_bytes, src->bytes);
+            c->stats.bytes_read_planned += b_hi - b_lo;
+            c->stats.bytes_written_planned += (b_hi - b_lo) * tt.dst.size();
+            c->stats.fanout_tasks++;
+            ++i;
+        }
+        if (w.n_tasks == 0) return HPL_ERR_INVALID;
+        if (!c->device) {   // schedule-only context: planned and counted, not run
+            c->stats.kernel_launches++;
+            c->stats.fanout_launches++;
+            c->stats.tiles += w.total_tiles;
+            continue;
+        }
+        if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
+        int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
+        if (grid < 1) grid = 1;
+        if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
+        w.status = next_wave_status(c);
+        {
+            LaunchTimer timer(c, 1);
+            if (launch_fanout_wave(w, grid, c->stream) != 0) return HPL_ERR_CUDA;
+        }
+        c->stats.kernel_launches++;
+        c->stats.fanout_launches++;
+        c->stats.tiles += w.total_tiles;
+        c->stats.last_kernel_grid = (uint64_t)grid;
+        c->work_in_flight = true;
+    }
+    return HPL_OK;
+}
+
+}  // namespace hpl
