@@ -453,7 +453,7 @@ def main():
     ap.add_argument("--realtime", action="store_true", help="also measure cfg3 with puts at their real arrival offsets")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads measured briefly and reported under 'also'")
+    ap.add_argument("--also", default="cfg2,cfg3,cfg5", help="extra workloads measured briefly and reported under 'also' (cfg5 = the 1 GiB point of the fault-tolerant sweep, both modes)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -553,21 +553,35 @@ def main():
 
     if rank == 0 and world == 1 and args.also:
         also = {}
+        names = []
         for nm in [x for x in args.also.split(",") if x and x != "none" and x != w.name]:
-            ww = wl.workload(nm)
-            rr = Runner(ww, device)
-            r2 = time_steps(rr, 5, 3)
+            names += [("cfg5_1GiB_lazy", wl.cfg5_at(1 << 30), False), ("cfg5_1GiB_eager", wl.cfg5_at(1 << 30), True)] if nm == "cfg5" \
+                else [(nm, wl.workload(nm), True)]
+        rr = None
+        for label, ww, eager in names:
+            if rr is None or rr.w.name != ww.name or ww.name != "cfg5":
+                if rr is not None:
+                    rr.close()
+                    del rr
+                    torch.cuda.empty_cache()
+                rr = Runner(ww, device, ft_eager=eager)
+            rr.ft_eager = eager                  # the two cfg5 modes share the 32 GiB of inputs
+            n2 = 3 if ww.name == "cfg5" else 5
+            r2 = time_steps(rr, n2, 3)
+            a2 = algorithmic_bytes(ww)
+            b2 = a2["reduce"] + a2["broadcast"]
+            g = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
+            s2 = r2["stats"]
+            kns = s2["reduce_kernel_ns"] + s2["fanout_kernel_ns"]
+            planned = s2["bytes_read_planned"] + s2["bytes_written_planned"]
+            kern = gbs(planned, kns / 1e6)       # bytes the planned tasks move / their summed launch time
+            also[label] = {"GBps": g, "ms_per_step": float(np.mean(r2["total_ms"])), "kernel_GBps": kern,
+                           "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / n2,
+                           "planned_over_algorithmic_bytes": planned / (b2 * n2)}
+        if rr is not None:
             rr.close()
             del rr
             torch.cuda.empty_cache()
-            a2 = algorithmic_bytes(ww)
-            b2 = a2["reduce"] + a2["broadcast"]
-            g = gbs(b2 * 5, float(np.sum(r2["total_ms"])))
-            s2 = r2["stats"]
-            kn, kl = ("reduce_kernel_ns", "reduce_launches") if a2["reduce"] else ("fanout_kernel_ns", "fanout_launches")
-            kern = gbs(b2 * 5 / max(1, s2[kl]), s2[kn] / max(1, s2[kl]) / 1e6)
-            also[nm] = {"GBps": g, "ms_per_step": float(np.mean(r2["total_ms"])), "kernel_GBps": kern,
-                        "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / 5}
         line["also"] = also
 
     if rank == 0 and world == 1 and args.realtime:
