@@ -71,7 +71,9 @@ typedef struct hpl_config {
                                  summed into hpl_stats_t at the next wait (for benchmarks) */
     void*    arena;           /* device memory the library may use for the directory, partial results, reduce
                                  targets and copies of host objects; owned by the caller, must outlive the
-                                 context.  NULL = schedule-only context (no device work; hpl_get fails). */
+                                 context.  NULL = schedule-only context: schedules are built and work is planned and counted
+                                 (hpl_stats) exactly as with a device, but nothing is launched and hpl_get returns
+                                 HPL_ERR_CUDA where it would otherwise succeed. */
     uint64_t arena_bytes;
     uint64_t model_latency_ns;     /* L of Eq. 1: latency of one hop; used only when reduce_degree == 0 */
     uint64_t model_bandwidth_bps;  /* B of Eq. 1: bytes per second into one node; used only when reduce_degree == 0 */
