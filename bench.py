@@ -159,6 +159,7 @@ class Runner:
         self.a_dst_ids = C.ids_array([6000 + j for j in range(w.n_receivers)])
         self.a_dst_workers = [1000 + j for j in range(w.n_receivers)]
         self.a_dst_ptrs = C.ptr_array([t.data_ptr() for t in self.recv])
+        self.a_dst_out = C.ptr_array([0] * w.n_receivers)
         self.a_src_ids = C.ids_array(list(range(n_src)))
         self.a_src_workers = list(range(n_src))
         self.a_src_ptrs = C.ptr_array([t.data_ptr() for t in self.src])
@@ -204,8 +205,7 @@ class Runner:
                 ctx.progress()
                 ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
                 ctx.reduce(base + 9000, [base + i for i in range(w.n_objects)], w.k, self.hpl.HPL_SUM, self.dt)
-            for dd in dsts:
-                ctx.get(dd)
+            ctx.get_batch(self.a_dst_ids, self.a_dst_out)      # every receiver's Get
             if self.host_buffers:
                 ctx.get_host(dsts[-1], self.host_recv.data_ptr(), S)
                 d2h += S

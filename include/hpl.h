@@ -119,6 +119,10 @@ int hpl_put_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const void
 int hpl_join_batch(hpl_ctx* ctx, int32_t n, const int64_t* dst_ids, void* const* dst_bufs /* host array of DEVICE
                    pointers */, int32_t* n_done);
 
+/* Many hpl_get calls, in array order; dev_ptrs[i] (may be NULL as a whole) receives the pointer of object i.
+ * Stops at the first failure and returns its code. */
+int hpl_get_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const void** dev_ptrs, int32_t* n_done);
+
 /* Reduce (Table 1, Section 3.4.2).  Non-blocking.  Creates `target_id` (fp32, library-owned, in the arena)
  * from `k_first_ready` of the `n` objects `src_ids` -- those that arrive first; ties by index in src_ids --
  * combined with `op` in the association order of the degree-d tree.  All sources have dtype `dtype` and one

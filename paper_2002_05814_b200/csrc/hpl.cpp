@@ -704,6 +704,14 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
     return HPL_OK;
 }
 
+int hpl_get_batch(hpl_ctx* c, int32_t n, const int64_t* ids, const void** dev_ptrs, int32_t* n_done) {
+    if (!c || n < 0 || (n && !ids)) return HPL_ERR_INVALID;
+    int rc = HPL_OK, i = 0;
+    for (; i < n && rc == HPL_OK; ++i) rc = hpl_get(c, ids[i], dev_ptrs ? &dev_ptrs[i] : nullptr, nullptr);
+    if (n_done) *n_done = rc == HPL_OK ? i : i - 1;
+    return rc;
+}
+
 int hpl_get_host(hpl_ctx* c, int64_t id, void* dst, uint64_t cap) {
     if (!c || !dst) return HPL_ERR_INVALID;
     const void* p = nullptr;

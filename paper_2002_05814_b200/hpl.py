@@ -74,6 +74,7 @@ def load_library():
         "hpl_create_batch": [VP, I32, P(I64), P(I32), U64, I32, P(I32)],
         "hpl_put_batch": [VP, I32, P(I64), P(VP), P(U64), P(I32)],
         "hpl_join_batch": [VP, I32, P(I64), P(VP), P(I32)],
+        "hpl_get_batch": [VP, I32, P(I64), P(VP), P(I32)],
         "hpl_reduce": [VP, I64, P(I64), I32, I32, I32, I32],
         "hpl_broadcast": [VP, I64, P(I64), I32],
         "hpl_join": [VP, I64, VP],
@@ -184,6 +185,13 @@ class Context:
         ids = ids if isinstance(ids, C.Array) else self.ids_array(ids)
         ptrs = dev_ptrs if isinstance(dev_ptrs, C.Array) else self.ptr_array(dev_ptrs)
         self._check(self._lib.hpl_join_batch(self._h, len(ids), ids, ptrs, None), "hpl_join_batch")
+
+    def get_batch(self, ids, out_ptrs=None):
+        """``hpl_get`` for every id; returns the device pointers (or fills the ctypes array ``out_ptrs``)."""
+        ids = ids if isinstance(ids, C.Array) else self.ids_array(ids)
+        out = out_ptrs if out_ptrs is not None else (C.c_void_p * len(ids))()
+        self._check(self._lib.hpl_get_batch(self._h, len(ids), ids, out, None), "hpl_get_batch")
+        return out if out_ptrs is not None else list(out)
 
     def put_host(self, object_id: int, host_buf, nbytes: int):
         self._check(self._lib.hpl_put_host(self._h, object_id, C.c_void_p(_addr(host_buf)), nbytes), "hpl_put_host")

@@ -92,6 +92,9 @@ def test_batch_calls_are_the_single_calls_in_array_order():
         b.join(51, 24576)
         assert a.schedule_dump(5) == b.schedule_dump(5)
         with pytest.raises(hpl.HplError) as ei:
+            a.get_batch([5, 50])                        # object 5 is complete, but there is no device
+        assert ei.value.code == hpl.HPL_ERR_CUDA
+        with pytest.raises(hpl.HplError) as ei:
             a.create_batch([60, 5], [0, 0], 256)        # the second id exists: the first was still created
         assert ei.value.code == hpl.HPL_ERR_EXISTS
         with pytest.raises(hpl.HplError):
