@@ -451,6 +451,9 @@ def main():
                     help="cfg5: 'eager' runs hpl_progress before the failure (chunks delivered by every worker are reduced, "
                          "then partly redone); 'lazy' applies the compressed timeline and plans at the Get")
     ap.add_argument("--realtime", action="store_true", help="also measure cfg3 with puts at their real arrival offsets")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also measure GB/s against object size: the fault-tolerant reduce (32 objects, both modes) and a "
+                         "broadcast to 16 receivers, for 1 KiB ... 1 GiB in powers of 4")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--also", default="cfg2,cfg3,cfg5", help="extra workloads measured briefly and reported under 'also' (cfg5 = the 1 GiB point of the fault-tolerant sweep, both modes)")
@@ -586,6 +589,38 @@ def main():
 
     if rank == 0 and world == 1 and args.realtime:
         line["realtime_cfg3"] = realtime_rounds(device)
+
+    if rank == 0 and world == 1 and args.sweep:
+        rows = []
+        for size in wl.workload("cfg5").extra["sizes_bytes"]:
+            row = {"object_bytes": size}
+            n2 = 20 if size <= (16 << 20) else (5 if size <= (256 << 20) else 3)
+            ww = wl.cfg5_at(size)
+            rr = Runner(ww, device)
+            for mode in ("lazy", "eager"):
+                rr.ft_eager = mode == "eager"
+                r2 = time_steps(rr, n2, 3)
+                b2 = algorithmic_bytes(ww)["reduce"]
+                row[f"reduce_{mode}_GBps"] = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
+                row[f"reduce_{mode}_ms"] = float(np.mean(r2["total_ms"]))
+                s2 = r2["stats"]
+                row[f"reduce_{mode}_kernel_ms"] = s2["reduce_kernel_ns"] / 1e6 / n2
+            rr.close()
+            del rr
+            torch.cuda.empty_cache()
+            bw = wl.Workload("bcast", "broadcast", "f32", ("uniform",), size // 4, min(1 << 20, size), 2, n_receivers=16,
+                             extra={"join_window_ns": 1_000_000})
+            rr = Runner(bw, device)
+            r2 = time_steps(rr, n2, 3)
+            b2 = algorithmic_bytes(bw)["broadcast"]
+            row["broadcast16_GBps"] = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
+            row["broadcast16_ms"] = float(np.mean(r2["total_ms"]))
+            row["broadcast16_kernel_ms"] = r2["stats"]["fanout_kernel_ns"] / 1e6 / n2
+            rr.close()
+            del rr
+            torch.cuda.empty_cache()
+            rows.append(row)
+        line["sweep"] = rows
 
     if not args.no_e2e:
         e_steps = max(1, min(args.steps, 3))
