@@ -228,8 +228,15 @@ class Runner:
             if not early:
                 ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
             tmax = 0
-            if w.kind == "round" and not self.host_buffers:      # all returned objects are ready at once
-                ctx.put_batch(self.a_src_ids, self.a_src_ptrs, S)
+            if not self.host_buffers and max(arr) == 0:           # all objects are put at the same instant: one call
+                if w.kind == "ft_reduce":
+                    fw = w.extra["fail_worker"]
+                    part = int(w.extra["fail_fraction"] * wl.n_chunks(S, w.chunk_bytes)) * w.chunk_bytes
+                    sel = [i for i in range(n) if i != fw or part > 0]
+                    ctx.put_batch([ids[i] for i in sel], [self.src[i].data_ptr() for i in sel],
+                                  [part if i == fw else S for i in sel])
+                else:
+                    ctx.put_batch(self.a_src_ids, self.a_src_ptrs, S)
                 order = []
             for i in order:
                 ctx.advance(max(self.t + arr[i], self.t + tmax))
