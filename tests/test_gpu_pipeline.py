@@ -179,3 +179,30 @@ def test_waits_are_counted():
     p.check_target_bits(100)
     assert p.c.stats()["device_waits"] >= 1 and p.c.stats()["device_timeouts"] == 0
     p.close()
+
+
+def test_pageable_host_memory_and_get_host_of_every_kind_of_object():
+    elems, chunk = 50_000, 32 << 10
+    p = Pair(chunk, 2, 2, arena_bytes=32 << 20)
+    a = [gen(("uniform",), 77, i, elems) for i in range(3)]        # ordinary (pageable) numpy memory
+    for i in range(3):
+        p.host[i] = a[i]
+        p.c.create(i, i, a[i].nbytes, DT_F32)
+        p.o.create(i, i, a[i].nbytes, DT_F32)
+        p.c.put_host(i, a[i].ctypes.data, a[i].nbytes)
+        p.o.put(i, a[i], a[i].nbytes)
+    p.create(9, 9, nbytes=elems * 4, dtype=DT_F32)
+    p.reduce(100, [0, 1, 2], 3)
+    p.broadcast(1, [9])
+    p.join(9)
+    out = np.empty(elems, np.float32)
+    p.c.get_host(100, out.ctypes.data, out.nbytes)                   # a Reduce output
+    assert np.array_equal(out.view(np.uint32), p.o.get(100).view(np.uint32))
+    p.c.get_host(9, out.ctypes.data, out.nbytes)                     # a broadcast copy
+    assert out.tobytes() == a[1].tobytes()
+    p.c.get_host(2, out.ctypes.data, out.nbytes)                     # a put object (its copy in the store)
+    assert out.tobytes() == a[2].tobytes()
+    with pytest.raises(hpl.HplError) as ei:
+        p.c.get_host(2, out.ctypes.data, 16)                         # destination too small
+    assert ei.value.code == hpl.HPL_ERR_INVALID
+    p.close()
