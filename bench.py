@@ -377,6 +377,42 @@ def realtime_rounds(device, rounds: int = 8):
         out["eager" if eager else "lazy"] = {"latency_after_last_needed_arrival_us": float(np.mean(lat)),
                                              "std_us": float(np.std(lat)), "bytes_moved_in_that_tail": float(np.mean(tail_bytes)),
                                              "rounds": rounds}
+    # the same view for the broadcast shape (cfg2): receivers join at their real offsets; each join starts the
+    # copy for that receiver (from its sender's copy once that is complete); the figure is the time from the
+    # last join until every receiver holds the object
+    w2 = wl.workload("cfg2")
+    S2 = w2.object_bytes
+    ctx = hpl.Context(w2.chunk_bytes, w2.degree, w2.degree, arena=arena.data_ptr(), arena_bytes=arena.numel(),
+                      stream=torch.cuda.current_stream().cuda_stream, eager=True)
+    srcb = wl.values_torch(w2.dist, w2.seed, 0, 0, w2.elems, "f32", device=device)
+    recv = [torch.empty(w2.elems, dtype=torch.float32, device=device) for _ in range(w2.n_receivers)]
+    torch.cuda.synchronize()
+    lat = []
+    t_base = 0
+    for r in range(rounds + 1):
+        offs = wl.uniform_offsets_ns(w2.seed + r, w2.n_receivers, w2.extra["join_window_ns"])
+        order = sorted(range(w2.n_receivers), key=lambda j: (offs[j], j))
+        t_base += 1_000_000_000
+        ctx.advance(t_base)
+        ids = [100 + j for j in range(w2.n_receivers)]
+        ctx.create(0, 99, S2)
+        ctx.put(0, srcb.data_ptr(), S2)
+        ctx.create_batch(ids, ids, S2)
+        ctx.broadcast(0, ids)
+        t0 = time.perf_counter_ns()
+        for j in order:
+            while time.perf_counter_ns() - t0 < offs[j]:
+                pass
+            ctx.advance(t_base + offs[j])
+            ctx.join(ids[j], recv[j].data_ptr())
+        t_last = time.perf_counter_ns()
+        ctx.get_batch(ids)
+        if r > 0:
+            lat.append((time.perf_counter_ns() - t_last) / 1e3)
+        ctx.delete(0)
+    ctx.shutdown()
+    out["broadcast_cfg2"] = {"latency_after_last_join_us": float(np.mean(lat)), "std_us": float(np.std(lat)), "rounds": rounds,
+                             "note": "joins at real offsets over 1 ms, every join starts that receiver's copy"}
     out["note"] = ("eager: every Put also runs what became runnable (arrived operands are merged into their parents' partial "
                    "results); lazy: everything is planned at the Get, one fused pass over the 8 members")
     return out
