@@ -732,8 +732,9 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
     if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
     for (auto& kv : c->reduces)
         if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
-    if (c->device) {
-        // rows and arena memory are recycled only when nothing enqueued can still read them
+    if (c->device && (c->work_in_flight || c->copy_pending || c->ctl_pending)) {
+        // rows and arena memory are recycled only when nothing enqueued can still read them (nothing of the
+        // library's is in flight after a Get or a wait, so a round's Deletes cost no device wait)
         cudaStreamSynchronize(c->ctl_stream);
         cudaStreamSynchronize(c->copy_stream);
         cudaStreamSynchronize(c->stream);
