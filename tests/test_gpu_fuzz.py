@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import paper_2002_05814_b200 as hpl
-from oracle.store import StoreError, OK, DT_F32
+from oracle.store import StoreError, OK, DT_F32, DT_BF16
 from tests.harness import Pair, gen
 
 pytestmark = pytest.mark.gpu
@@ -56,16 +56,31 @@ def _timeline(seed):
         elems -= elems % 8
     nbytes = elems * 4
     size_of = {}
+    host_put = set()
+
+    def put(i, nb_):
+        if i in host_put:
+            p.c.put_host(i, p.host[i].ctypes.data, nb_)
+            p.o.put(i, p.host[i], nb_)
+        else:
+            p.put(i, nb_)
+
     for i in range(n):
         bf = a_bf16 and i < na
         data = gen(("normal", 0.02), 1000 + seed, i, elems, "bf16") if bf else \
             gen(("smallint", 30) if seed % 2 else ("uniform",), 1000 + seed, i, elems)
         size_of[i] = data.nbytes
-        p.create(i, int(rng.integers(0, n_workers)), data)
+        if rng.random() < 0.3:                        # this worker hands its object over from host memory
+            host_put.add(i)
+            p.host[i] = data
+            wk = int(rng.integers(0, n_workers))
+            p.c.create(i, wk, data.nbytes, DT_BF16 if bf else DT_F32)
+            p.o.create(i, wk, data.nbytes, DT_BF16 if bf else DT_F32)
+        else:
+            p.create(i, int(rng.integers(0, n_workers)), data)
     for j in range(R):
         p.create(500 + j, 100 + int(rng.integers(0, 2)), nbytes=nbytes, dtype=DT_F32)
     A, B = 1000, 2000
-    from oracle.store import DT_BF16
     p.reduce(A, list(range(na)), ka, 0, DT_BF16 if a_bf16 else DT_F32)
     p.reduce(B, [A] + list(range(na, n)), kb)
     p.broadcast(B, [500 + j for j in range(R)])
@@ -81,7 +96,7 @@ def _timeline(seed):
             e = p.o.objects[i]
             if e.alive:
                 nb_ = size_of[i] if rng.random() < 0.5 else min(size_of[i], prefix[i] + chunk)
-                p.put(i, nb_)
+                put(i, nb_)
                 prefix[i] = nb_
         elif r < 0.6:
             p.fail(int(rng.integers(0, n_workers)))
@@ -107,7 +122,7 @@ def _timeline(seed):
         if p.o.objects[i].alive:
             t = max(t + 5, p.o.now)
             p.advance(t)
-            p.put(i, size_of[i])
+            put(i, size_of[i])
     for oid in [A, B] + [500 + j for j in range(R)]:
         _get_both(p, oid, plan_ahead)
     p.check_schedule(A)
