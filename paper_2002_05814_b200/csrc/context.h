@@ -239,6 +239,7 @@ struct hpl_ctx {
     std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
     Journal journal;
     bool work_in_flight = false;
+    bool polling_in_flight = false;   // some wave in flight polls progress counters (only those can record an error)
     uint64_t launch_seq = 0;       // waves launched so far
     uint64_t first_unchecked = 0;  // the first wave whose error record has not been read back
     uint64_t batch_tag = 0;        // launch_seq when the current planning pass began

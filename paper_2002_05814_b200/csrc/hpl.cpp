@@ -99,6 +99,16 @@ int sync_and_check(hpl_ctx* c) {
         c->journal.clear();
         return HPL_OK;
     }
+    if (!c->polling_in_flight) {
+        // no wave in flight waits on a counter, so no error record can have been written: nothing to read back
+        CUDA_TRY(cudaStreamSynchronize(c->stream));
+        c->work_in_flight = false;
+        collect_kernel_times(c);
+        c->first_unchecked = c->launch_seq;
+        c->wave_tag.clear();
+        c->journal.clear();
+        return HPL_OK;
+    }
     const uint32_t used = (uint32_t)std::min<uint64_t>(c->launch_seq - c->first_unchecked, kStatusSlots);
     CUDA_TRY(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(DeviceStatus) * used, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(cudaStreamSynchronize(c->stream));
@@ -116,6 +126,7 @@ int sync_and_check(hpl_ctx* c) {
     }
     c->first_unchecked = c->launch_seq;
     c->wave_tag.clear();
+    c->polling_in_flight = false;
     // the records are cleared behind everything launched so far; later launches are ordered after that
     CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus) * used, c->stream));
     if (failed) {

@@ -121,6 +121,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
             d.dst_begin = n_dst;
             d.n_dst = (uint32_t)tt.dst.size();
             d.poll = tt.poll ? 1u : 0u;
+            if (tt.poll) c->polling_in_flight = true;
             d.bytes = src->bytes;
             d.chunk_bytes = chunk_bytes;
             for (int r : tt.dst) w.dst_rows[n_dst++] = (uint32_t)find(c, locs[r].obj)->row;

@@ -308,6 +308,7 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 d.n_steps = (uint32_t)t.steps.size();
                 d.red_op = (uint32_t)op.red_op;
                 d.poll = t.poll ? 1u : 0u;
+                if (t.poll) c->polling_in_flight = true;
                 d.pad = 0;
                 std::memcpy(&w.steps[n_steps], t.steps.data(), t.steps.size() * sizeof(ReduceStep));
                 n_steps += d.n_steps;
