@@ -177,7 +177,8 @@ int hpl_progress(hpl_ctx* ctx);
  * the next hpl_progress). */
 int hpl_sync(hpl_ctx* ctx);
 
-/* Serialises the schedule of the collective named by its reduce target id or broadcast source id into
+/* Serialises the schedule of the collective named by its reduce target id or broadcast source id (an id that is
+ * both names the Reduce; any receiver id names the broadcast it belongs to) into
  * `words` (capacity `cap` 64-bit words); `*len` receives the number of words needed (HPL_ERR_INVALID if
  * cap is too small; *len is still set).
  *   Reduce:    0x48504C52, target, n, k requested, k now, d, #placements, {object, position}*, object at each

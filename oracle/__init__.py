@@ -24,8 +24,13 @@ What each module restates:
                         Reduce / Delete (Table 1) driven by a timeline of events.
 
 Parity status of the parts the paper does not fix:
-the tree after a failure that leaves fewer live sources than requested ("shrink"), and
-the broadcast sender choice for more than one send slot per location, are build-defined
-readings -- **parity unpinned** beyond the invariants and brute-force value checks in
-``tests/test_oracle_*.py``.
+the tree after a failure that leaves fewer live sources than requested ("shrink"), the
+broadcast sender choice for more than one send slot per location, the order in which the
+orphans of one failure ask again, and the way a prefix crosses dtypes in composed collectives
+are build-defined readings.  Each is held to a hand-worked example under ``tests/golden/``
+(``reduce_shrink_example``, ``broadcast_two_slots_example``, ``broadcast_orphans_example``,
+``composition_cross_dtype``; ``tests/test_golden_rules.py``) besides the invariants and
+brute-force value checks in ``tests/test_oracle_*.py``.  One rule stays **parity unpinned**:
+the order in which SEVERAL waiting receivers are served -- no timeline was found in which two
+receivers wait at once (a second orphan can always fetch from the first).
 """

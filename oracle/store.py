@@ -260,6 +260,8 @@ class OracleStore:
             return self.reduces[op_id]["sched"].words(op_id)
         if op_id in self.bcasts:
             return self.bcasts[op_id]["sched"].words()
+        if op_id in self.dst_of:          # a receiver names the broadcast it belongs to
+            return self.bcasts[self.dst_of[op_id]]["sched"].words()
         raise StoreError(ERR_NOT_FOUND)
 
     # ------------------------------------------------------------------ helpers

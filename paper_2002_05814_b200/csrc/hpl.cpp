@@ -792,8 +792,14 @@ int hpl_schedule_dump(hpl_ctx* c, int64_t op_id, int64_t* words, uint64_t cap, u
         c->reduces.at(r->second).sched->dump(op_id, w);
     else if (b != c->bcast_of_src.end())
         c->bcasts.at(b->second).sched->dump(w);
-    else
-        return HPL_ERR_NOT_FOUND;
+    else {
+        // a receiver names the broadcast it belongs to (the only handle on it when the source is a Reduce output)
+        Object* o = find(c, op_id);
+        if (!o || o->kind != OBJ_RECEIVER) return HPL_ERR_NOT_FOUND;
+        auto bo = c->bcast_of_src.find(o->op_key);
+        if (bo == c->bcast_of_src.end()) return HPL_ERR_NOT_FOUND;
+        c->bcasts.at(bo->second).sched->dump(w);
+    }
     *len = w.size();
     if (!words || cap < w.size()) return HPL_ERR_INVALID;
     std::memcpy(words, w.data(), w.size() * sizeof(int64_t));
