@@ -230,7 +230,8 @@ const char* hpl_strerror(int code);
  * The few KiB of device memory the kernel needs besides inputs and output (directory rows of the operands,
  * status record) are a fixed array inside the library image, held by every GPU that loads the library until
  * the process exits.  Hence the limits: n <= HPL_NOALLOC_MAX_SOURCES and elems <= HPL_NOALLOC_MAX_ELEMS;
- * a tree deeper than the kernel can fuse in registers (8 accumulators) is refused too.  Anything beyond
+ * a tree deeper than the kernel can fuse in registers (8 accumulators) would be refused too (no degree reaches
+ * that depth within the limit on n).  Anything beyond
  * returns HPL_ERR_INVALID and does nothing.  No cudaMalloc / cudaFree / allocating routine is called.
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and the SM count;
  * make that first call outside any stream capture.  All calls share the one array and each call rewrites

@@ -22,7 +22,7 @@ class Pair:
         self.stream = torch.cuda.current_stream().cuda_stream
         self.c = hpl.Context(chunk_bytes, d_reduce, d_bcast, arena=self.arena.data_ptr(), arena_bytes=arena_bytes,
                              stream=self.stream, virt_chunk_ns=tau, **flags)
-        self.o = OracleStore(chunk_bytes, d_reduce, d_bcast, tau)
+        self.o = OracleStore(chunk_bytes, d_reduce, d_bcast, tau, flags.get("model_latency_ns", 0), flags.get("model_bandwidth_bps", 0))
         self.host: dict[int, np.ndarray] = {}
         self.dev: dict[int, torch.Tensor] = {}
         self.guarded: dict[int, torch.Tensor] = {}

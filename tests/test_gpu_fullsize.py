@@ -24,12 +24,13 @@ def _lib():
 
 
 def _windows(elems, chunk_elems, rng, n_random=6, width=5000):
+    width = min(width, elems)
     w = [(0, width), (elems - width, elems), (elems - 3, elems)]
     if elems > chunk_elems:
         last = (elems - 1) // chunk_elems * chunk_elems
         w += [(chunk_elems - 100, chunk_elems + 100), (last - 64, min(elems, last + 4096 + 64))]
     for _ in range(n_random):
-        lo = int(rng.integers(0, elems - width))
+        lo = int(rng.integers(0, elems - width + 1))
         w.append((lo, lo + width))
     return [(max(0, a), min(elems, b)) for a, b in w]
 
@@ -105,33 +106,45 @@ def test_cfg2_broadcast_64mib_to_16_receivers():
     c.shutdown()
 
 
-def test_cfg3_one_round_first_8_of_16_gradients():
+def test_cfg3_fifty_rounds_first_8_of_16_gradients():
+    """All 50 rounds of the async-SGD configuration, each with fresh object contents and fresh arrival times
+    (seed = base + round).  The context and its arena are reused: every round ends with its Deletes."""
     w = wl.workload("cfg3")
     S = w.object_bytes
     arena, c = _ctx(w, (64 << 20) + 2 * S)
-    sh = Shadow(w)
-    seeds = {i: w.seed + i for i in range(16)}
-    dev = [wl.values_torch(w.dist, seeds[i], i, 0, w.elems, "f32") for i in range(16)]
-    for i in range(16):
-        c.create(i, i, S)
-        sh.o.create(i, i, S, DT_F32)
-    c.reduce(100, list(range(16)), 8)
-    sh.o.reduce(100, list(range(16)), 8)
-    arr = wl.exponential_arrivals_ns(w.seed, 16, w.extra["mean_arrival_ns"])
-    for i in sorted(range(16), key=lambda i: (arr[i], i)):
-        c.advance(arr[i])
-        sh.o.advance(arr[i])
-        c.put(i, dev[i].data_ptr(), S)
-        sh.o.put(i, sh.placeholder(S, DT_F32), S)
-    ptr, n = c.get(100)
-    assert n == w.elems * 4 and c.schedule_dump(100) == sh.o.dump(100)
-    off = ptr - arena.data_ptr()
-    out = arena[off:off + n].view(torch.float32)
-    obj_at = sh.o.reduces[100]["sched"].obj_at
-    assert sorted(obj_at) == sorted(sorted(range(16), key=lambda i: (arr[i], i))[:8])
-    _check_reduce_windows(w, obj_at, seeds, out, np.random.default_rng(1))
-    st = c.stats()
-    assert st["kernel_launches"] == 1 and st["bytes_read_planned"] == 8 * S
+    rng = np.random.default_rng(1)
+    t0 = 0
+    for rnd in range(50):
+        sh = Shadow(w)
+        seeds = {i: w.seed + rnd for i in range(16)}          # contents are a function of (seed, object index)
+        dev = [wl.values_torch(w.dist, seeds[i], i, 0, w.elems, "f32") for i in range(16)]
+        t0 += 1_000_000_000
+        c.advance(t0)
+        sh.o.advance(t0)
+        for i in range(16):
+            c.create(i, i, S)
+            sh.o.create(i, i, S, DT_F32)
+        c.reduce(100, list(range(16)), 8)
+        sh.o.reduce(100, list(range(16)), 8)
+        arr = wl.exponential_arrivals_ns(w.seed + rnd, 16, w.extra["mean_arrival_ns"])
+        for i in sorted(range(16), key=lambda i: (arr[i], i)):
+            c.advance(t0 + arr[i])
+            sh.o.advance(t0 + arr[i])
+            c.put(i, dev[i].data_ptr(), S)
+            sh.o.put(i, sh.placeholder(S, DT_F32), S)
+        st0 = c.stats()
+        ptr, n = c.get(100)
+        assert n == w.elems * 4 and c.schedule_dump(100) == sh.o.dump(100)
+        off = ptr - arena.data_ptr()
+        out = arena[off:off + n].view(torch.float32)
+        obj_at = sh.o.reduces[100]["sched"].obj_at
+        assert sorted(obj_at) == sorted(sorted(range(16), key=lambda i: (arr[i], i))[:8])
+        _check_reduce_windows(w, obj_at, seeds, out, rng)
+        st = c.stats()
+        assert st["kernel_launches"] - st0["kernel_launches"] == 1 and st["bytes_read_planned"] - st0["bytes_read_planned"] == 8 * S
+        for i in [100] + list(range(16)):
+            c.delete(i)
+        del dev
     c.shutdown()
 
 
@@ -181,7 +194,7 @@ def test_cfg4_policy_round_bf16():
     c.shutdown()
 
 
-@pytest.mark.parametrize("size", [64 << 20, 4 << 20, 1 << 30])
+@pytest.mark.parametrize("size", [(1 << 10) << (2 * j) for j in range(11)])     # 1 KiB ... 1 GiB in powers of 4
 def test_cfg5_fault_tolerant_reduce(size):
     w = wl.cfg5_at(size)
     S = w.object_bytes
@@ -190,6 +203,7 @@ def test_cfg5_fault_tolerant_reduce(size):
     seeds = {i: w.seed + i for i in range(32)}
     dev = [wl.values_torch(w.dist, seeds[i], i, 0, w.elems, "f32") for i in range(32)]
     C = wl.n_chunks(S, w.chunk_bytes)
+    assert w.chunk_bytes == min(4 << 20, S)          # the configuration's own chunk: whole object if smaller
     h = int(0.4 * C)
     for i in range(32):
         c.create(i, i, S)

@@ -106,6 +106,23 @@ def test_min_max(op):
     p.close()
 
 
+@pytest.mark.parametrize("elems,want_d", [(256, 8), (25_000, 2), (400_000, 1)])
+def test_degree_chosen_per_reduce_by_eq_1(elems, want_d):
+    """reduce_degree = 0: the degree comes from Eq. 1 with the context's latency / bandwidth model (Section 4).
+    With L = 10 us and B = 10 GB/s and 8 objects: 1 KiB -> the star, 100 KB -> binary, 1.6 MB -> the chain."""
+    p = Pair(16 << 10, 0, model_latency_ns=10_000, model_bandwidth_bps=10_000_000_000)
+    for i in range(8):
+        p.create(i, i, gen(("uniform",), 13, i, elems))
+        p.advance(i + 1)
+        p.put(i)
+    p.reduce(100, list(range(8)), 8)
+    p.check_schedule(100)
+    assert p.c.schedule_dump(100)[5] == want_d == hpl.choose_degree(8, elems * 4, 10e-6, 10e9)
+    got = p.check_target_bits(100).cpu().numpy()
+    assert _norm_err(got, ov.naive_sum_f64(list(range(8)), p.host)) <= 1e-5 * 3
+    p.close()
+
+
 @pytest.mark.parametrize("fuse", [True, False])
 def test_progress_between_arrivals_materialises_and_reuses_partials(fuse):
     """Objects arrive one by one and the library is asked to progress after each: subtrees are
