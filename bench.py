@@ -136,9 +136,9 @@ class Runner:
         if w.kind == "ft_reduce":
             arena_bytes += 8 * w.elems * 4       # partial results of the subtrees beside the failing worker's root path
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
-        self.ctx = hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=arena_bytes,
-                               stream=torch.cuda.current_stream().cuda_stream, time_kernels=True,
-                               plan_ahead=plan_ahead)
+        self.plan_ahead = plan_ahead
+        self.ctx = None
+        self.open_context(time_kernels=False)
         self.src = [wl.values_torch(w.dist, w.seed + i, i, 0, w.elems, w.dtype, device=device) for i in range(n_src)]
         self.policy = None
         self.recv = []
@@ -154,120 +154,133 @@ class Runner:
                 self.host_recv = torch.empty(S, dtype=torch.uint8).pin_memory()
             if n_src:
                 self.host_out = torch.empty(w.elems, dtype=torch.float32).pin_memory()
-        # argument arrays of the batch calls (events that share one time are submitted together)
-        C = self.ctx
-        self.a_dst_ids = C.ids_array([6000 + j for j in range(w.n_receivers)])
-        self.a_dst_workers = [1000 + j for j in range(w.n_receivers)]
-        self.a_dst_ptrs = C.ptr_array([t.data_ptr() for t in self.recv])
-        self.a_dst_out = C.ptr_array([0] * w.n_receivers)
-        self.a_src_ids = C.ids_array(list(range(n_src)))
-        self.a_src_workers = list(range(n_src))
-        self.a_src_ptrs = C.ptr_array([t.data_ptr() for t in self.src])
         self.round = 0
-        self.t = 0
+        self.prepared = {}
         torch.cuda.synchronize()
+
+    def open_context(self, time_kernels: bool):
+        """(Re)creates the context on the same arena and buffers.  Per-launch event timing is a mode of its own: its
+        two event records per launch would otherwise sit inside the step times they are compared with."""
+        torch, w = self.torch, self.w
+        if self.ctx is not None:
+            self.ctx.shutdown()
+        self.ctx = self.hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=self.arena.numel(),
+                                    stream=torch.cuda.current_stream().cuda_stream, time_kernels=time_kernels,
+                                    plan_ahead=self.plan_ahead)
+        self.prepared = {}
 
     def close(self):
         self.ctx.shutdown()
 
-    # one pass of the whole path; returns (h2d bytes, d2h bytes) of the step
-    def step(self):
-        w, ctx, r = self.w, self.ctx, self.round
-        base = 0
+    # ---- the timeline of one round, prepared outside the timed region (it is input data, like the objects)
+    def build_round(self, r: int, marks=None):
+        """Event lists of round ``r``: (first part, second part, deletes, h2d bytes, d2h bytes).  The first part
+        holds the broadcast of the round (if any), the second the reduce; each is applied by ONE hpl_submit.
+        ``marks``: three CUDA event handles the library records on its stream at the start of the step, between
+        the two parts and at the end (device timing without a foreign call of its own)."""
+        H, w = self.hpl, self.w
         S = w.object_bytes
+        t = (r + 1) * 2_000_000_000
+        n, R = w.n_objects, w.n_receivers
+        e1, e2, dl = H.EventList(12 + 3 * R + n), H.EventList(12 + 3 * n), H.EventList(4 + n)
         h2d = d2h = 0
-        self.t += 1_000_000_000
-        ctx.advance(self.t)
-        ids_to_delete = []
+        put_kind = H.HPL_EV_PUT_HOST if self.host_buffers else H.HPL_EV_PUT
+        ids = list(range(n))
+        tgt = 9000
+        early = w.kind == "round" and not self.host_buffers
+        first = e1 if w.kind in ("broadcast", "round") else e2
+        if marks:
+            first.add(H.HPL_EV_MARK, 0, ptr=marks[0])
         if w.kind in ("broadcast", "round"):
-            src_id = base + 5000
-            dsts = [base + 6000 + j for j in range(w.n_receivers)]
-            ctx.create(src_id, 900, S, self.dt)
+            src_id = 5000
+            dsts = [6000 + j for j in range(R)]
+            e1.add(H.HPL_EV_CREATE, t, src_id, 900, nbytes=S, dtype=self.dt)
             if self.host_buffers:
-                ctx.put_host(src_id, self.host_policy.data_ptr(), S)
+                e1.add(put_kind, t, src_id, ptr=self.host_policy.data_ptr(), nbytes=S)
                 h2d += S
             else:
-                ctx.put(src_id, self.policy.data_ptr(), S)
-            ctx.create_batch(self.a_dst_ids, self.a_dst_workers, S, self.dt)
-            ctx.broadcast(src_id, dsts)
+                e1.add(put_kind, t, src_id, ptr=self.policy.data_ptr(), nbytes=S)
+            for j in range(R):
+                e1.add(H.HPL_EV_CREATE, t, dsts[j], 1000 + j, nbytes=S, dtype=self.dt)
+            e1.add(H.HPL_EV_BROADCAST, t, src_id, ids=dsts)
             if w.kind == "broadcast":
-                offs = wl.uniform_offsets_ns(w.seed + r, w.n_receivers, w.extra["join_window_ns"])
-                order = sorted(range(w.n_receivers), key=lambda j: (offs[j], j))
-                for j in order:
-                    ctx.advance(self.t + offs[j])
-                    ctx.join(dsts[j], self.recv[j].data_ptr())
-                self.t += w.extra["join_window_ns"]
+                offs = wl.uniform_offsets_ns(w.seed + r, R, w.extra["join_window_ns"])
+                for j in sorted(range(R), key=lambda j: (offs[j], j)):
+                    e1.add(H.HPL_EV_JOIN, t + offs[j], dsts[j], ptr=self.recv[j].data_ptr())
+                t += w.extra["join_window_ns"]
             else:
-                ctx.join_batch(self.a_dst_ids, self.a_dst_ptrs)
-            if w.kind == "round" and not self.host_buffers:
+                for j in range(R):
+                    e1.add(H.HPL_EV_JOIN, t, dsts[j], ptr=self.recv[j].data_ptr())
+            if early:
                 # the Reduce of the objects the workers will return is requested with futures while the
                 # broadcast is still running (the pattern of the paper's Fig. 1)
-                ctx.progress()
-                ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
-                ctx.reduce(base + 9000, [base + i for i in range(w.n_objects)], w.k, self.hpl.HPL_SUM, self.dt)
-            ctx.get_batch(self.a_dst_ids, self.a_dst_out)      # every receiver's Get
-            if self.host_buffers:
-                ctx.get_host(dsts[-1], self.host_recv.data_ptr(), S)
-                d2h += S
-            self.t += 100_000_000          # the Gets let virtual time run until the copies had landed
-            ctx.advance(self.t)
-            ids_to_delete.append(src_id)
-        self.mid_event()
+                e1.add(H.HPL_EV_PROGRESS)
+                for i in ids:
+                    e1.add(H.HPL_EV_CREATE, t, i, i, nbytes=S, dtype=self.dt)
+                e1.add(H.HPL_EV_REDUCE, t, tgt, ids=ids, k=w.k, op=H.HPL_SUM, dtype=self.dt)
+            for j in range(R):
+                e1.add(H.HPL_EV_GET, 0, dsts[j])          # every receiver's Get
+            t += 200_000_000                             # the Gets let virtual time run until the copies had landed
+            dl.add(H.HPL_EV_DELETE, 0, src_id)
+        if marks:
+            first.add(H.HPL_EV_MARK, 0, ptr=marks[1])
         if w.kind in ("reduce", "round", "ft_reduce"):
-            n = w.n_objects
-            ids = [base + i for i in range(n)]
-            tgt = base + 9000
-            early = w.kind == "round" and not self.host_buffers      # created and requested above
             if not early:
-                ctx.create_batch(self.a_src_ids, self.a_src_workers, S, self.dt)
+                for i in ids:
+                    e2.add(H.HPL_EV_CREATE, t, i, i, nbytes=S, dtype=self.dt)
+                e2.add(H.HPL_EV_REDUCE, t, tgt, ids=ids, k=w.k, op=H.HPL_SUM, dtype=self.dt)
             if w.kind == "reduce" and "mean_arrival_ns" in w.extra:
                 arr = wl.exponential_arrivals_ns(w.seed + r, n, w.extra["mean_arrival_ns"])
             else:
                 arr = [0] * n
-            order = sorted(range(n), key=lambda i: (arr[i], i))
-            if not early:
-                ctx.reduce(tgt, ids, w.k, self.hpl.HPL_SUM, self.dt)
-            tmax = 0
-            if not self.host_buffers and max(arr) == 0:           # all objects are put at the same instant: one call
-                if w.kind == "ft_reduce":
-                    fw = w.extra["fail_worker"]
-                    part = int(w.extra["fail_fraction"] * wl.n_chunks(S, w.chunk_bytes)) * w.chunk_bytes
-                    sel = [i for i in range(n) if i != fw or part > 0]
-                    ctx.put_batch([ids[i] for i in sel], [self.src[i].data_ptr() for i in sel],
-                                  [part if i == fw else S for i in sel])
-                else:
-                    ctx.put_batch(self.a_src_ids, self.a_src_ptrs, S)
-                order = []
-            for i in order:
-                ctx.advance(max(self.t + arr[i], self.t + tmax))
-                tmax = max(tmax, arr[i])
+            for i in sorted(ids, key=lambda i: (arr[i], i)):
                 nbytes = S
                 if w.kind == "ft_reduce" and i == w.extra["fail_worker"]:
-                    C = wl.n_chunks(S, w.chunk_bytes)
-                    nbytes = int(w.extra["fail_fraction"] * C) * w.chunk_bytes
+                    nbytes = int(w.extra["fail_fraction"] * wl.n_chunks(S, w.chunk_bytes)) * w.chunk_bytes
                     if nbytes == 0:
                         continue
                 if self.host_buffers:
-                    ctx.put_host(ids[i], self.host_src[i % len(self.host_src)].data_ptr(), nbytes)
+                    e2.add(put_kind, t + arr[i], i, ptr=self.host_src[i % len(self.host_src)].data_ptr(), nbytes=nbytes)
                     h2d += nbytes
                 else:
-                    ctx.put(ids[i], self.src[i].data_ptr(), nbytes)
-            self.t += tmax
+                    e2.add(put_kind, t + arr[i], i, ptr=self.src[i].data_ptr(), nbytes=nbytes)
+            t += max(arr)
             if w.kind == "ft_reduce":
                 if self.ft_eager:
-                    ctx.progress()                   # chunks delivered by every worker are reduced before the failure
-                self.t += 1
-                ctx.advance(self.t)
-                ctx.fail(w.extra["fail_worker"])
+                    e2.add(H.HPL_EV_PROGRESS)            # chunks delivered by every worker are reduced before the failure
+                e2.add(H.HPL_EV_FAIL, t + 1, worker=w.extra["fail_worker"])
+            if not self.host_buffers:
+                e2.add(H.HPL_EV_GET, 0, tgt)
+            for i in [tgt] + ids:
+                dl.add(H.HPL_EV_DELETE, 0, i)
+        if marks:
+            (e2 if len(e2) else e1).add(H.HPL_EV_MARK, 0, ptr=marks[2])
+        return e1, e2, dl, h2d, d2h
+
+    def prepare(self, n_rounds: int, marks=None):
+        for i, r in enumerate(range(self.round, self.round + n_rounds)):
+            self.prepared[r] = self.build_round(r, marks[i] if marks else None)
+
+    # one pass of the whole path; returns (h2d bytes, d2h bytes) of the step
+    def step(self):
+        w, ctx = self.w, self.ctx
+        if self.round not in self.prepared:
+            self.prepare(1)
+        e1, e2, dl, h2d, d2h = self.prepared.pop(self.round)
+        S = w.object_bytes
+        if len(e1):
+            ctx.submit(e1)
             if self.host_buffers:
-                ctx.get_host(tgt, self.host_out.data_ptr(), w.elems * 4)
+                ctx.get_host(6000 + w.n_receivers - 1, self.host_recv.data_ptr(), S)
+                d2h += S
+        self.mid_event()
+        if len(e2):
+            ctx.submit(e2)
+            if self.host_buffers:
+                ctx.get_host(9000, self.host_out.data_ptr(), w.elems * 4)
                 d2h += w.elems * 4
-            else:
-                ctx.get(tgt)
-            ids_to_delete += [tgt] + ids
         self.end_event()
-        for i in ids_to_delete:
-            ctx.delete(i)
+        ctx.submit(dl)
         self.round += 1
         return h2d, d2h
 
@@ -280,12 +293,23 @@ class Runner:
 
 def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
     torch = runner.torch
+    runner.prepare(warmup)              # the timelines are inputs: built before the timed region
     for _ in range(warmup):
         runner.step()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
     cur = {"i": 0}
-    runner.mid_event = lambda: ev[cur["i"]][1].record()
-    runner.end_event = lambda: ev[cur["i"]][2].record()
+    if runner.host_buffers:
+        # the end-to-end step leaves the library between its parts (hpl_get_host): events recorded from here
+        runner.prepare(steps)
+        runner.mid_event = lambda: ev[cur["i"]][1].record()
+        runner.end_event = lambda: ev[cur["i"]][2].record()
+    else:
+        # device-resident step: the library records the three events itself, inside hpl_submit (HPL_EV_MARK)
+        for tri in ev:
+            for e in tri:
+                e.record()              # creates the underlying CUDA event
+        torch.cuda.synchronize()
+        runner.prepare(steps, [[e.cuda_event for e in tri] for tri in ev])
     st0 = runner.ctx.stats()
     if dist is not None:
         dist.barrier()
@@ -294,7 +318,8 @@ def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
     h2d = d2h = 0
     for i in range(steps):
         cur["i"] = i
-        ev[i][0].record()
+        if runner.host_buffers:
+            ev[i][0].record()
         a, b = runner.step()
         h2d, d2h = a, b
     torch.cuda.synchronize()
@@ -553,6 +578,10 @@ def main():
     sampler.start()
     res = time_steps(runner, args.steps, args.warmup, dist)
     clocks = sampler.stop()
+    # per-launch device times for the roofline come from a short pass of their own, with event timing switched on
+    k_steps = max(1, min(args.steps, 10))
+    runner.open_context(time_kernels=True)
+    res_k = time_steps(runner, k_steps, 3)
     runner.close()
     del runner
     torch.cuda.empty_cache()
@@ -560,7 +589,7 @@ def main():
     total_ms, wall_ms = max_over_ranks([float(np.sum(res["total_ms"])), res["wall_ms"]], dist, device)
     value = whole_job_value(step_bytes, args.steps, world, total_ms)
     peak, peak_kind = measured_peak()
-    st = res["stats"]
+    st = res_k["stats"]
 
     def roof(kind_ns, kind_launches, per_launch_bytes, traffic=None):
         if st[kind_launches] == 0:
@@ -572,20 +601,20 @@ def main():
                 "algorithmic_bytes_per_launch": per_launch_bytes, "frac_of_8TBs_nominal": ach / 8000.0}
 
     traf = NCU_TRAFFIC.get(w.name, {}) if args.shrink == 1 else {}
-    r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * args.steps / max(1, st["reduce_launches"]), traf.get("reduce")) if ab["reduce"] else None
-    r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * args.steps / max(1, st["fanout_launches"]), traf.get("fanout")) if ab["broadcast"] else None
+    r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * k_steps / max(1, st["reduce_launches"]), traf.get("reduce")) if ab["reduce"] else None
+    r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * k_steps / max(1, st["fanout_launches"]), traf.get("fanout")) if ab["broadcast"] else None
     line = {"metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value, "unit": "GB/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if w.dtype == "f32" else "f32 (bf16 inputs widened)", "data": "synthetic",
-            "config": config, "clocks": clocks, "gpu_launches": int(st["kernel_launches"]),
+            "config": config, "clocks": clocks, "gpu_launches": int(res["stats"]["kernel_launches"]),
             "wall_ms_per_step": wall_ms / args.steps,
             "frac_of_hbm_peak": {"measured_copy": value / world / peak, "nominal_8TBs": value / world / 8000.0},
             "roofline": r_red if r_red is not None else r_fan}
     if r_red is not None and r_fan is not None:
         line["roofline_fanout"] = r_fan
-    planned = (st["bytes_read_planned"] + st["bytes_written_planned"]) / args.steps
-    kern_ms = (st["reduce_kernel_ns"] + st["fanout_kernel_ns"]) / 1e6 / args.steps
+    planned = (st["bytes_read_planned"] + st["bytes_written_planned"]) / k_steps
+    kern_ms = (st["reduce_kernel_ns"] + st["fanout_kernel_ns"]) / 1e6 / k_steps
     line["planned_traffic"] = {"bytes_per_step": planned, "over_algorithmic": planned / step_bytes,
                                "kernel_GBps_on_planned_bytes": gbs(planned, kern_ms), "kernel_ms_per_step": kern_ms}
     if w.kind == "ft_reduce":
@@ -612,16 +641,19 @@ def main():
                     torch.cuda.empty_cache()
                 rr = Runner(ww, device, ft_eager=eager)
             rr.ft_eager = eager                  # the two cfg5 modes share the 32 GiB of inputs
-            n2 = 3 if ww.name == "cfg5" else 5
+            n2 = 3 if ww.name == "cfg5" else 10
+            rr.open_context(time_kernels=False)
             r2 = time_steps(rr, n2, 3)
             a2 = algorithmic_bytes(ww)
             b2 = a2["reduce"] + a2["broadcast"]
             g = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
-            s2 = r2["stats"]
+            rr.open_context(time_kernels=True)
+            s2 = time_steps(rr, n2, 1)["stats"]
             kns = s2["reduce_kernel_ns"] + s2["fanout_kernel_ns"]
             planned = s2["bytes_read_planned"] + s2["bytes_written_planned"]
             kern = gbs(planned, kns / 1e6)       # bytes the planned tasks move / their summed launch time
-            also[label] = {"GBps": g, "ms_per_step": float(np.mean(r2["total_ms"])), "kernel_GBps": kern,
+            also[label] = {"GBps": g, "frac_of_measured_copy": g / peak, "ms_per_step": float(np.mean(r2["total_ms"])),
+                           "ms_std": float(np.std(r2["total_ms"])), "steps": n2, "kernel_GBps": kern,
                            "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / n2,
                            "planned_over_algorithmic_bytes": planned / (b2 * n2)}
         if rr is not None:

@@ -119,6 +119,57 @@ int hpl_put_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const void
 int hpl_join_batch(hpl_ctx* ctx, int32_t n, const int64_t* dst_ids, void* const* dst_bufs /* host array of DEVICE
                    pointers */, int32_t* n_done);
 
+/* A timeline handed over in one call: `n` events in non-decreasing time, each applied exactly as the single call
+ * of its kind would be (the same checks, the same codes).  A harness that stands for many task workers -- or a
+ * framework that has collected a round's requests -- thereby pays one foreign call for a whole round instead of one
+ * per worker.  Before each event the clock is set to its t_ns as by hpl_advance (t_ns == 0: the clock stays).
+ * Stops at the first event that fails and returns its code; *n_done (may be NULL) receives how many were applied.
+ * HPL_EV_GET writes its results back into the event (ptr, bytes): the array is in/out.
+ *
+ *   kind               fields used
+ *   HPL_EV_CREATE      object_id, worker, bytes (total size), dtype            -> hpl_create
+ *   HPL_EV_PUT         object_id, ptr (DEVICE buffer), bytes (valid prefix)     -> hpl_put
+ *   HPL_EV_PUT_HOST    object_id, ptr (HOST buffer), bytes                      -> hpl_put_host
+ *   HPL_EV_REDUCE      object_id (target), ids (host array of n_ids sources), k, op, dtype -> hpl_reduce
+ *   HPL_EV_BROADCAST   object_id (source), ids (host array of n_ids receivers)  -> hpl_broadcast
+ *   HPL_EV_JOIN        object_id (receiver), ptr (DEVICE buffer)                -> hpl_join
+ *   HPL_EV_FAIL        worker                                                   -> hpl_fail
+ *   HPL_EV_REJOIN      worker                                                   -> hpl_rejoin
+ *   HPL_EV_PROGRESS    --                                                       -> hpl_progress
+ *   HPL_EV_GET         object_id; out: ptr (device pointer), bytes              -> hpl_get
+ *   HPL_EV_DELETE      object_id                                                -> hpl_delete
+ *   HPL_EV_SYNC        --                                                       -> hpl_sync
+ *   HPL_EV_MARK        ptr (a cudaEvent_t of the caller): recorded on the context's stream at this point of the
+ *                      timeline, so that a harness can time parts of it on the device without leaving the call
+ * Events at one time must come in the order the Conventions give (failures, creations / puts, requests). */
+#define HPL_EV_CREATE    1
+#define HPL_EV_PUT       2
+#define HPL_EV_PUT_HOST  3
+#define HPL_EV_REDUCE    4
+#define HPL_EV_BROADCAST 5
+#define HPL_EV_JOIN      6
+#define HPL_EV_FAIL      7
+#define HPL_EV_REJOIN    8
+#define HPL_EV_PROGRESS  9
+#define HPL_EV_GET       10
+#define HPL_EV_DELETE    11
+#define HPL_EV_SYNC      12
+#define HPL_EV_MARK      13
+typedef struct hpl_event {
+    uint64_t t_ns;
+    int32_t  kind;
+    int32_t  worker;
+    int64_t  object_id;
+    void*    ptr;
+    uint64_t bytes;
+    const int64_t* ids;
+    int32_t  n_ids;
+    int32_t  k;
+    int32_t  op;
+    int32_t  dtype;
+} hpl_event;
+int hpl_submit(hpl_ctx* ctx, hpl_event* events, int32_t n, int32_t* n_done);
+
 /* Many hpl_get calls, in array order; dev_ptrs[i] (may be NULL as a whole) receives the pointer of object i.
  * Stops at the first failure and returns its code. */
 int hpl_get_batch(hpl_ctx* ctx, int32_t n, const int64_t* object_ids, const void** dev_ptrs, int32_t* n_done);

@@ -9,4 +9,6 @@ from .hpl import (  # noqa: F401
     HPL_F32, HPL_BF16, HPL_SUM, HPL_MIN, HPL_MAX,
     HPL_OK, HPL_ERR_INVALID, HPL_ERR_NOT_FOUND, HPL_ERR_EXISTS, HPL_ERR_TIMEOUT,
     HPL_ERR_INSUFFICIENT, HPL_ERR_FAILED_WORKER, HPL_ERR_CUDA, HPL_ERR_NOMEM,
+    Event, EventList, HPL_EV_CREATE, HPL_EV_PUT, HPL_EV_PUT_HOST, HPL_EV_REDUCE, HPL_EV_BROADCAST, HPL_EV_JOIN,
+    HPL_EV_FAIL, HPL_EV_REJOIN, HPL_EV_PROGRESS, HPL_EV_GET, HPL_EV_DELETE, HPL_EV_SYNC, HPL_EV_MARK,
 )

@@ -220,6 +220,7 @@ struct hpl_ctx {
     bool device = false;
     bool copy_pending = false;
     bool ctl_pending = false;   // directory updates on the control stream not yet ordered before the main stream
+    bool ctl_unconfirmed = false;   // counters of device puts went out on the control stream (plan-ahead) and no wait has confirmed them
     int n_sm = 0;
     uint64_t now = 0, tau = 1, seq = 0;
     int64_t next_internal = -1;  // ids of partial buffers: negative, never visible outside

@@ -38,13 +38,24 @@ enum : uint8_t { SRC_F32 = 0, SRC_BF16 = 1 };
 
 // One step of a fused subtree evaluation.  LOAD: acc[a] = operand; ADD_LOAD: acc[a] = acc[a] (+) operand;
 // ADD_ACC: acc[a] = acc[a] (+) acc[b].  The result of a task is acc[0].
+// A step travels to the kernel as one 64-bit record: the operand's device address in the low 56 bits (known to
+// the planner when the task is planned, so a launch does not depend on a directory update that is still on its
+// way) and, in the top byte, code (2 bits), accumulator (3 bits), operand kind (1 bit).  The directory row of
+// the operand travels beside it: it is what a polling task waits on.
 struct ReduceStep {
     uint8_t code;
     uint8_t a;
     uint8_t b;
     uint8_t kind;       // SRC_F32 / SRC_BF16 for loads
     uint32_t row;       // directory row of the operand
+    unsigned long long ptr;   // device address of the operand (loads)
 };
+
+constexpr int kRecShift = 56;
+inline unsigned long long pack_step(const ReduceStep& st) {
+    const unsigned long long meta = (unsigned long long)st.code | ((unsigned long long)st.a << 2) | ((unsigned long long)st.kind << 5);
+    return (st.ptr & ((1ull << kRecShift) - 1)) | (meta << kRecShift);
+}
 
 struct ReduceTask {
     unsigned long long out_ptr;   // fp32 result (partial or target)
@@ -69,11 +80,13 @@ struct ReduceWave {
     uint32_t n_tasks;
     uint32_t total_tiles;
     ReduceTask tasks[kMaxTasksPerWave];
-    ReduceStep steps[kMaxStepsPerWave];
+    unsigned long long recs[kMaxStepsPerWave];   // packed steps (pack_step)
+    uint32_t rows[kMaxStepsPerWave];             // directory row of each load step's operand
 };
 
 struct FanoutTask {
-    uint32_t src_row;
+    unsigned long long src_ptr;      // device address of the copy that is read
+    uint32_t src_row;                // its directory row (polled when the task polls)
     uint32_t c_begin, c_end;
     uint32_t tiles_per_chunk;
     uint32_t tile_begin;
@@ -93,7 +106,7 @@ struct FanoutWave {
     uint32_t n_tasks;
     uint32_t total_tiles;
     FanoutTask tasks[kMaxFanoutTasks];
-    uint32_t dst_rows[kMaxFanoutDst];
+    unsigned long long dst_ptrs[kMaxFanoutDst];   // device addresses of the receivers' buffers
 };
 
 // Launchers (kernels.cu).  Return a cudaError_t as int.

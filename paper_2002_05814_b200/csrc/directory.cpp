@@ -67,23 +67,16 @@ int alloc_row(hpl_ctx* c, Object& o) {
     r.ready_chunks = (o.kind == OBJ_PLAIN) ? 0u : o.C;
     r.dtype = (unsigned)o.dtype;
     r.owner = (unsigned)o.worker;
-    // With plan-ahead a kernel that polls may occupy the main stream for a while, so directory rows travel
-    // on the control stream (tiny copies only) and the main stream is ordered after it before each launch.
-    if (!c->device) {
-        // schedule-only context: the mirror is all there is (the planners run, nothing is launched)
-    } else if (c->cfg.plan_ahead) {
-        CUDA_TRY(cudaMemcpyAsync(c->d_dir + o.row, &r, sizeof(DirRow), cudaMemcpyHostToDevice, c->ctl_stream));
-        c->ctl_pending = true;
-    } else {
-        c->dirty_rows.push_back(o.row);   // travels with the next flush, before the next launch
-    }
+    // The row travels with the next flush (below), from a snapshot: the mirror itself keeps changing.
+    if (c->device) c->dirty_rows.push_back(o.row);
     return HPL_OK;
 }
 
 
-// Batched mode (no plan-ahead): all rows changed since the last flush go to the device in one copy per run of
-// consecutive rows, from an immutable pinned snapshot, ordered on the main stream before whatever is
-// launched next.  A Put is then a few stores on the host; its cost on the device is amortised over the batch.
+// All rows changed on the host since the last flush go to the device in one copy per run of consecutive rows,
+// from an immutable pinned snapshot, on the control stream: tiny copies only, which no polling kernel can hold
+// up.  Kernels get the addresses of their operands with the launch, so a launch does not wait for these copies;
+// only a wave that POLLS progress counters is ordered behind them (order_main_after_control).
 int flush_directory(hpl_ctx* c) {
     if (!c->device) c->dirty_rows.clear();
     if (c->dirty_rows.empty()) return HPL_OK;
@@ -95,16 +88,17 @@ int flush_directory(hpl_ctx* c) {
         while (j < c->dirty_rows.size() && c->dirty_rows[j] == c->dirty_rows[j - 1] + 1) ++j;
         const uint32_t n = (uint32_t)(j - i);
         if (c->stage_cursor + n > kStageRows) {
-            CUDA_TRY(cudaStreamSynchronize(c->stream));   // every earlier snapshot has been consumed
+            CUDA_TRY(cudaStreamSynchronize(c->ctl_stream));   // every earlier snapshot has been consumed
             c->stage_cursor = 0;
         }
         DirRow* snap = c->h_stage + c->stage_cursor;
         std::memcpy(snap, c->h_dir + c->dirty_rows[i], n * sizeof(DirRow));
-        CUDA_TRY(cudaMemcpyAsync(c->d_dir + c->dirty_rows[i], snap, n * sizeof(DirRow), cudaMemcpyHostToDevice, c->stream));
+        CUDA_TRY(cudaMemcpyAsync(c->d_dir + c->dirty_rows[i], snap, n * sizeof(DirRow), cudaMemcpyHostToDevice, c->ctl_stream));
         c->stage_cursor += n;
         i = j;
     }
     c->dirty_rows.clear();
+    c->ctl_pending = true;
     return HPL_OK;
 }
 
@@ -116,17 +110,19 @@ int order_main_after_control(hpl_ctx* c) {
     return HPL_OK;
 }
 
-// Publishes the chunk prefix of a put object in the device directory, ordered on `s`.
+// Publishes the chunk prefix of a put object in the device directory.  On the copy stream (chunks of a host
+// object, behind the copy that brings them) it is a 4-byte update of the counter alone; otherwise the row is
+// marked changed and travels with the next flush -- at once when kernels may be polling for it (plan-ahead).
 int publish_counter(hpl_ctx* c, Object& o, uint32_t chunks, cudaStream_t s) {
     if (o.row < 0) return HPL_OK;
     c->h_dir[o.row].ready_chunks = chunks;   // the host mirror always holds the published value
     if (!c->device) return HPL_OK;
-    if (s == c->stream && !c->cfg.plan_ahead) {
-        c->dirty_rows.push_back(o.row);
+    if (s == c->copy_stream) {
+        CUDA_TRY(cudaMemcpyAsync(&c->d_dir[o.row].ready_chunks, &c->h_iota[chunks], sizeof(uint32_t), cudaMemcpyHostToDevice, s));
         return HPL_OK;
     }
-    CUDA_TRY(cudaMemcpyAsync(&c->d_dir[o.row].ready_chunks, &c->h_iota[chunks], sizeof(uint32_t), cudaMemcpyHostToDevice, s));
-    return HPL_OK;
+    c->dirty_rows.push_back(o.row);
+    return c->cfg.plan_ahead ? flush_directory(c) : HPL_OK;
 }
 
 // The error record of the wave that is about to be launched.

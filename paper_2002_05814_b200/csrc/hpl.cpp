@@ -21,9 +21,7 @@ int progress(hpl_ctx* c);
 int progress(hpl_ctx* c) {
     // (a schedule-only context plans as well -- its planned tasks are counted, nothing is launched)
     {
-        int rc = order_main_after_control(c);
-        if (rc != HPL_OK) return rc;
-        rc = flush_directory(c);
+        int rc = flush_directory(c);
         if (rc != HPL_OK) return rc;
     }
     if (c->copy_pending && !c->cfg.plan_ahead) {
@@ -87,11 +85,12 @@ int sync_and_check(hpl_ctx* c) {
         c->journal.clear();
         return HPL_OK;
     }
-    if (c->copy_pending || c->ctl_pending) {
+    if (c->copy_pending || c->ctl_unconfirmed) {
         CUDA_TRY(cudaStreamSynchronize(c->ctl_stream));
         CUDA_TRY(cudaStreamSynchronize(c->copy_stream));
         c->copy_pending = false;
         c->ctl_pending = false;
+        c->ctl_unconfirmed = false;
         for (auto& kv : c->objects)
             if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
@@ -352,7 +351,7 @@ int hpl_put(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
         if (after != before || first) {
             rc = publish_counter(c, *o, after, c->ctl_stream);
             if (rc != HPL_OK) return rc;
-            c->ctl_pending = true;
+            c->ctl_unconfirmed = true;
         }
     } else {
         if (after != before || first) {
@@ -384,11 +383,10 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
             o->lib_owned = false;
             return rc;
         }
-        // the row (pointer) must be in the directory before any copy-stream counter update can matter
-        cudaStream_t row_stream = c->cfg.plan_ahead ? c->ctl_stream : c->stream;
+        // the row must be in the directory (with a zero counter) before any copy-stream counter update
         rc = flush_directory(c);
         if (rc != HPL_OK) return rc;
-        CUDA_TRY(cudaEventRecord(c->copy_ev, row_stream));
+        CUDA_TRY(cudaEventRecord(c->copy_ev, c->ctl_stream));
         CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
     }
     const uint64_t old_bytes = o->ready_bytes;
@@ -723,6 +721,49 @@ int hpl_get_batch(hpl_ctx* c, int32_t n, const int64_t* ids, const void** dev_pt
     return rc;
 }
 
+int hpl_submit(hpl_ctx* c, hpl_event* ev, int32_t n, int32_t* n_done) {
+    if (!c || n < 0 || (n && !ev)) return HPL_ERR_INVALID;
+    int rc = HPL_OK, done = 0;
+    for (int i = 0; i < n; ++i) {
+        hpl_event& e = ev[i];
+        if (e.t_ns != 0 && e.t_ns != c->now) {
+            rc = hpl_advance(c, e.t_ns);
+            if (rc != HPL_OK) break;
+        }
+        switch (e.kind) {
+            case HPL_EV_CREATE: rc = hpl_create(c, e.object_id, e.worker, e.bytes, e.dtype); break;
+            case HPL_EV_PUT: rc = hpl_put(c, e.object_id, e.ptr, e.bytes); break;
+            case HPL_EV_PUT_HOST: rc = hpl_put_host(c, e.object_id, e.ptr, e.bytes); break;
+            case HPL_EV_REDUCE: rc = hpl_reduce(c, e.object_id, e.ids, e.n_ids, e.k, e.op, e.dtype); break;
+            case HPL_EV_BROADCAST: rc = hpl_broadcast(c, e.object_id, e.ids, e.n_ids); break;
+            case HPL_EV_JOIN: rc = hpl_join(c, e.object_id, e.ptr); break;
+            case HPL_EV_FAIL: rc = hpl_fail(c, e.worker); break;
+            case HPL_EV_REJOIN: rc = hpl_rejoin(c, e.worker); break;
+            case HPL_EV_PROGRESS: rc = hpl_progress(c); break;
+            case HPL_EV_GET: {
+                const void* p = nullptr;
+                uint64_t nb = 0;
+                rc = hpl_get(c, e.object_id, &p, &nb);
+                if (rc == HPL_OK) {
+                    e.ptr = const_cast<void*>(p);
+                    e.bytes = nb;
+                }
+                break;
+            }
+            case HPL_EV_DELETE: rc = hpl_delete(c, e.object_id); break;
+            case HPL_EV_SYNC: rc = hpl_sync(c); break;
+            case HPL_EV_MARK:
+                if (c->device && (!e.ptr || cudaEventRecord((cudaEvent_t)e.ptr, c->stream) != cudaSuccess)) rc = HPL_ERR_CUDA;
+                break;
+            default: rc = HPL_ERR_INVALID;
+        }
+        if (rc != HPL_OK) break;
+        ++done;
+    }
+    if (n_done) *n_done = done;
+    return rc;
+}
+
 int hpl_get_host(hpl_ctx* c, int64_t id, void* dst, uint64_t cap) {
     if (!c || !dst) return HPL_ERR_INVALID;
     const void* p = nullptr;
@@ -743,7 +784,7 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
     if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
     for (auto& kv : c->reduces)
         if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
-    if (c->device && (c->work_in_flight || c->copy_pending || c->ctl_pending)) {
+    if (c->device && (c->work_in_flight || c->copy_pending || c->ctl_unconfirmed)) {
         // rows and arena memory are recycled only when nothing enqueued can still read them (nothing of the
         // library's is in flight after a Get or a wait, so a round's Deletes cost no device wait)
         cudaStreamSynchronize(c->ctl_stream);

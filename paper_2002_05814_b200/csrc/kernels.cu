@@ -79,13 +79,9 @@ struct StagesFor {
     static constexpr int smem_bytes = value * kStageBytes;
 };
 
-// A step as the kernel keeps it in shared memory: operand base address in the low 56 bits, and on top
-// code (2 bits), accumulator (3 bits), operand kind (1 bit).
-constexpr int kRecShift = 56;
-__device__ __forceinline__ unsigned long long make_rec(const ReduceStep st, unsigned long long ptr) {
-    const unsigned long long meta = (unsigned long long)st.code | ((unsigned long long)st.a << 2) | ((unsigned long long)st.kind << 5);
-    return (ptr & ((1ull << kRecShift) - 1)) | (meta << kRecShift);
-}
+// A step as the kernel keeps it in shared memory: the packed record of the wave (operand address in the low
+// 56 bits; code, accumulator and operand kind on top).  A load step whose address is 0 is resolved through the
+// device directory (the row beside it) when the task's records are set up.
 __device__ __forceinline__ unsigned int rec_meta(unsigned long long rec) { return (unsigned int)(rec >> kRecShift); }
 __device__ __forceinline__ unsigned int meta_code(unsigned int m) { return m & 3u; }
 __device__ __forceinline__ unsigned int meta_acc(unsigned int m) { return (m >> 2) & 7u; }
@@ -325,8 +321,10 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
         if (ti != cached_task) {
             __syncthreads();  // everyone is done with the previous task's records
             for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
-                const ReduceStep st = w.steps[task.step_begin + i];
-                s_rec[i] = make_rec(st, st.code == OPC_ADD_ACC ? 0ull : w.dir[st.row].ptr);
+                unsigned long long rec = w.recs[task.step_begin + i];
+                if (meta_code(rec_meta(rec)) != OPC_ADD_ACC && (rec & ((1ull << kRecShift) - 1)) == 0ull)
+                    rec |= w.dir[w.rows[task.step_begin + i]].ptr & ((1ull << kRecShift) - 1);
+                s_rec[i] = rec;
             }
             cached_task = ti;
             __syncthreads();
@@ -344,8 +342,8 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
         if (task.poll) {
             int ok = 1;
             for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
-                const ReduceStep st = w.steps[task.step_begin + i];
-                if (st.code != OPC_ADD_ACC) ok &= wait_chunk(w.dir, w.status, st.row, c, t_start, w.budget_ns) ? 1 : 0;
+                if (meta_code(rec_meta(w.recs[task.step_begin + i])) != OPC_ADD_ACC)
+                    ok &= wait_chunk(w.dir, w.status, w.rows[task.step_begin + i], c, t_start, w.budget_ns) ? 1 : 0;
             }
             if (!__syncthreads_and(ok)) return;
         }
@@ -383,8 +381,8 @@ __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __gri
         const FanoutTask& task = w.tasks[ti];
         if (ti != cached_task) {
             __syncthreads();
-            for (unsigned int i = t; i < task.n_dst; i += kFanoutThreads) s_dst[i] = w.dir[w.dst_rows[task.dst_begin + i]].ptr;
-            if (t == 0) s_src = w.dir[task.src_row].ptr;
+            for (unsigned int i = t; i < task.n_dst; i += kFanoutThreads) s_dst[i] = w.dst_ptrs[task.dst_begin + i];
+            if (t == 0) s_src = task.src_ptr;
             cached_task = ti;
             __syncthreads();
         }

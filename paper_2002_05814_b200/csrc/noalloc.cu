@@ -173,7 +173,10 @@ extern "C" int hpl_reduce_noalloc(const void* const* src_bufs, int32_t n, int32_
     t.red_op = (uint32_t)op;
     t.poll = 0;
     t.pad = 0;
-    for (size_t i = 0; i < steps.size(); ++i) w.steps[i] = steps[i];
+    for (size_t i = 0; i < steps.size(); ++i) {
+        w.recs[i] = pack_step(steps[i]);   // address 0: the kernel takes it from the row in the scratch array
+        w.rows[i] = steps[i].row;
+    }
     w.total_tiles = C * tpc;
     const bool bf16 = dtype == HPL_BF16;
     int occ = reduce_ctas_per_sm(n_acc, bf16);

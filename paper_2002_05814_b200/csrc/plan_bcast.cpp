@@ -114,6 +114,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
             FanoutTask& d = w.tasks[w.n_tasks++];
             Object* lo = tt.loc == 0 ? src : find(c, locs[tt.loc].obj);
             d.src_row = (uint32_t)lo->row;
+            d.src_ptr = (unsigned long long)(uintptr_t)lo->ptr;
             d.c_begin = tt.a;
             d.c_end = tt.b;
             d.tiles_per_chunk = tpc;
@@ -124,7 +125,7 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
             if (tt.poll) c->polling_in_flight = true;
             d.bytes = src->bytes;
             d.chunk_bytes = chunk_bytes;
-            for (int r : tt.dst) w.dst_rows[n_dst++] = (uint32_t)find(c, locs[r].obj)->row;
+            for (int r : tt.dst) w.dst_ptrs[n_dst++] = (unsigned long long)(uintptr_t)find(c, locs[r].obj)->ptr;
             w.total_tiles += (tt.b - tt.a) * tpc;
             const uint64_t b_lo = (uint64_t)tt.a * chunk_bytes, b_hi = std::min<uint64_t>((uint64_t)tt.b * chunk_bytes, src->bytes);
             c->stats.bytes_read_planned += b_hi - b_lo;
@@ -143,6 +144,9 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
         if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
+        bool polls = false;
+        for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
+        if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counter it waits on is a row of the directory
         w.status = next_wave_status(c);
         {
             LaunchTimer timer(c, 1);

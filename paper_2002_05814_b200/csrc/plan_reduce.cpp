@@ -58,10 +58,14 @@ void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial
     st.a = (uint8_t)acc;
     if (partial) {
         st.kind = SRC_F32;
-        st.row = (uint32_t)find(p.c, q == 0 ? op.target : op.partial_key[q])->row;
+        const Object* o = find(p.c, q == 0 ? op.target : op.partial_key[q]);
+        st.row = (uint32_t)o->row;
+        st.ptr = (unsigned long long)(uintptr_t)o->ptr;
     } else {
         st.kind = op.in_dtype == HPL_BF16 ? SRC_BF16 : SRC_F32;
-        st.row = (uint32_t)find(p.c, op.sched->object_at(q))->row;
+        const Object* o = find(p.c, op.sched->object_at(q));
+        st.row = (uint32_t)o->row;
+        st.ptr = (unsigned long long)(uintptr_t)o->ptr;
         if (p.landed[q] < p.b) task.poll = true;  // not yet known to be visible: the kernel polls its counter
     }
     task.steps.push_back(st);
@@ -310,7 +314,10 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 d.poll = t.poll ? 1u : 0u;
                 if (t.poll) c->polling_in_flight = true;
                 d.pad = 0;
-                std::memcpy(&w.steps[n_steps], t.steps.data(), t.steps.size() * sizeof(ReduceStep));
+                for (size_t q = 0; q < t.steps.size(); ++q) {
+                    w.recs[n_steps + q] = pack_step(t.steps[q]);
+                    w.rows[n_steps + q] = t.steps[q].row;
+                }
                 n_steps += d.n_steps;
                 w.total_tiles += (t.b - t.a) * tpc_full;
                 n_acc = std::max(n_acc, t.n_acc);
@@ -334,6 +341,9 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
             if (grid < 1) grid = 1;
             if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
+            bool polls = false;
+            for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
+            if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counters it waits on are rows of the directory
             w.status = next_wave_status(c);
             {
                 LaunchTimer timer(c, 0);

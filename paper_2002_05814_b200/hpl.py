@@ -14,6 +14,8 @@ HPL_ERR_INVALID, HPL_ERR_NOT_FOUND, HPL_ERR_EXISTS, HPL_ERR_TIMEOUT = -1, -2, -3
 HPL_ERR_INSUFFICIENT, HPL_ERR_FAILED_WORKER, HPL_ERR_CUDA, HPL_ERR_NOMEM = -5, -6, -7, -8
 HPL_F32, HPL_BF16 = 0, 1
 HPL_SUM, HPL_MIN, HPL_MAX = 0, 1, 2
+(HPL_EV_CREATE, HPL_EV_PUT, HPL_EV_PUT_HOST, HPL_EV_REDUCE, HPL_EV_BROADCAST, HPL_EV_JOIN, HPL_EV_FAIL, HPL_EV_REJOIN,
+ HPL_EV_PROGRESS, HPL_EV_GET, HPL_EV_DELETE, HPL_EV_SYNC, HPL_EV_MARK) = range(1, 14)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
@@ -39,6 +41,38 @@ class Stats(C.Structure):
                                           "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
                                           "reduce_launches", "fanout_launches", "reduce_kernel_ns",
                                           "fanout_kernel_ns", "device_waits")]
+
+
+class Event(C.Structure):
+    """Mirror of ``hpl_event``."""
+    _fields_ = [("t_ns", C.c_uint64), ("kind", C.c_int32), ("worker", C.c_int32), ("object_id", C.c_int64),
+                ("ptr", C.c_void_p), ("bytes", C.c_uint64), ("ids", C.POINTER(C.c_int64)), ("n_ids", C.c_int32),
+                ("k", C.c_int32), ("op", C.c_int32), ("dtype", C.c_int32)]
+
+
+class EventList:
+    """A timeline prepared once for ``Context.submit``: a ctypes array of ``hpl_event`` plus the id arrays its
+    Reduce / broadcast requests point to (kept alive here).  ``add`` takes the fields by name."""
+
+    def __init__(self, capacity: int):
+        self.array = (Event * capacity)()
+        self.n = 0
+        self._keep = []
+
+    def add(self, kind: int, t_ns: int = 0, object_id: int = 0, worker: int = 0, ptr: int = 0, nbytes: int = 0, ids=None,
+            k: int = 0, op: int = HPL_SUM, dtype: int = HPL_F32):
+        e = self.array[self.n]
+        self.n += 1
+        e.t_ns, e.kind, e.worker, e.object_id, e.ptr, e.bytes = t_ns, kind, worker, object_id, ptr or None, nbytes
+        e.k, e.op, e.dtype = k, op, dtype
+        if ids is not None:
+            arr = (C.c_int64 * len(ids))(*ids)
+            self._keep.append(arr)
+            e.ids, e.n_ids = arr, len(ids)
+        return self
+
+    def __len__(self):
+        return self.n
 
 
 class HplError(RuntimeError):
@@ -75,6 +109,7 @@ def load_library():
         "hpl_put_batch": [VP, I32, P(I64), P(VP), P(U64), P(I32)],
         "hpl_join_batch": [VP, I32, P(I64), P(VP), P(I32)],
         "hpl_get_batch": [VP, I32, P(I64), P(VP), P(I32)],
+        "hpl_submit": [VP, P(Event), I32, P(I32)],
         "hpl_reduce": [VP, I64, P(I64), I32, I32, I32, I32],
         "hpl_broadcast": [VP, I64, P(I64), I32],
         "hpl_join": [VP, I64, VP],
@@ -192,6 +227,13 @@ class Context:
         out = out_ptrs if out_ptrs is not None else (C.c_void_p * len(ids))()
         self._check(self._lib.hpl_get_batch(self._h, len(ids), ids, out, None), "hpl_get_batch")
         return out if out_ptrs is not None else list(out)
+
+    def submit(self, events: EventList):
+        """``hpl_submit``: the whole prepared timeline in one call.  Results of Get events are in ``events.array``."""
+        done = C.c_int32()
+        rc = self._lib.hpl_submit(self._h, events.array, events.n, C.byref(done))
+        if rc:
+            raise HplError(rc, f"hpl_submit (event {done.value} of {events.n})")
 
     def put_host(self, object_id: int, host_buf, nbytes: int):
         self._check(self._lib.hpl_put_host(self._h, object_id, C.c_void_p(_addr(host_buf)), nbytes), "hpl_put_host")
