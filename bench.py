@@ -35,11 +35,33 @@ import workloads as wl  # noqa: E402
 MiB = 1 << 20
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per full-size launch, from the ncu captures summarised in
-# profiles/ (taken on objects shrunk 4x and scaled by the elements processed; traffic is proportional).
-# Valid only for the kernels as captured: set an entry to None when its kernel changes.
-NCU_TRAFFIC = {"cfg4": {"reduce": 4.4227e9, "fanout": 4.1236e9},     # shrunk 4x, scaled
-               "cfg2": {"fanout": 1.0780e9}, "cfg3": {"reduce": 0.9077e9}}          # captured at full size
+KERNEL_SOURCES = ("paper_2002_05814_b200/csrc/kernels.cu", "paper_2002_05814_b200/csrc/device_types.h")
+
+
+def kernel_source_hash() -> str:
+    """Hash of the kernel sources as they stand: an ncu figure is only quoted for the kernels it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per full-size launch, from the record line of the ncu summary
+    under profiles/ (`bench-record: workload=... kernel=... traffic_bytes=... kernel_sources=<hash>`).  None when
+    there is no record or the kernels have changed since the counters were taken."""
+    import glob
+    import re
+    cur = kernel_source_hash()
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        with open(path) as f:
+            for ln in f:
+                m = re.search(r"bench-record: workload=(\S+) kernel=(\S+) traffic_bytes=(\S+) kernel_sources=(\S+)", ln)
+                if m and m.group(1) == workload and m.group(2) == kernel:
+                    return float(m.group(3)) if m.group(4) == cur else None
+    return None
 
 
 # ----------------------------------------------------------------------------------------- helpers
@@ -448,16 +470,17 @@ def gbs(nbytes, ms):
 
 
 # ----------------------------------------------------------------------------------------- oracle arm
-def oracle_sample(w: wl.Workload, budget_s: float = 12.0):
+def oracle_sample(w: wl.Workload, budget_s: float = 12.0, window: int = 0, raw: bool = False):
     """Times the oracle, as it stands, on a bounded sample of the workload: the same objects cut to a
     window of their elements (same chunk size, same tree, same timeline).  Returns GB/s on the
-    algorithmic bytes of the sample."""
+    algorithmic bytes of the sample.  ``window`` picks which 1/16 of the elements (0 = the first)."""
     from oracle.store import OracleStore, DT_F32, DT_BF16
 
     frac = 16
     elems = max(4096, (w.elems // frac) // 8 * 8)
     dt = DT_BF16 if w.dtype == "bf16" else DT_F32
-    distinct = [wl.values_np(w.dist, w.seed + i, i, 0, elems, w.dtype) for i in range(min(8, max(1, w.n_objects)))]
+    start = (window % frac) * elems if (window % frac + 1) * elems <= w.elems else 0
+    distinct = [wl.values_np(w.dist, w.seed + i, i, start, elems, w.dtype) for i in range(min(8, max(1, w.n_objects)))]
     S = distinct[0].nbytes
     sw = wl.Workload(**{**w.__dict__, "elems": elems})
     ab = algorithmic_bytes(sw)
@@ -499,10 +522,82 @@ def oracle_sample(w: wl.Workload, budget_s: float = 12.0):
             o.get(9000)
         t_total += time.perf_counter() - t0
         reps += 1
+    if raw:
+        return total_bytes * reps, t_total, elems
     value = total_bytes * reps / t_total / 1e9
     sample = (f"{reps} pass(es) of the oracle over the first {elems} of {w.elems} elements of every object "
               f"({total_bytes * reps / 1e9:.2f} GB algorithmic, {t_total:.1f} s, numpy single thread)")
     return value, sample, t_total / reps * 1e3
+
+
+def _oracle_worker(args):
+    w, budget_s, window = args
+    return oracle_sample(w, budget_s, window, raw=True)
+
+
+def oracle_all_cores(w: wl.Workload, budget_s: float = 8.0):
+    """The same oracle passes on every core the process may use: one process per core (started with `spawn`), each
+    over its own window of the elements.  Throughput = bytes of all processes / the slowest one's time."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0))
+    with mp.get_context("spawn").Pool(cores) as pool:
+        out = pool.map(_oracle_worker, [(w, budget_s, i) for i in range(cores)])
+    nbytes = sum(o[0] for o in out)
+    t = max(o[1] for o in out)
+    sample = (f"{cores} processes, each the oracle's passes over its own window of {out[0][2]} of {w.elems} elements of every "
+              f"object ({nbytes / 1e9:.2f} GB algorithmic in all, slowest process {t:.1f} s, numpy, one thread each)")
+    return nbytes / t / 1e9, cores, sample
+
+
+# ----------------------------------------------------------------------------------------- measured points
+def measure_point(rr: "Runner", steps: int, warmup: int, peak: float, k_steps: int = 0):
+    """Step throughput of the runner's workload (event timing off) and, from a pass of its own with event timing on,
+    the kernels' figures."""
+    ab = algorithmic_bytes(rr.w)
+    b = ab["reduce"] + ab["broadcast"]
+    rr.open_context(time_kernels=False)
+    r = time_steps(rr, steps, warmup)
+    g = gbs(b * steps, float(np.sum(r["total_ms"])))
+    k_steps = k_steps or min(steps, 10)
+    rr.open_context(time_kernels=True)
+    s2 = time_steps(rr, k_steps, 1)["stats"]
+    kns = s2["reduce_kernel_ns"] + s2["fanout_kernel_ns"]
+    planned = s2["bytes_read_planned"] + s2["bytes_written_planned"]
+    kern = gbs(planned, kns / 1e6)       # bytes the planned tasks move / their summed launch time
+    return {"GBps": g, "frac_of_measured_copy": g / peak, "ms_per_step": float(np.mean(r["total_ms"])),
+            "ms_std": float(np.std(r["total_ms"])), "steps": steps, "kernel_GBps": kern,
+            "kernel_frac_of_measured_copy": kern / peak, "kernel_ms_per_step": kns / 1e6 / k_steps,
+            "launches_per_step": s2["kernel_launches"] / k_steps, "planned_over_algorithmic_bytes": planned / (b * k_steps)}
+
+
+def size_sweep(device, peak: float):
+    """The metric's curve: effective GB/s and fraction of the HBM peak against object size, 1 KiB ... 1 GiB in powers
+    of 4, for the fault-tolerant reduce of 32 objects (the compressed timeline planned at the Get, and with the chunks
+    delivered before the failure reduced first) and for a broadcast to 16 receivers."""
+    import torch
+    rows = []
+    for size in wl.workload("cfg5").extra["sizes_bytes"]:
+        n = 20 if size <= (16 << 20) else (5 if size <= (256 << 20) else 3)
+        row = {"object_bytes": size}
+        rr = Runner(wl.cfg5_at(size), device)
+        for mode in ("lazy", "eager"):
+            rr.ft_eager = mode == "eager"
+            m = measure_point(rr, n, 3, peak, k_steps=min(n, 5))
+            row[f"reduce_{mode}"] = {k: m[k] for k in ("GBps", "frac_of_measured_copy", "ms_per_step", "kernel_ms_per_step",
+                                                         "planned_over_algorithmic_bytes", "launches_per_step")}
+        rr.close()
+        del rr
+        torch.cuda.empty_cache()
+        bw = wl.Workload("bcast16", "broadcast", "f32", ("uniform",), size // 4, min(1 << 20, size), 2, n_receivers=16,
+                         extra={"join_window_ns": 1_000_000})
+        rr = Runner(bw, device)
+        m = measure_point(rr, n, 3, peak, k_steps=min(n, 5))
+        row["broadcast16"] = {k: m[k] for k in ("GBps", "frac_of_measured_copy", "ms_per_step", "kernel_ms_per_step")}
+        rr.close()
+        del rr
+        torch.cuda.empty_cache()
+        rows.append(row)
+    return rows
 
 
 # ----------------------------------------------------------------------------------------- main
@@ -518,13 +613,13 @@ def main():
     ap.add_argument("--ft-mode", default="eager", choices=["eager", "lazy"],
                     help="cfg5: 'eager' runs hpl_progress before the failure (chunks delivered by every worker are reduced, "
                          "then partly redone); 'lazy' applies the compressed timeline and plans at the Get")
-    ap.add_argument("--realtime", action="store_true", help="also measure cfg3 with puts at their real arrival offsets")
-    ap.add_argument("--sweep", action="store_true",
-                    help="also measure GB/s against object size: the fault-tolerant reduce (32 objects, both modes) and a "
+    ap.add_argument("--no-realtime", action="store_true", help="skip the view with puts / joins at their real offsets (cfg3, cfg2)")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip GB/s against object size: the fault-tolerant reduce (32 objects, both modes) and a "
                          "broadcast to 16 receivers, for 1 KiB ... 1 GiB in powers of 4")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--also", default="cfg2,cfg3,cfg5", help="extra workloads measured briefly and reported under 'also' (cfg5 = the 1 GiB point of the fault-tolerant sweep, both modes)")
+    ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads reported under 'also' (cfg3 for its 50 rounds); 'none' skips them")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -600,7 +695,7 @@ def main():
                 "peak_kind": f"of {peak_kind} (copy bandwidth)", "avg_launch_ms": avg_ms, "launches": st[kind_launches],
                 "algorithmic_bytes_per_launch": per_launch_bytes, "frac_of_8TBs_nominal": ach / 8000.0}
 
-    traf = NCU_TRAFFIC.get(w.name, {}) if args.shrink == 1 else {}
+    traf = {k: ncu_traffic(w.name, k) for k in ("reduce", "fanout")} if args.shrink == 1 else {}
     r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * k_steps / max(1, st["reduce_launches"]), traf.get("reduce")) if ab["reduce"] else None
     r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * k_steps / max(1, st["fanout_launches"]), traf.get("fanout")) if ab["broadcast"] else None
     line = {"metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value, "unit": "GB/s",
@@ -628,74 +723,28 @@ def main():
 
     if rank == 0 and world == 1 and args.also:
         also = {}
-        names = []
         for nm in [x for x in args.also.split(",") if x and x != "none" and x != w.name]:
-            names += [("cfg5_1GiB_lazy", wl.cfg5_at(1 << 30), False), ("cfg5_1GiB_eager", wl.cfg5_at(1 << 30), True)] if nm == "cfg5" \
-                else [(nm, wl.workload(nm), True)]
-        rr = None
-        for label, ww, eager in names:
-            if rr is None or rr.w.name != ww.name or ww.name != "cfg5":
-                if rr is not None:
-                    rr.close()
-                    del rr
-                    torch.cuda.empty_cache()
-                rr = Runner(ww, device, ft_eager=eager)
-            rr.ft_eager = eager                  # the two cfg5 modes share the 32 GiB of inputs
-            n2 = 3 if ww.name == "cfg5" else 10
-            rr.open_context(time_kernels=False)
-            r2 = time_steps(rr, n2, 3)
-            a2 = algorithmic_bytes(ww)
-            b2 = a2["reduce"] + a2["broadcast"]
-            g = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
-            rr.open_context(time_kernels=True)
-            s2 = time_steps(rr, n2, 1)["stats"]
-            kns = s2["reduce_kernel_ns"] + s2["fanout_kernel_ns"]
-            planned = s2["bytes_read_planned"] + s2["bytes_written_planned"]
-            kern = gbs(planned, kns / 1e6)       # bytes the planned tasks move / their summed launch time
-            also[label] = {"GBps": g, "frac_of_measured_copy": g / peak, "ms_per_step": float(np.mean(r2["total_ms"])),
-                           "ms_std": float(np.std(r2["total_ms"])), "steps": n2, "kernel_GBps": kern,
-                           "kernel_frac_of_measured_copy": kern / peak, "launches_per_step": s2["kernel_launches"] / n2,
-                           "planned_over_algorithmic_bytes": planned / (b2 * n2)}
-        if rr is not None:
+            ww = wl.workload(nm)
+            rr = Runner(ww, device)
+            also[nm] = measure_point(rr, ww.rounds if ww.rounds > 1 else 30, 5, peak)
             rr.close()
             del rr
             torch.cuda.empty_cache()
         line["also"] = also
 
-    if rank == 0 and world == 1 and args.realtime:
-        line["realtime_cfg3"] = realtime_rounds(device)
-
-    if rank == 0 and world == 1 and args.sweep:
-        rows = []
-        for size in wl.workload("cfg5").extra["sizes_bytes"]:
-            row = {"object_bytes": size}
-            n2 = 20 if size <= (16 << 20) else (5 if size <= (256 << 20) else 3)
-            ww = wl.cfg5_at(size)
-            rr = Runner(ww, device)
-            for mode in ("lazy", "eager"):
-                rr.ft_eager = mode == "eager"
-                r2 = time_steps(rr, n2, 3)
-                b2 = algorithmic_bytes(ww)["reduce"]
-                row[f"reduce_{mode}_GBps"] = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
-                row[f"reduce_{mode}_ms"] = float(np.mean(r2["total_ms"]))
-                s2 = r2["stats"]
-                row[f"reduce_{mode}_kernel_ms"] = s2["reduce_kernel_ns"] / 1e6 / n2
-            rr.close()
-            del rr
-            torch.cuda.empty_cache()
-            bw = wl.Workload("bcast", "broadcast", "f32", ("uniform",), size // 4, min(1 << 20, size), 2, n_receivers=16,
-                             extra={"join_window_ns": 1_000_000})
-            rr = Runner(bw, device)
-            r2 = time_steps(rr, n2, 3)
-            b2 = algorithmic_bytes(bw)["broadcast"]
-            row["broadcast16_GBps"] = gbs(b2 * n2, float(np.sum(r2["total_ms"])))
-            row["broadcast16_ms"] = float(np.mean(r2["total_ms"]))
-            row["broadcast16_kernel_ms"] = r2["stats"]["fanout_kernel_ns"] / 1e6 / n2
-            rr.close()
-            del rr
-            torch.cuda.empty_cache()
-            rows.append(row)
+    if rank == 0 and world == 1 and not args.no_sweep and args.shrink == 1:
+        rows = size_sweep(device, peak)
         line["sweep"] = rows
+        big = [r for r in rows if r["object_bytes"] >= (64 << 20)]
+        line["sweep_summary"] = {
+            "min_frac_reduce_at_64MiB_and_above": min(r["reduce_lazy"]["frac_of_measured_copy"] for r in big),
+            "min_frac_broadcast_at_64MiB_and_above": min(r["broadcast16"]["frac_of_measured_copy"] for r in big),
+            "max_ms_per_step_up_to_4MiB": max(max(r["reduce_lazy"]["ms_per_step"], r["broadcast16"]["ms_per_step"])
+                                              for r in rows if r["object_bytes"] <= (4 << 20)),
+            "of": "measured copy bandwidth; reduce = fault-tolerant reduce of 32 objects planned at the Get"}
+
+    if rank == 0 and world == 1 and not args.no_realtime and args.shrink == 1:
+        line["realtime"] = realtime_rounds(device)
 
     if not args.no_e2e:
         e_steps = max(1, min(args.steps, 3))
@@ -711,7 +760,9 @@ def main():
 
     if rank == 0 and world == 1 and not args.no_cpu:
         v, sample, _ = oracle_sample(w)
-        line["cpu_baseline"] = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample}
+        va, cores, sample_all = oracle_all_cores(w)
+        line["cpu_baseline"] = {"value": va, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample_all}
+        line["cpu_baseline_one_core"] = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample}
 
     if rank == 0:
         print(json.dumps(line))
