@@ -137,6 +137,11 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
         out["reduce"] = (w.k - 1) * S + w.elems * 4          # the survivors and the result
     if w.kind in ("broadcast", "round"):
         out["broadcast"] = S + w.n_receivers * S
+    if w.kind == "allreduce":
+        # reduce followed by broadcast of its output: the sources read once, the result written once to the target
+        # and once to every receiver (reading the target back is not part of what the method must move)
+        out["reduce"] = w.k * S + w.elems * 4
+        out["broadcast"] = w.n_receivers * w.elems * 4
     return out
 
 
@@ -144,7 +149,8 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
 class Runner:
     """Holds the device buffers of one workload and runs steps through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device, host_buffers: bool = False, plan_ahead: bool = False, ft_eager: bool = True):
+    def __init__(self, w: wl.Workload, device, host_buffers: bool = False, plan_ahead: bool = False, ft_eager: bool = True,
+                 fuse_fanout: bool = True):
         import torch
         import paper_2002_05814_b200 as hpl
 
@@ -159,14 +165,17 @@ class Runner:
             arena_bytes += 8 * w.elems * 4       # partial results of the subtrees beside the failing worker's root path
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
         self.plan_ahead = plan_ahead
+        self.fuse_fanout = fuse_fanout
         self.ctx = None
         self.open_context(time_kernels=False)
         self.src = [wl.values_torch(w.dist, w.seed + i, i, 0, w.elems, w.dtype, device=device) for i in range(n_src)]
         self.policy = None
         self.recv = []
         if w.n_receivers:
-            self.policy = wl.values_torch(w.dist, w.seed + 1000, 1000, 0, w.elems, w.dtype, device=device)
-            self.recv = [torch.empty(S, dtype=torch.uint8, device=device) for _ in range(w.n_receivers)]
+            if w.kind != "allreduce":
+                self.policy = wl.values_torch(w.dist, w.seed + 1000, 1000, 0, w.elems, w.dtype, device=device)
+            self.recv = [torch.empty(w.elems * 4 if w.kind == "allreduce" else S, dtype=torch.uint8, device=device)
+                         for _ in range(w.n_receivers)]
         self.host_src, self.host_policy, self.host_out, self.host_recv = [], None, None, None
         if host_buffers:
             n_distinct = min(n_src, 8)      # pinned host images; objects beyond the 8th reuse them (same bytes to copy)
@@ -188,7 +197,7 @@ class Runner:
             self.ctx.shutdown()
         self.ctx = self.hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=self.arena.numel(),
                                     stream=torch.cuda.current_stream().cuda_stream, time_kernels=time_kernels,
-                                    plan_ahead=self.plan_ahead)
+                                    plan_ahead=self.plan_ahead, fuse_fanout=self.fuse_fanout)
         self.prepared = {}
 
     def close(self):
@@ -204,7 +213,7 @@ class Runner:
         S = w.object_bytes
         t = (r + 1) * 2_000_000_000
         n, R = w.n_objects, w.n_receivers
-        e1, e2, dl = H.EventList(12 + 3 * R + n), H.EventList(12 + 3 * n), H.EventList(4 + n)
+        e1, e2, dl = H.EventList(12 + 3 * R + n), H.EventList(12 + 3 * n + 3 * R), H.EventList(4 + n)
         h2d = d2h = 0
         put_kind = H.HPL_EV_PUT_HOST if self.host_buffers else H.HPL_EV_PUT
         ids = list(range(n))
@@ -273,6 +282,24 @@ class Runner:
                 e2.add(H.HPL_EV_FAIL, t + 1, worker=w.extra["fail_worker"])
             if not self.host_buffers:
                 e2.add(H.HPL_EV_GET, 0, tgt)
+            for i in [tgt] + ids:
+                dl.add(H.HPL_EV_DELETE, 0, i)
+        if w.kind == "allreduce":
+            # the allreduce of Section 3.4.3: a Reduce whose output is broadcast to the R participants.  Puts first,
+            # then the requests (equal-time order), then every receiver's Get.
+            dsts = [6000 + j for j in range(R)]
+            for i in ids:
+                e2.add(H.HPL_EV_CREATE, t, i, i, nbytes=S, dtype=self.dt)
+                e2.add(H.HPL_EV_PUT, t, i, ptr=self.src[i].data_ptr(), nbytes=S)
+            for j in range(R):
+                e2.add(H.HPL_EV_CREATE, t, dsts[j], 1000 + j, nbytes=w.elems * 4, dtype=H.HPL_F32)
+            e2.add(H.HPL_EV_REDUCE, t, tgt, ids=ids, k=w.k, op=H.HPL_SUM, dtype=self.dt)
+            e2.add(H.HPL_EV_BROADCAST, t, tgt, ids=dsts)
+            for j in range(R):
+                e2.add(H.HPL_EV_JOIN, t, dsts[j], ptr=self.recv[j].data_ptr())
+            for j in range(R):
+                e2.add(H.HPL_EV_GET, 0, dsts[j])
+            e2.add(H.HPL_EV_GET, 0, tgt)
             for i in [tgt] + ids:
                 dl.add(H.HPL_EV_DELETE, 0, i)
         if marks:
@@ -727,6 +754,15 @@ def main():
             ww = wl.workload(nm)
             rr = Runner(ww, device)
             also[nm] = measure_point(rr, ww.rounds if ww.rounds > 1 else 30, 5, peak)
+            rr.close()
+            del rr
+            torch.cuda.empty_cache()
+        # reduce followed by broadcast (the allreduce microbenchmark of Section 5.1): 8 x 64 MiB fp32 to 8 receivers, with
+        # the result tile fanned out from the reduce pass and, for comparison, with the broadcast reading the target
+        aw = wl.Workload("allreduce", "allreduce", "f32", ("uniform",), 16 * MiB, 4 * MiB, 2, n_objects=8, k=8, n_receivers=8)
+        for label, fused in (("allreduce_8x64MiB_fused", True), ("allreduce_8x64MiB_two_waves", False)):
+            rr = Runner(aw, device, fuse_fanout=fused)
+            also[label] = measure_point(rr, 20, 5, peak)
             rr.close()
             del rr
             torch.cuda.empty_cache()

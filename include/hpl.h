@@ -77,6 +77,11 @@ typedef struct hpl_config {
     uint64_t arena_bytes;
     uint64_t model_latency_ns;     /* L of Eq. 1: latency of one hop; used only when reduce_degree == 0 */
     uint64_t model_bandwidth_bps;  /* B of Eq. 1: bytes per second into one node; used only when reduce_degree == 0 */
+    int32_t  fuse_fanout;     /* 1: when the output of a Reduce is being broadcast (reduce followed by broadcast, the
+                                 allreduce of Section 3.4.3), receivers that have joined take each result tile straight
+                                 from the reduce pass -- the output is written once to the target and once to each of
+                                 them and is not read again; 0: the broadcast always reads the target */
+    int32_t  reserved;
 } hpl_config;
 
 /* Creates a context.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Nothing is
@@ -261,6 +266,7 @@ typedef struct hpl_stats_t {
     uint64_t reduce_kernel_ns;     /* summed device time of reduce launches (time_kernels = 1; updated by waits) */
     uint64_t fanout_kernel_ns;
     uint64_t device_waits;         /* polls of a progress counter that did not succeed at the first look (updated by waits) */
+    uint64_t fused_fanout_tasks;   /* reduce tasks that also wrote their result to broadcast receivers */
 } hpl_stats_t;
 
 int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);

@@ -246,7 +246,7 @@ struct hpl_ctx {
     uint64_t batch_tag = 0;        // launch_seq when the current planning pass began
     std::vector<uint64_t> wave_tag;  // for the waves in flight (seq - first_unchecked): the tag of their planning pass
     hpl_stats_t stats{};
-    int occ_reduce[2][3] = {{0, 0, 0}, {0, 0, 0}};
+    int occ_reduce[2][2][3] = {};   // [bf16][fan][accumulator class]
     int occ_fanout = 0;
     struct Timed { cudaEvent_t a, b; int kind; };
     std::vector<Timed> timed;            // event pairs of launches not yet read back

@@ -67,11 +67,14 @@ struct ReduceTask {
     uint32_t step_begin, n_steps;
     uint32_t red_op;
     uint32_t poll;                // 1: operands' progress counters must be polled before each chunk
+    uint32_t fan_begin, n_fan;    // receivers of a broadcast of this result that take each tile straight from the
+                                  // reduce (indices into ReduceWave::fan_ptrs); 0 = the result goes to out_ptr only
     uint32_t pad;
 };
 
 constexpr int kMaxTasksPerWave = 24;
 constexpr int kMaxStepsPerWave = 640;
+constexpr int kMaxFusedDst = 128;       // receivers served by the reduce tasks of one wave
 
 struct ReduceWave {
     const DirRow* dir;
@@ -82,6 +85,7 @@ struct ReduceWave {
     ReduceTask tasks[kMaxTasksPerWave];
     unsigned long long recs[kMaxStepsPerWave];   // packed steps (pack_step)
     uint32_t rows[kMaxStepsPerWave];             // directory row of each load step's operand
+    unsigned long long fan_ptrs[kMaxFusedDst];   // device addresses of receivers' buffers (fused reduce -> fan-out)
 };
 
 struct FanoutTask {
@@ -110,9 +114,9 @@ struct FanoutWave {
 };
 
 // Launchers (kernels.cu).  Return a cudaError_t as int.
-int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, int grid, void* stream);
+int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, bool fan, int grid, void* stream);
 int launch_fanout_wave(const FanoutWave& w, int grid, void* stream);
-int reduce_ctas_per_sm(int n_acc, bool bf16);
+int reduce_ctas_per_sm(int n_acc, bool bf16, bool fan);
 int fanout_ctas_per_sm();
 
 }  // namespace hpl

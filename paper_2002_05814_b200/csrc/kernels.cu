@@ -15,6 +15,10 @@
 // of the adds, so that 80 KiB and more per SM are in flight without holding registers.
 #include <cuda_runtime.h>
 
+#include <array>
+#include <mutex>
+#include <vector>
+
 #include "device_types.h"
 
 namespace hpl {
@@ -72,11 +76,13 @@ __device__ __forceinline__ float combine(float a, float b, unsigned int red_op) 
 // CTA and gets 12 stages instead.
 constexpr int kStageBytes = 4 * kReduceThreads * 16;
 constexpr int kVecStride = kReduceThreads * 16;   // bytes between a thread's consecutive vectors, in shared and (mostly) global
-template <int A>
+// A variant that also fans its result out (FAN) keeps one more 16 KiB buffer for the result tile, from which the
+// bulk copies read, and gives up one stage for it where two CTAs share an SM.
+template <int A, bool FAN = false>
 struct StagesFor {
-    static constexpr int value = A <= 4 ? 6 : 12;
+    static constexpr int value = A <= 4 ? (FAN ? 5 : 6) : 12;
     static constexpr int min_ctas = A <= 4 ? 2 : 1;
-    static constexpr int smem_bytes = value * kStageBytes;
+    static constexpr int smem_bytes = value * kStageBytes + (FAN ? kStageBytes : 0);
 };
 
 // A step as the kernel keeps it in shared memory: the packed record of the wave (operand address in the low
@@ -228,8 +234,8 @@ struct TileCtx {
 // Runs the steps that belong to accumulator L, starting at a LOAD into L, until a step that belongs to
 // a shallower accumulator.  A step into L+1 opens a fused child subtree: one more level of this
 // function, whose accumulator is a separate set of registers, closed by ADD_ACC(L, L+1).
-template <int L, int A, bool BF16>
-__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& cx, Acc& acc) {
+template <int L, int A, bool BF16, bool FAN>
+__device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A, FAN>::value>& cx, Acc& acc) {
     while (cx.pc < cx.n) {
         const unsigned int m = rec_meta(ld_shared_u64(cx.rec_base + cx.pc * 8));
         const unsigned int a = meta_acc(m);
@@ -246,7 +252,7 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& c
         } else {
             if constexpr (L + 1 < A) {
                 Acc sub;
-                eval_level<L + 1, A, BF16>(cx, sub);
+                eval_level<L + 1, A, BF16, FAN>(cx, sub);
                 cx.skip();  // the ADD_ACC(L, L+1) that closes the subtree
                 combine_acc(acc, sub, cx.red_op);
             } else {
@@ -256,10 +262,16 @@ __device__ __forceinline__ void eval_level(TileCtx<BF16, StagesFor<A>::value>& c
     }
 }
 
-template <int A, bool BF16>
+constexpr int kFanIssuers = 64;   // threads that issue the bulk copies of a fused fan-out
+
+__device__ __forceinline__ void bulk_store(unsigned long long gdst, unsigned int smem_src, unsigned int bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
+}
+
+template <int A, bool BF16, bool FAN>
 __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int stage_base, const ReduceTask& task, unsigned long long e0,
-                                         unsigned int count, unsigned int t) {
-    constexpr int kStages = StagesFor<A>::value;
+                                         unsigned int count, unsigned int t, const unsigned long long* fan_ptrs) {
+    constexpr int kStages = StagesFor<A, FAN>::value;
     TileCtx<BF16, kStages> cx;
     cx.rec_base = rec_base;
     cx.n = task.n_steps;
@@ -285,10 +297,48 @@ __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int sta
     for (int i = 0; i < kStages - 1; ++i) cx.issue();
 
     Acc acc;
-    eval_level<0, A, BF16>(cx, acc);
+    eval_level<0, A, BF16, FAN>(cx, acc);
     cp_async_wait<0>();
 
     float* out = reinterpret_cast<float*>(task.out_ptr) + e0;
+    if constexpr (FAN) {
+        if (task.n_fan != 0) {
+            // Fused fan-out (reduce followed by broadcast, Section 3.4.3): the result tile goes registers -> shared
+            // memory -> one bulk copy to the target and one to every receiver.  The tile's whole 16-byte vectors
+            // travel by bulk copy, the last elements of an object whose length is not a multiple of 4 by plain stores.
+            const unsigned int s_out = stage_base + kStages * kStageBytes;
+            if (t < kFanIssuers) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the previous tile's copies have read the buffer
+            __syncthreads();
+            const unsigned int n_vec_bytes = (count / 4u) * 16u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const unsigned int off = BF16 ? ((q >> 1) * kReduceThreads + t) * 8 + (q & 1) * 4 : (q * kReduceThreads + t) * 4;
+                unsigned int r[4];
+                unpack2(acc.p[q * 2 + 0], r[0], r[1]);
+                unpack2(acc.p[q * 2 + 1], r[2], r[3]);
+                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(s_out + off * 4u), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+                if (off < count && off + 4 > count) {     // the ragged last vector: element by element, to every destination
+                    for (unsigned int d = 0; d <= task.n_fan; ++d) {
+                        float* o = d == 0 ? out : reinterpret_cast<float*>(fan_ptrs[task.fan_begin + d - 1]) + e0;
+                        for (int i = 0; i < 4; ++i)
+                            if (off + i < count) o[off + i] = __uint_as_float(r[i]);
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tile visible to the bulk-copy engine
+            __syncthreads();
+            if (t < kFanIssuers) {
+                if (n_vec_bytes != 0) {
+                    for (unsigned int d = t; d <= task.n_fan; d += kFanIssuers) {
+                        const unsigned long long base = d == 0 ? task.out_ptr : fan_ptrs[task.fan_begin + d - 1];
+                        bulk_store(base + e0 * 4ull, s_out, n_vec_bytes);
+                    }
+                }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            return;
+        }
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         const unsigned int off = BF16 ? ((q >> 1) * kReduceThreads + t) * 8 + (q & 1) * 4 : (q * kReduceThreads + t) * 4;
@@ -304,8 +354,8 @@ __device__ __forceinline__ void run_tile(unsigned int rec_base, unsigned int sta
     }
 }
 
-template <int A, bool BF16>
-__global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
+template <int A, bool BF16, bool FAN>
+__global__ void __launch_bounds__(kReduceThreads, StagesFor<A, FAN>::min_ctas) reduce_wave_kernel(const __grid_constant__ ReduceWave w) {
     extern __shared__ __align__(16) unsigned char s_stage[];
     __shared__ unsigned long long s_rec[kMaxStepsPerWave];
     const unsigned int t = threadIdx.x;
@@ -345,11 +395,15 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
                 if (meta_code(rec_meta(w.recs[task.step_begin + i])) != OPC_ADD_ACC)
                     ok &= wait_chunk(w.dir, w.status, w.rows[task.step_begin + i], c, t_start, w.budget_ns) ? 1 : 0;
             }
-            if (!__syncthreads_and(ok)) return;
+            if (!__syncthreads_and(ok)) break;
         }
 
         const unsigned int count = (unsigned int)(e1 - e0);
-        run_tile<A, BF16>(rec_base, stage_base, task, e0, count, t);
+        run_tile<A, BF16, FAN>(rec_base, stage_base, task, e0, count, t, w.fan_ptrs);
+    }
+    if constexpr (FAN) {
+        // shared memory must stay valid until the bulk copies have read it, and their writes must be complete
+        if (t < kFanIssuers) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 }
 
@@ -361,10 +415,6 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A>::min_ctas) reduce
 // (cp.async.bulk.wait_group), which always complete.
 constexpr int kFanoutIssuers = 64;
 constexpr int kFanoutSmemBytes = 2 * kFanoutTileBytes;
-
-__device__ __forceinline__ void bulk_store(unsigned long long gdst, unsigned int smem_src, unsigned int bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
-}
 
 __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __grid_constant__ FanoutWave w) {
     extern __shared__ __align__(128) unsigned char s_tile[];
@@ -444,56 +494,93 @@ __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __gri
 }
 
 // ------------------------------------------------------------------------------------------ launchers
-template <int A, bool BF16>
-static int launch_reduce_t(const ReduceWave& w, int grid, cudaStream_t s) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, StagesFor<A>::smem_bytes);
-        if (e != cudaSuccess) return (int)e;
-        attr_set = true;
-    }
-    reduce_wave_kernel<A, BF16><<<grid, kReduceThreads, StagesFor<A>::smem_bytes, s>>>(w);
-    return (int)cudaGetLastError();
-}
+// Per device and kernel variant: the dynamic shared memory attribute is set and the occupancy asked for once,
+// under a lock (cudaFuncSetAttribute is per device; contexts and hpl_reduce_noalloc may run on several threads).
+namespace {
 
-int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, int grid, void* stream) {
-    cudaStream_t s = (cudaStream_t)stream;
-    if (n_acc <= 2) return bf16 ? launch_reduce_t<2, true>(w, grid, s) : launch_reduce_t<2, false>(w, grid, s);
-    if (n_acc <= 4) return bf16 ? launch_reduce_t<4, true>(w, grid, s) : launch_reduce_t<4, false>(w, grid, s);
-    return bf16 ? launch_reduce_t<kMaxAcc, true>(w, grid, s) : launch_reduce_t<kMaxAcc, false>(w, grid, s);
-}
+constexpr int kVariants = 13;   // 3 accumulator classes x {f32, bf16} x {plain, fan} reduce variants + the fan-out kernel
+std::mutex g_variant_mu;
+std::vector<std::array<int, kVariants>> g_occ_of_device;   // 0 = not prepared yet
 
-int launch_fanout_wave(const FanoutWave& w, int grid, void* stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(fanout_wave_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFanoutSmemBytes);
-        if (e != cudaSuccess) return (int)e;
-        attr_set = true;
-    }
-    fanout_wave_kernel<<<grid, kFanoutThreads, kFanoutSmemBytes, (cudaStream_t)stream>>>(w);
-    return (int)cudaGetLastError();
-}
+int variant_index(int n_acc, bool bf16, bool fan) { return ((n_acc <= 2 ? 0 : (n_acc <= 4 ? 1 : 2)) * 2 + (bf16 ? 1 : 0)) * 2 + (fan ? 1 : 0); }
 
-template <int A, bool BF16>
-static int occ_t() {
+template <int A, bool BF16, bool FAN>
+int prepare_reduce_variant() {
     int n = 0;
-    if (cudaFuncSetAttribute(reduce_wave_kernel<A, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, StagesFor<A>::smem_bytes) != cudaSuccess) return 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reduce_wave_kernel<A, BF16>, kReduceThreads, StagesFor<A>::smem_bytes) != cudaSuccess) return 1;
+    if (cudaFuncSetAttribute(reduce_wave_kernel<A, BF16, FAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, StagesFor<A, FAN>::smem_bytes) != cudaSuccess) return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reduce_wave_kernel<A, BF16, FAN>, kReduceThreads, StagesFor<A, FAN>::smem_bytes) != cudaSuccess) return -1;
     return n < 1 ? 1 : n;
 }
 
-int reduce_ctas_per_sm(int n_acc, bool bf16) {
-    if (n_acc <= 2) return bf16 ? occ_t<2, true>() : occ_t<2, false>();
-    if (n_acc <= 4) return bf16 ? occ_t<4, true>() : occ_t<4, false>();
-    return bf16 ? occ_t<kMaxAcc, true>() : occ_t<kMaxAcc, false>();
+template <int A>
+int prepare_reduce_a(bool bf16, bool fan) {
+    if (bf16) return fan ? prepare_reduce_variant<A, true, true>() : prepare_reduce_variant<A, true, false>();
+    return fan ? prepare_reduce_variant<A, false, true>() : prepare_reduce_variant<A, false, false>();
+}
+
+int prepare_fanout() {
+    int n = 0;
+    if (cudaFuncSetAttribute(fanout_wave_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFanoutSmemBytes) != cudaSuccess) return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fanout_wave_kernel, kFanoutThreads, kFanoutSmemBytes) != cudaSuccess) return -1;
+    if (n > 2) n = 2;   // two CTAs per SM already saturate the write path
+    return n < 1 ? 1 : n;
+}
+
+// CTAs per SM of a variant on the current device (prepares it at first use); -1 on a CUDA error.
+int variant_occupancy(int idx, int n_acc, bool bf16, bool fan) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    std::lock_guard<std::mutex> lock(g_variant_mu);
+    if ((int)g_occ_of_device.size() <= dev) g_occ_of_device.resize(dev + 1, std::array<int, kVariants>{});
+    int& occ = g_occ_of_device[dev][idx];
+    if (occ == 0) {
+        int n;
+        if (idx == kVariants - 1) n = prepare_fanout();
+        else if (n_acc <= 2) n = prepare_reduce_a<2>(bf16, fan);
+        else if (n_acc <= 4) n = prepare_reduce_a<4>(bf16, fan);
+        else n = prepare_reduce_a<kMaxAcc>(bf16, fan);
+        if (n < 0) return -1;
+        occ = n;
+    }
+    return occ;
+}
+
+template <int A, bool BF16, bool FAN>
+int launch_reduce_t(const ReduceWave& w, int grid, cudaStream_t s) {
+    reduce_wave_kernel<A, BF16, FAN><<<grid, kReduceThreads, StagesFor<A, FAN>::smem_bytes, s>>>(w);
+    return (int)cudaGetLastError();
+}
+
+template <int A>
+int launch_reduce_a(const ReduceWave& w, bool bf16, bool fan, int grid, cudaStream_t s) {
+    if (bf16) return fan ? launch_reduce_t<A, true, true>(w, grid, s) : launch_reduce_t<A, true, false>(w, grid, s);
+    return fan ? launch_reduce_t<A, false, true>(w, grid, s) : launch_reduce_t<A, false, false>(w, grid, s);
+}
+
+}  // namespace
+
+int reduce_ctas_per_sm(int n_acc, bool bf16, bool fan) {
+    const int n = variant_occupancy(variant_index(n_acc, bf16, fan), n_acc, bf16, fan);
+    return n < 1 ? 1 : n;
 }
 
 int fanout_ctas_per_sm() {
-    int n = 0;
-    if (cudaFuncSetAttribute(fanout_wave_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFanoutSmemBytes) != cudaSuccess) return 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fanout_wave_kernel, kFanoutThreads, kFanoutSmemBytes) != cudaSuccess) return 1;
-    if (n > 2) n = 2;   // two CTAs per SM already saturate the write path
+    const int n = variant_occupancy(kVariants - 1, 0, false, false);
     return n < 1 ? 1 : n;
+}
+
+int launch_reduce_wave(const ReduceWave& w, int n_acc, bool bf16, bool fan, int grid, void* stream) {
+    cudaStream_t s = (cudaStream_t)stream;
+    if (variant_occupancy(variant_index(n_acc, bf16, fan), n_acc, bf16, fan) < 0) return (int)cudaErrorUnknown;
+    if (n_acc <= 2) return launch_reduce_a<2>(w, bf16, fan, grid, s);
+    if (n_acc <= 4) return launch_reduce_a<4>(w, bf16, fan, grid, s);
+    return launch_reduce_a<kMaxAcc>(w, bf16, fan, grid, s);
+}
+
+int launch_fanout_wave(const FanoutWave& w, int grid, void* stream) {
+    if (variant_occupancy(kVariants - 1, 0, false, false) < 0) return (int)cudaErrorUnknown;
+    fanout_wave_kernel<<<grid, kFanoutThreads, kFanoutSmemBytes, (cudaStream_t)stream>>>(w);
+    return (int)cudaGetLastError();
 }
 
 }  // namespace hpl

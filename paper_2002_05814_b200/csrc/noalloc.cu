@@ -172,6 +172,7 @@ extern "C" int hpl_reduce_noalloc(const void* const* src_bufs, int32_t n, int32_
     t.n_steps = (uint32_t)steps.size();
     t.red_op = (uint32_t)op;
     t.poll = 0;
+    t.fan_begin = t.n_fan = 0;
     t.pad = 0;
     for (size_t i = 0; i < steps.size(); ++i) {
         w.recs[i] = pack_step(steps[i]);   // address 0: the kernel takes it from the row in the scratch array
@@ -179,10 +180,10 @@ extern "C" int hpl_reduce_noalloc(const void* const* src_bufs, int32_t n, int32_
     }
     w.total_tiles = C * tpc;
     const bool bf16 = dtype == HPL_BF16;
-    int occ = reduce_ctas_per_sm(n_acc, bf16);
+    int occ = reduce_ctas_per_sm(n_acc, bf16, false);
     uint64_t grid = (uint64_t)n_sm * (occ < 1 ? 1 : occ);
     if (grid > w.total_tiles) grid = w.total_tiles;
     if (grid < 1) grid = 1;
-    if (launch_reduce_wave(w, n_acc, bf16, (int)grid, stream) != 0) return HPL_ERR_CUDA;
+    if (launch_reduce_wave(w, n_acc, bf16, false, (int)grid, stream) != 0) return HPL_ERR_CUDA;
     return HPL_OK;
 }

@@ -274,6 +274,35 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
 
 int occ_index(int n_acc) { return n_acc <= 2 ? 0 : (n_acc <= 4 ? 1 : 2); }
 
+// Reduce followed by broadcast (Section 3.4.3): receivers of a broadcast of this Reduce's output that need exactly
+// the elements a root task is about to produce take them from that task -- its result tile goes to the target and
+// to them in one pass, instead of being written and read again by a fan-out wave.  Returns the receivers' buffer
+// addresses (at most `room`); their holdings are advanced like those of a planned fan-out task.
+static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, const PlannedReduceTask& t, size_t room, std::vector<unsigned long long>& out) {
+    out.clear();
+    if (!c->cfg.fuse_fanout || room == 0 || t.pos != 0 || t.end != op.n_ops(0)) return;
+    auto bi = c->bcast_of_src.find(op.target);
+    if (bi == c->bcast_of_src.end()) return;
+    BcastOp& b = c->bcasts.at(bi->second);
+    Object* tgt = find(c, op.target);
+    if (!tgt || !tgt->alive) return;
+    // the task's elements in chunks of the broadcast (the output's own chunks)
+    const uint64_t cbe = object_chunk_elems(c, *tgt);
+    const uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
+    if (e_lo % cbe != 0 || (e_hi % cbe != 0 && e_hi != op.elems)) return;
+    const int64_t a_b = (int64_t)(e_lo / cbe), b_b = e_hi == op.elems ? (int64_t)tgt->C : (int64_t)(e_hi / cbe);
+    const auto& locs = b.sched->locations();
+    b.phys_have.resize(locs.size(), 0);
+    for (size_t r = 1; r < locs.size() && out.size() < room; ++r) {
+        if (!locs[r].alive || locs[r].last_sender < 0 || b.phys_have[r] != a_b) continue;
+        Object* o = find(c, locs[r].obj);
+        if (!o || !o->alive || !o->ptr || o->row < 0) continue;
+        c->journal.b.push_back({b.src, (int)r, b.phys_have[r], c->batch_tag});
+        b.phys_have[r] = b_b;
+        out.push_back((unsigned long long)(uintptr_t)o->ptr);
+    }
+}
+
 int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
     if (tasks.empty()) return HPL_OK;
     int max_level = 0;
@@ -292,8 +321,9 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             w.budget_ns = c->cfg.poll_budget_ns;
             w.n_tasks = 0;
             w.total_tiles = 0;
-            uint32_t n_steps = 0;
+            uint32_t n_steps = 0, n_fan = 0;
             int n_acc = 1;
+            std::vector<unsigned long long> fan;
             while (i < lv.size() && w.n_tasks < (uint32_t)kMaxTasksPerWave &&
                    n_steps + lv[i]->steps.size() <= (size_t)kMaxStepsPerWave) {
                 PlannedReduceTask& t = *lv[i];
@@ -313,6 +343,10 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 d.red_op = (uint32_t)op.red_op;
                 d.poll = t.poll ? 1u : 0u;
                 if (t.poll) c->polling_in_flight = true;
+                claim_fused_receivers(c, op, t, (size_t)kMaxFusedDst - n_fan, fan);
+                d.fan_begin = n_fan;
+                d.n_fan = (uint32_t)fan.size();
+                for (unsigned long long p : fan) w.fan_ptrs[n_fan++] = p;
                 d.pad = 0;
                 for (size_t q = 0; q < t.steps.size(); ++q) {
                     w.recs[n_steps + q] = pack_step(t.steps[q]);
@@ -325,8 +359,9 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
                 for (auto& st : t.steps)
                     if (st.code != OPC_ADD_ACC) c->stats.bytes_read_planned += (e_hi - e_lo) * (st.kind == SRC_BF16 ? 2 : 4);
-                c->stats.bytes_written_planned += (e_hi - e_lo) * 4;
+                c->stats.bytes_written_planned += (e_hi - e_lo) * 4 * (1 + fan.size());
                 c->stats.reduce_tasks++;
+                if (!fan.empty()) c->stats.fused_fanout_tasks++;
                 ++i;
             }
             if (w.n_tasks == 0) return HPL_ERR_INVALID;  // a single task larger than a wave: tree too wide
@@ -336,8 +371,9 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
                 c->stats.tiles += w.total_tiles;
                 continue;
             }
-            int& occ = c->occ_reduce[bf16 ? 1 : 0][occ_index(n_acc)];
-            if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16);
+            const bool fanned = n_fan != 0;
+            int& occ = c->occ_reduce[bf16 ? 1 : 0][fanned ? 1 : 0][occ_index(n_acc)];
+            if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16, fanned);
             int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
             if (grid < 1) grid = 1;
             if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
@@ -347,7 +383,7 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
             w.status = next_wave_status(c);
             {
                 LaunchTimer timer(c, 0);
-                if (launch_reduce_wave(w, n_acc, bf16, grid, c->stream) != 0) return HPL_ERR_CUDA;
+                if (launch_reduce_wave(w, n_acc, bf16, fanned, grid, c->stream) != 0) return HPL_ERR_CUDA;
             }
             c->stats.kernel_launches++;
             c->stats.reduce_launches++;

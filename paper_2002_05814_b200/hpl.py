@@ -31,7 +31,8 @@ class Config(C.Structure):
                 ("virt_chunk_ns", C.c_uint64), ("poll_budget_ns", C.c_uint64), ("eager", C.c_int32),
                 ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
-                ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64)]
+                ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64),
+                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -40,7 +41,7 @@ class Stats(C.Structure):
                                           "bytes_read_planned", "bytes_written_planned", "device_timeouts",
                                           "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
                                           "reduce_launches", "fanout_launches", "reduce_kernel_ns",
-                                          "fanout_kernel_ns", "device_waits")]
+                                          "fanout_kernel_ns", "device_waits", "fused_fanout_tasks")]
 
 
 class Event(C.Structure):
@@ -154,11 +155,11 @@ class Context:
     def __init__(self, chunk_bytes: int, reduce_degree: int = 2, bcast_degree: int = 2, *, arena=0,
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
                  eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False,
-                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0):
+                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0, fuse_fanout: bool = True):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
                      int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes,
-                     model_latency_ns, model_bandwidth_bps)
+                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0)
         self._h = C.c_void_p()
         self._p, self._n = C.c_void_p(), C.c_uint64()
         self._pref, self._nref = C.byref(self._p), C.byref(self._n)

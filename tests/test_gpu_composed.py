@@ -57,9 +57,10 @@ def test_bf16_first_stage_feeds_an_fp32_second_stage():
     p.close()
 
 
-def test_allreduce_is_reduce_then_broadcast():
+@pytest.mark.parametrize("fuse_fanout", [True, False])
+def test_allreduce_is_reduce_then_broadcast(fuse_fanout):
     elems, chunk, R = 5 * 4096 + 12, 16 << 10, 6
-    p = Pair(chunk, 2, 2, tau=50)
+    p = Pair(chunk, 2, 2, tau=50, fuse_fanout=fuse_fanout)
     for i in range(4):
         p.create(i, i, gen(("uniform",), 93, i, elems))
     for j in range(R):
@@ -88,6 +89,66 @@ def test_allreduce_is_reduce_then_broadcast():
         p.check_receiver_bytes(50 + j)
         assert p.dev[50 + j].view(torch.uint8).cpu().numpy().tobytes() == want.tobytes()
     p.check_schedule(100)
+    p.close()
+
+
+@pytest.mark.parametrize("dtype,k,R,elems,chunk,d", [("f32", 8, 8, 3 * 4096 + 7, 16 << 10, 2), ("bf16", 8, 8, 70_001, 32 << 10, 2),
+                                                     ("bf16", 64, 64, 24_576, 16 << 10, 4), ("f32", 3, 5, 6, 4096, 1),
+                                                     ("f32", 1, 3, 5000, 4096, 2), ("bf16", 5, 130, 9000, 8 << 10, 4)])
+def test_fused_allreduce_every_receiver_holds_the_target_bits(dtype, k, R, elems, chunk, d):
+    """Reduce followed by broadcast with all receivers joined before anything runs: one pass writes the target and every
+    receiver (ragged tiles, bf16 inputs whose chunks are twice the output's, more receivers than one wave serves)."""
+    p = Pair(chunk, d, 2)
+    code = DT_BF16 if dtype == "bf16" else DT_F32
+    for i in range(k):
+        p.create(i, i, gen(("uniform",) if dtype == "f32" else ("normal", 0.02), 97, i, elems, dtype))
+    for j in range(R):
+        p.create(1000 + j, 500 + j, nbytes=elems * 4, dtype=DT_F32)
+    p.reduce(100, list(range(k)), k, 0, code)
+    p.broadcast(100, [1000 + j for j in range(R)])
+    for j in range(R):
+        p.join(1000 + j)
+    p.advance(5)
+    for i in range(k):
+        p.put(i)
+    want = p.check_target_bits(100).cpu().numpy()
+    for j in range(R):
+        p.check_receiver_bytes(1000 + j)
+        assert p.dev[1000 + j].view(torch.uint8).cpu().numpy().tobytes() == want.tobytes()
+    st = p.c.stats()
+    assert st["fused_fanout_tasks"] >= 1 and st["bytes_read_planned"] <= k * p.host[0].nbytes + max(0, R - 128) * elems * 4
+    assert st["bytes_written_planned"] == (R + 1) * elems * 4
+    p.close()
+
+
+def test_fused_allreduce_with_a_member_lost_half_way_is_redone_for_target_and_receivers():
+    elems, chunk, k, R = 8 * 4096 + 5, 16 << 10, 6, 4
+    p = Pair(chunk, 2, 2)
+    for i in range(k + 1):
+        p.create(i, i, gen(("uniform",), 98, i, elems))
+    for j in range(R):
+        p.create(1000 + j, 500 + j, nbytes=elems * 4, dtype=DT_F32)
+    p.reduce(100, list(range(k + 1)), k)               # object k is the spare
+    p.broadcast(100, [1000 + j for j in range(R)])
+    for j in range(R):
+        p.join(1000 + j)
+    for i in range(k):
+        p.advance(i + 1)
+        p.put(i, 4 * chunk)                            # half of every object
+    p.progress()                                       # half of the result is in the target and in the receivers
+    assert p.c.stats()["fused_fanout_tasks"] >= 1
+    p.advance(50)
+    p.fail(2)
+    p.advance(60)
+    p.put(k)
+    for i in range(k):
+        if i != 2:
+            p.put(i)
+    want = p.check_target_bits(100).cpu().numpy()
+    p.check_schedule(100)
+    for j in range(R):
+        p.check_receiver_bytes(1000 + j)
+        assert p.dev[1000 + j].view(torch.uint8).cpu().numpy().tobytes() == want.tobytes()
     p.close()
 
 

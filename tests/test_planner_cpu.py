@@ -111,9 +111,10 @@ def test_a_tree_larger_than_one_task_is_cut_and_launched_in_levels():
         assert ei.value.code == hpl.HPL_ERR_INVALID
 
 
-def test_composed_collectives_are_planned_in_creation_order():
+@pytest.mark.parametrize("fuse_fanout", [False, True])
+def test_composed_collectives_are_planned_in_creation_order(fuse_fanout):
     S = 1 << 18
-    with hpl.Context(64 << 10, 2, 2) as c:
+    with hpl.Context(64 << 10, 2, 2, fuse_fanout=fuse_fanout) as c:
         for i in range(6):
             c.create(i, i, S)
             c.put(i, _addr(i), S)
@@ -123,5 +124,29 @@ def test_composed_collectives_are_planned_in_creation_order():
         c.broadcast(200, [300])
         c.join(300, _addr(30))
         st = _plan_get(c, 300)
-        assert st["reduce_tasks"] == 2 and st["fanout_tasks"] == 1
-        assert st["bytes_read_planned"] == 3 * S + 4 * S + S      # inputs of each stage, then the output once
+        if fuse_fanout:      # the second stage's result goes to its target and to the receiver in the same pass
+            assert st["reduce_tasks"] == 2 and st["fanout_tasks"] == 0 and st["fused_fanout_tasks"] == 1
+            assert st["bytes_read_planned"] == 3 * S + 4 * S and st["bytes_written_planned"] == 3 * S
+            assert st["kernel_launches"] == 2
+        else:
+            assert st["reduce_tasks"] == 2 and st["fanout_tasks"] == 1
+            assert st["bytes_read_planned"] == 3 * S + 4 * S + S      # inputs of each stage, then the output once
+
+
+def test_allreduce_of_8_to_8_is_one_pass_that_never_reads_the_target():
+    """Reduce followed by broadcast (Section 3.4.3) with every receiver joined: k objects read, the result written to
+    the target and to each receiver, one launch."""
+    S, k, R = 1 << 20, 8, 8
+    with hpl.Context(64 << 10, 2, 2) as c:
+        for i in range(k):
+            c.create(i, i, S)
+            c.put(i, _addr(i), S)
+        c.reduce(100, list(range(k)), k)
+        for j in range(R):
+            c.create(200 + j, 50 + j, S)
+        c.broadcast(100, [200 + j for j in range(R)])
+        for j in range(R):
+            c.join(200 + j, _addr(40 + j))
+        st = _plan_get(c, 200)
+        assert st["kernel_launches"] == 1 and st["reduce_launches"] == 1 and st["fanout_launches"] == 0
+        assert st["bytes_read_planned"] == k * S and st["bytes_written_planned"] == (R + 1) * S
