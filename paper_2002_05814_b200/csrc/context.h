@@ -24,6 +24,7 @@ constexpr uint32_t kStatusSlots = 256;   // one error record per wave in flight;
 constexpr uint32_t kMaxChunks = 1u << 20;
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kStageRows = 4 * kMaxRows;
+constexpr uint64_t kSmallObjectBytes = 64 * 1024;   // Section 3.2's threshold for small objects
 
 // Per tree position: for which chunks how many leading operands of the node (first child, own object, second
 // child, ...) have been merged into its result buffer.  All operands merged = the node's result is complete.
@@ -179,6 +180,7 @@ struct PlannedReduceTask {
     int n_acc;
     bool poll;
     std::vector<ReduceStep> steps;
+    std::vector<unsigned long long> fan;   // buffers of broadcast receivers that take the result from this task (root tasks only)
 };
 
 struct ReduceOp {
@@ -299,11 +301,13 @@ void release_object_memory(hpl_ctx* c, Object& o);
 // plan_reduce.cpp
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);
 int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);
+int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedReduceTask*>>& group, bool bf16);
 void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv);
 
 // plan_bcast.cpp
 int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks);
 int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks);
+int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanout>>& group);
 
 // Brackets one launch with events when kernel timing is on (kind 0 = reduce, 1 = fan-out).
 struct LaunchTimer {

@@ -18,6 +18,47 @@ namespace {
 int sync_and_check(hpl_ctx* c);
 int progress(hpl_ctx* c);
 
+// Small objects (Section 3.2 treats objects under 64 KB apart: for them latency, not bandwidth, is the cost).
+// Their collectives do not get launches of their own: the tasks planned for them in one pass are gathered and
+// packed into shared waves -- one launch serves many small collectives, and a batch of Gets waits once.  A task is
+// placed in the stage after everything it reads from: the levels of its own collective, and the collectives
+// whose output it consumes.  Polling tasks stay out (a wait that runs out voids the wave it is in).
+struct SmallBatch {
+    struct R { ReduceOp* op; std::vector<PlannedReduceTask> tasks; int base; };
+    struct F { BcastOp* op; std::vector<PlannedFanout> tasks; int stage; };
+    std::vector<R> r;
+    std::vector<F> f;
+    std::unordered_map<int64_t, int> end_stage;   // output id -> last stage that writes it in this batch
+    bool empty() const { return r.empty() && f.empty(); }
+};
+
+int flush_small(hpl_ctx* c, SmallBatch& sb) {
+    if (sb.empty()) return HPL_OK;
+    int last = 0;
+    for (auto& x : sb.r)
+        for (auto& t : x.tasks) last = std::max(last, x.base + t.level);
+    for (auto& x : sb.f) last = std::max(last, x.stage);
+    for (int stage = 1; stage <= last; ++stage) {
+        for (int bf = 0; bf < 2; ++bf) {
+            std::vector<std::pair<ReduceOp*, PlannedReduceTask*>> g;
+            for (auto& x : sb.r)
+                if ((x.op->in_dtype == HPL_BF16) == (bf == 1))
+                    for (auto& t : x.tasks)
+                        if (x.base + t.level == stage) g.push_back({x.op, &t});
+            int rc = launch_reduce_group(c, g, bf == 1);
+            if (rc != HPL_OK) return rc;
+        }
+        std::vector<std::pair<BcastOp*, PlannedFanout>> g;
+        for (auto& x : sb.f)
+            if (x.stage == stage)
+                for (auto& t : x.tasks) g.push_back({x.op, std::move(t)});
+        int rc = launch_fanout_group(c, g);
+        if (rc != HPL_OK) return rc;
+    }
+    sb = SmallBatch();
+    return HPL_OK;
+}
+
 int progress(hpl_ctx* c) {
     // (a schedule-only context plans as well -- its planned tasks are counted, nothing is launched)
     {
@@ -34,28 +75,58 @@ int progress(hpl_ctx* c) {
     }
     // collectives in creation order, so that one that consumes another's output (composed Reduce, reduce
     // followed by broadcast) is planned after its producer and launched behind it on the stream
+    SmallBatch sb;
     auto ri = c->reduces.begin();
     auto bi = c->bcasts.begin();
     while (ri != c->reduces.end() || bi != c->bcasts.end()) {
         const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
         c->batch_tag = c->launch_seq;
         if (take_reduce) {
+            ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
-            int rc = plan_reduce(c, ri->second, tasks);
+            int rc = plan_reduce(c, op, tasks);
             if (rc != HPL_OK) return rc;
-            rc = launch_reduce_tasks(c, ri->second, tasks);
-            if (rc != HPL_OK) return rc;
+            bool small = op.elems * 4 <= kSmallObjectBytes;
+            for (auto& t : tasks) small = small && !t.poll;
+            if (small && !tasks.empty()) {
+                int base = 0, top = 0;
+                for (int p = 0; p < op.sched->k(); ++p) {   // behind the collectives whose output is a member
+                    auto e = sb.end_stage.find(op.sched->object_at(p));
+                    if (e != sb.end_stage.end()) base = std::max(base, e->second);
+                }
+                for (auto& t : tasks) top = std::max(top, t.level);
+                sb.end_stage[op.target] = base + top;
+                sb.r.push_back({&op, std::move(tasks), base});
+            } else if (!tasks.empty()) {
+                rc = flush_small(c, sb);     // what was planned earlier is launched earlier
+                if (rc != HPL_OK) return rc;
+                c->batch_tag = c->launch_seq;
+                rc = launch_reduce_tasks(c, op, tasks);
+                if (rc != HPL_OK) return rc;
+            }
             ++ri;
         } else {
+            BcastOp& op = bi->second;
             std::vector<PlannedFanout> tasks;
-            int rc = plan_bcast(c, bi->second, tasks);
+            int rc = plan_bcast(c, op, tasks);
             if (rc != HPL_OK) return rc;
-            rc = launch_fanout_tasks(c, bi->second, tasks);
-            if (rc != HPL_OK) return rc;
+            Object* src = find(c, op.src);
+            bool small = src && src->bytes <= kSmallObjectBytes;
+            for (auto& t : tasks) small = small && !t.poll;
+            if (small && !tasks.empty()) {
+                auto e = sb.end_stage.find(op.src);
+                sb.f.push_back({&op, std::move(tasks), (e == sb.end_stage.end() ? 0 : e->second) + 1});
+            } else if (!tasks.empty()) {
+                rc = flush_small(c, sb);
+                if (rc != HPL_OK) return rc;
+                c->batch_tag = c->launch_seq;
+                rc = launch_fanout_tasks(c, op, tasks);
+                if (rc != HPL_OK) return rc;
+            }
             ++bi;
         }
     }
-    return HPL_OK;
+    return flush_small(c, sb);
 }
 
 // Voids what was planned by the passes whose waves have seq >= from_tag (a wave of that pass gave up, and
@@ -654,6 +725,12 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
     if (o->kind == OBJ_TARGET) {
         ReduceOp& op = c->reduces.at(c->reduce_of_target.at(id));
         if (op.sched->k() == 0) return HPL_ERR_INSUFFICIENT;
+        if (c->device && !c->work_in_flight && !c->copy_pending && !c->ctl_unconfirmed && op.sched->full() &&
+            op.merged[0].covers(0, op.C, op.n_ops(0))) {
+            if (dev_ptr) *dev_ptr = o->ptr;   // computed and waited for already (e.g. by an earlier Get of a batch)
+            if (bytes) *bytes = o->bytes;
+            return HPL_OK;
+        }
         int rc = progress(c);   // whatever can run now runs, even if the target cannot complete yet
         if (rc != HPL_OK) return rc;
         if (!op.sched->full()) return HPL_ERR_TIMEOUT;

@@ -84,12 +84,10 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
     return HPL_OK;
 }
 
-int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+// Packs fan-out tasks (of one broadcast, or of several small ones) into waves and launches them.
+int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanout>>& tasks) {
     if (tasks.empty()) return HPL_OK;
-    Object* src = find(c, op.src);
-    const auto& locs = op.sched->locations();
     const uint64_t chunk_bytes = c->cfg.chunk_bytes;
-    const uint32_t tpc = (uint32_t)((std::min<uint64_t>(chunk_bytes, src->bytes) + kFanoutTileBytes - 1) / kFanoutTileBytes);
     size_t i = 0;
     while (i < tasks.size()) {
         static thread_local FanoutWave w;
@@ -100,17 +98,20 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         w.total_tiles = 0;
         uint32_t n_dst = 0;
         while (i < tasks.size() && w.n_tasks < (uint32_t)kMaxFanoutTasks) {
-            PlannedFanout& t = tasks[i];
-            if (t.dst.size() > (size_t)kMaxFanoutDst) {
+            if (tasks[i].second.dst.size() > (size_t)kMaxFanoutDst) {
                 // more receivers than one task holds: split the receiver list
-                PlannedFanout rest = t;
-                rest.dst.assign(t.dst.begin() + kMaxFanoutDst, t.dst.end());
-                t.dst.resize(kMaxFanoutDst);
+                std::pair<BcastOp*, PlannedFanout> rest = tasks[i];
+                rest.second.dst.assign(tasks[i].second.dst.begin() + kMaxFanoutDst, tasks[i].second.dst.end());
+                tasks[i].second.dst.resize(kMaxFanoutDst);
                 tasks.insert(tasks.begin() + i + 1, rest);
                 continue;
             }
-            if (n_dst + tasks[i].dst.size() > (size_t)kMaxFanoutDst) break;
-            PlannedFanout& tt = tasks[i];
+            if (n_dst + tasks[i].second.dst.size() > (size_t)kMaxFanoutDst) break;
+            BcastOp& op = *tasks[i].first;
+            PlannedFanout& tt = tasks[i].second;
+            Object* src = find(c, op.src);
+            const auto& locs = op.sched->locations();
+            const uint32_t tpc = (uint32_t)((std::min<uint64_t>(chunk_bytes, src->bytes) + kFanoutTileBytes - 1) / kFanoutTileBytes);
             FanoutTask& d = w.tasks[w.n_tasks++];
             Object* lo = tt.loc == 0 ? src : find(c, locs[tt.loc].obj);
             d.src_row = (uint32_t)lo->row;
@@ -159,6 +160,12 @@ int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tas
         c->work_in_flight = true;
     }
     return HPL_OK;
+}
+
+int launch_fanout_tasks(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
+    std::vector<std::pair<BcastOp*, PlannedFanout>> g;
+    for (auto& t : tasks) g.push_back({&op, std::move(t)});
+    return launch_fanout_group(c, g);
 }
 
 }  // namespace hpl

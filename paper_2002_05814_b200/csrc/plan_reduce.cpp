@@ -184,6 +184,37 @@ void visit_for_progress(ReducePlanCtx& p, int v) {
     }
 }
 
+// Reduce followed by broadcast (Section 3.4.3): receivers of a broadcast of this Reduce's output that need exactly
+// the elements a root task is about to produce take them from that task -- its result tile goes to the target and
+// to them in one pass, instead of being written and read again by a fan-out wave.  Returns the receivers' buffer
+// addresses (at most `room`); their holdings are advanced like those of a planned fan-out task.
+static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, PlannedReduceTask& t) {
+    std::vector<unsigned long long>& out = t.fan;
+    const size_t room = kMaxFusedDst;
+    out.clear();
+    if (!c->cfg.fuse_fanout || t.pos != 0 || t.end != op.n_ops(0)) return;
+    auto bi = c->bcast_of_src.find(op.target);
+    if (bi == c->bcast_of_src.end()) return;
+    BcastOp& b = c->bcasts.at(bi->second);
+    Object* tgt = find(c, op.target);
+    if (!tgt || !tgt->alive) return;
+    // the task's elements in chunks of the broadcast (the output's own chunks)
+    const uint64_t cbe = object_chunk_elems(c, *tgt);
+    const uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
+    if (e_lo % cbe != 0 || (e_hi % cbe != 0 && e_hi != op.elems)) return;
+    const int64_t a_b = (int64_t)(e_lo / cbe), b_b = e_hi == op.elems ? (int64_t)tgt->C : (int64_t)(e_hi / cbe);
+    const auto& locs = b.sched->locations();
+    b.phys_have.resize(locs.size(), 0);
+    for (size_t r = 1; r < locs.size() && out.size() < room; ++r) {
+        if (!locs[r].alive || locs[r].last_sender < 0 || b.phys_have[r] != a_b) continue;
+        Object* o = find(c, locs[r].obj);
+        if (!o || !o->alive || !o->ptr || o->row < 0) continue;
+        c->journal.b.push_back({b.src, (int)r, b.phys_have[r], c->batch_tag});
+        b.phys_have[r] = b_b;
+        out.push_back((unsigned long long)(uintptr_t)o->ptr);
+    }
+}
+
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
     ReduceTreeSchedule& s = *op.sched;
     const int k = s.k();
@@ -269,128 +300,107 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
             if (!merged) tasks.push_back(std::move(t));
         }
     }
+    for (auto& t : tasks) claim_fused_receivers(c, op, t);   // on the final tasks: a claim is for exactly the task's elements
     return HPL_OK;
 }
 
 int occ_index(int n_acc) { return n_acc <= 2 ? 0 : (n_acc <= 4 ? 1 : 2); }
 
-// Reduce followed by broadcast (Section 3.4.3): receivers of a broadcast of this Reduce's output that need exactly
-// the elements a root task is about to produce take them from that task -- its result tile goes to the target and
-// to them in one pass, instead of being written and read again by a fan-out wave.  Returns the receivers' buffer
-// addresses (at most `room`); their holdings are advanced like those of a planned fan-out task.
-static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, const PlannedReduceTask& t, size_t room, std::vector<unsigned long long>& out) {
-    out.clear();
-    if (!c->cfg.fuse_fanout || room == 0 || t.pos != 0 || t.end != op.n_ops(0)) return;
-    auto bi = c->bcast_of_src.find(op.target);
-    if (bi == c->bcast_of_src.end()) return;
-    BcastOp& b = c->bcasts.at(bi->second);
-    Object* tgt = find(c, op.target);
-    if (!tgt || !tgt->alive) return;
-    // the task's elements in chunks of the broadcast (the output's own chunks)
-    const uint64_t cbe = object_chunk_elems(c, *tgt);
-    const uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
-    if (e_lo % cbe != 0 || (e_hi % cbe != 0 && e_hi != op.elems)) return;
-    const int64_t a_b = (int64_t)(e_lo / cbe), b_b = e_hi == op.elems ? (int64_t)tgt->C : (int64_t)(e_hi / cbe);
-    const auto& locs = b.sched->locations();
-    b.phys_have.resize(locs.size(), 0);
-    for (size_t r = 1; r < locs.size() && out.size() < room; ++r) {
-        if (!locs[r].alive || locs[r].last_sender < 0 || b.phys_have[r] != a_b) continue;
-        Object* o = find(c, locs[r].obj);
-        if (!o || !o->alive || !o->ptr || o->row < 0) continue;
-        c->journal.b.push_back({b.src, (int)r, b.phys_have[r], c->batch_tag});
-        b.phys_have[r] = b_b;
-        out.push_back((unsigned long long)(uintptr_t)o->ptr);
+// Packs the tasks of one dependency level (of one collective, or of several small ones) into waves and launches
+// them.  All tasks of a group read inputs of one dtype class (`bf16`); every task carries its own geometry.
+int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedReduceTask*>>& lv, bool bf16) {
+    size_t i = 0;
+    while (i < lv.size()) {
+        static thread_local ReduceWave w;
+        w.dir = c->d_dir;
+        w.status = nullptr;
+        w.budget_ns = c->cfg.poll_budget_ns;
+        w.n_tasks = 0;
+        w.total_tiles = 0;
+        uint32_t n_steps = 0, n_fan = 0;
+        int n_acc = 1;
+        while (i < lv.size() && w.n_tasks < (uint32_t)kMaxTasksPerWave &&
+               n_steps + lv[i].second->steps.size() <= (size_t)kMaxStepsPerWave && n_fan + lv[i].second->fan.size() <= (size_t)kMaxFusedDst) {
+            ReduceOp& op = *lv[i].first;
+            PlannedReduceTask& t = *lv[i].second;
+            const uint32_t tpc_full = (op.chunk_elems + kTileElems - 1) / kTileElems;
+            Object* out = nullptr;
+            int rc = ensure_partial_buffer(c, op, t.pos, &out);
+            if (rc != HPL_OK) return rc;
+            ReduceTask& d = w.tasks[w.n_tasks++];
+            d.out_ptr = (unsigned long long)(uintptr_t)out->ptr;
+            d.elems = op.elems;
+            d.chunk_elems = op.chunk_elems;
+            d.c_begin = t.a;
+            d.c_end = t.b;
+            d.tiles_per_chunk = tpc_full;
+            d.tile_begin = w.total_tiles;
+            d.step_begin = n_steps;
+            d.n_steps = (uint32_t)t.steps.size();
+            d.red_op = (uint32_t)op.red_op;
+            d.poll = t.poll ? 1u : 0u;
+            if (t.poll) c->polling_in_flight = true;
+            const std::vector<unsigned long long>& fan = t.fan;
+            d.fan_begin = n_fan;
+            d.n_fan = (uint32_t)fan.size();
+            for (unsigned long long p : fan) w.fan_ptrs[n_fan++] = p;
+            d.pad = 0;
+            for (size_t q = 0; q < t.steps.size(); ++q) {
+                w.recs[n_steps + q] = pack_step(t.steps[q]);
+                w.rows[n_steps + q] = t.steps[q].row;
+            }
+            n_steps += d.n_steps;
+            w.total_tiles += (t.b - t.a) * tpc_full;
+            n_acc = std::max(n_acc, t.n_acc);
+            // accounting: bytes the task moves
+            uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
+            for (auto& st : t.steps)
+                if (st.code != OPC_ADD_ACC) c->stats.bytes_read_planned += (e_hi - e_lo) * (st.kind == SRC_BF16 ? 2 : 4);
+            c->stats.bytes_written_planned += (e_hi - e_lo) * 4 * (1 + fan.size());
+            c->stats.reduce_tasks++;
+            if (!fan.empty()) c->stats.fused_fanout_tasks++;
+            ++i;
+        }
+        if (w.n_tasks == 0) return HPL_ERR_INVALID;  // a single task larger than a wave: tree too wide
+        if (!c->device) {   // schedule-only context: the wave is planned and counted, not run
+            c->stats.kernel_launches++;
+            c->stats.reduce_launches++;
+            c->stats.tiles += w.total_tiles;
+            continue;
+        }
+        const bool fanned = n_fan != 0;
+        int& occ = c->occ_reduce[bf16 ? 1 : 0][fanned ? 1 : 0][occ_index(n_acc)];
+        if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16, fanned);
+        int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
+        if (grid < 1) grid = 1;
+        if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
+        bool polls = false;
+        for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
+        if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counters it waits on are rows of the directory
+        w.status = next_wave_status(c);
+        {
+            LaunchTimer timer(c, 0);
+            if (launch_reduce_wave(w, n_acc, bf16, fanned, grid, c->stream) != 0) return HPL_ERR_CUDA;
+        }
+        c->stats.kernel_launches++;
+        c->stats.reduce_launches++;
+        c->stats.tiles += w.total_tiles;
+        c->stats.last_kernel_grid = (uint64_t)grid;
+        c->work_in_flight = true;
     }
+    return HPL_OK;
 }
 
 int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
     if (tasks.empty()) return HPL_OK;
     int max_level = 0;
     for (auto& t : tasks) max_level = std::max(max_level, t.level);
-    const bool bf16 = op.in_dtype == HPL_BF16;
-    const uint32_t tpc_full = (op.chunk_elems + kTileElems - 1) / kTileElems;
     for (int level = 1; level <= max_level; ++level) {
-        size_t i = 0;
-        std::vector<PlannedReduceTask*> lv;
+        std::vector<std::pair<ReduceOp*, PlannedReduceTask*>> lv;
         for (auto& t : tasks)
-            if (t.level == level) lv.push_back(&t);
-        while (i < lv.size()) {
-            static thread_local ReduceWave w;
-            w.dir = c->d_dir;
-            w.status = nullptr;
-            w.budget_ns = c->cfg.poll_budget_ns;
-            w.n_tasks = 0;
-            w.total_tiles = 0;
-            uint32_t n_steps = 0, n_fan = 0;
-            int n_acc = 1;
-            std::vector<unsigned long long> fan;
-            while (i < lv.size() && w.n_tasks < (uint32_t)kMaxTasksPerWave &&
-                   n_steps + lv[i]->steps.size() <= (size_t)kMaxStepsPerWave) {
-                PlannedReduceTask& t = *lv[i];
-                Object* out = nullptr;
-                int rc = ensure_partial_buffer(c, op, t.pos, &out);
-                if (rc != HPL_OK) return rc;
-                ReduceTask& d = w.tasks[w.n_tasks++];
-                d.out_ptr = (unsigned long long)(uintptr_t)out->ptr;
-                d.elems = op.elems;
-                d.chunk_elems = op.chunk_elems;
-                d.c_begin = t.a;
-                d.c_end = t.b;
-                d.tiles_per_chunk = tpc_full;
-                d.tile_begin = w.total_tiles;
-                d.step_begin = n_steps;
-                d.n_steps = (uint32_t)t.steps.size();
-                d.red_op = (uint32_t)op.red_op;
-                d.poll = t.poll ? 1u : 0u;
-                if (t.poll) c->polling_in_flight = true;
-                claim_fused_receivers(c, op, t, (size_t)kMaxFusedDst - n_fan, fan);
-                d.fan_begin = n_fan;
-                d.n_fan = (uint32_t)fan.size();
-                for (unsigned long long p : fan) w.fan_ptrs[n_fan++] = p;
-                d.pad = 0;
-                for (size_t q = 0; q < t.steps.size(); ++q) {
-                    w.recs[n_steps + q] = pack_step(t.steps[q]);
-                    w.rows[n_steps + q] = t.steps[q].row;
-                }
-                n_steps += d.n_steps;
-                w.total_tiles += (t.b - t.a) * tpc_full;
-                n_acc = std::max(n_acc, t.n_acc);
-                // accounting: bytes the task moves
-                uint64_t e_lo = (uint64_t)t.a * op.chunk_elems, e_hi = std::min<uint64_t>((uint64_t)t.b * op.chunk_elems, op.elems);
-                for (auto& st : t.steps)
-                    if (st.code != OPC_ADD_ACC) c->stats.bytes_read_planned += (e_hi - e_lo) * (st.kind == SRC_BF16 ? 2 : 4);
-                c->stats.bytes_written_planned += (e_hi - e_lo) * 4 * (1 + fan.size());
-                c->stats.reduce_tasks++;
-                if (!fan.empty()) c->stats.fused_fanout_tasks++;
-                ++i;
-            }
-            if (w.n_tasks == 0) return HPL_ERR_INVALID;  // a single task larger than a wave: tree too wide
-            if (!c->device) {   // schedule-only context: the wave is planned and counted, not run
-                c->stats.kernel_launches++;
-                c->stats.reduce_launches++;
-                c->stats.tiles += w.total_tiles;
-                continue;
-            }
-            const bool fanned = n_fan != 0;
-            int& occ = c->occ_reduce[bf16 ? 1 : 0][fanned ? 1 : 0][occ_index(n_acc)];
-            if (occ == 0) occ = reduce_ctas_per_sm(n_acc, bf16, fanned);
-            int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
-            if (grid < 1) grid = 1;
-            if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
-            bool polls = false;
-            for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
-            if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counters it waits on are rows of the directory
-            w.status = next_wave_status(c);
-            {
-                LaunchTimer timer(c, 0);
-                if (launch_reduce_wave(w, n_acc, bf16, fanned, grid, c->stream) != 0) return HPL_ERR_CUDA;
-            }
-            c->stats.kernel_launches++;
-            c->stats.reduce_launches++;
-            c->stats.tiles += w.total_tiles;
-            c->stats.last_kernel_grid = (uint64_t)grid;
-            c->work_in_flight = true;
-        }
+            if (t.level == level) lv.push_back({&op, &t});
+        int rc = launch_reduce_group(c, lv, op.in_dtype == HPL_BF16);
+        if (rc != HPL_OK) return rc;
     }
     return HPL_OK;
 }

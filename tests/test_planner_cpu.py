@@ -150,3 +150,38 @@ def test_allreduce_of_8_to_8_is_one_pass_that_never_reads_the_target():
         st = _plan_get(c, 200)
         assert st["kernel_launches"] == 1 and st["reduce_launches"] == 1 and st["fanout_launches"] == 0
         assert st["bytes_read_planned"] == k * S and st["bytes_written_planned"] == (R + 1) * S
+
+
+def test_small_collectives_planned_in_one_pass_share_their_launches():
+    """Objects under 64 KiB (Section 3.2's small objects): 32 Reduces and 8 broadcasts requested together are served by
+    a few shared waves instead of one launch each; a Reduce that consumes another's output sits one stage later."""
+    S = 4096
+    with hpl.Context(64 << 10, 2, 2) as c:
+        oid = 0
+        for r in range(32):
+            ids = list(range(oid, oid + 4))
+            oid += 4
+            for i in ids:
+                c.create(i, i, S)
+                c.put(i, _addr(i), S)
+            c.reduce(10_000 + r, ids, 4)
+        c.reduce(20_000, [10_000, 10_001], 2)              # composed: one stage behind its producers
+        for b in range(8):
+            c.create(30_000 + b, 900, S)
+            c.put(30_000 + b, _addr(7), S)
+            c.create(31_000 + b, 901 + b, S)
+            c.broadcast(30_000 + b, [31_000 + b])
+            c.join(31_000 + b, _addr(9))
+        c.progress()
+        st = c.stats()
+        assert st["reduce_tasks"] == 33 and st["fanout_tasks"] == 8
+        assert st["reduce_launches"] == 3 and st["fanout_launches"] == 1     # 24 + 8 tasks, then the composed one; 8 fan-outs
+    with hpl.Context(64 << 10, 2, 2) as c:                 # objects above the threshold keep launches of their own
+        for r in range(3):
+            ids = list(range(4 * r, 4 * r + 4))
+            for i in ids:
+                c.create(i, i, 128 << 10)
+                c.put(i, _addr(i), 128 << 10)
+            c.reduce(10_000 + r, ids, 4)
+        c.progress()
+        assert c.stats()["reduce_launches"] == 3
