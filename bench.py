@@ -137,6 +137,8 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
         out["reduce"] = (w.k - 1) * S + w.elems * 4          # the survivors and the result
     if w.kind in ("broadcast", "round"):
         out["broadcast"] = S + w.n_receivers * S
+    if w.kind == "multi_reduce":
+        out["reduce"] = w.extra["collectives"] * (w.k * S + w.elems * 4)
     if w.kind == "allreduce":
         # reduce followed by broadcast of its output: the sources read once, the result written once to the target
         # and once to every receiver (reading the target back is not part of what the method must move)
@@ -159,7 +161,7 @@ class Runner:
         S = w.object_bytes
         self.host_buffers = host_buffers
         self.ft_eager = ft_eager
-        n_src = w.n_objects
+        n_src = w.n_objects * w.extra.get("collectives", 1)
         arena_bytes = 64 * MiB + 2 * w.elems * 4 + (n_src + 2) * S * (1 if host_buffers else 0)
         if w.kind == "ft_reduce":
             arena_bytes += 8 * w.elems * 4       # partial results of the subtrees beside the failing worker's root path
@@ -213,6 +215,29 @@ class Runner:
         S = w.object_bytes
         t = (r + 1) * 2_000_000_000
         n, R = w.n_objects, w.n_receivers
+        if w.kind == "multi_reduce":
+            # many small collectives requested together: their tasks share waves and the Gets wait once
+            m = w.extra["collectives"]
+            e2, dl = H.EventList(8 + m * (2 * n + 2)), H.EventList(4 + m * (n + 1))
+            if marks:
+                e2.add(H.HPL_EV_MARK, 0, ptr=marks[0])
+                e2.add(H.HPL_EV_MARK, 0, ptr=marks[1])
+            for q in range(m):
+                ids = list(range(q * n, (q + 1) * n))
+                for i in ids:
+                    e2.add(H.HPL_EV_CREATE, t, i, i, nbytes=w.object_bytes, dtype=self.dt)
+                    e2.add(H.HPL_EV_PUT, t, i, ptr=self.src[i].data_ptr(), nbytes=w.object_bytes)
+            for q in range(m):
+                e2.add(H.HPL_EV_REDUCE, t, 100_000 + q, ids=list(range(q * n, (q + 1) * n)), k=w.k, op=H.HPL_SUM, dtype=self.dt)
+            for q in range(m):
+                e2.add(H.HPL_EV_GET, 0, 100_000 + q)
+            for q in range(m):
+                dl.add(H.HPL_EV_DELETE, 0, 100_000 + q)
+                for i in range(q * n, (q + 1) * n):
+                    dl.add(H.HPL_EV_DELETE, 0, i)
+            if marks:
+                e2.add(H.HPL_EV_MARK, 0, ptr=marks[2])
+            return H.EventList(1), e2, dl, 0, 0
         e1, e2, dl = H.EventList(12 + 3 * R + n), H.EventList(12 + 3 * n + 3 * R), H.EventList(4 + n)
         h2d = d2h = 0
         put_kind = H.HPL_EV_PUT_HOST if self.host_buffers else H.HPL_EV_PUT
@@ -615,6 +640,18 @@ def size_sweep(device, peak: float):
         rr.close()
         del rr
         torch.cuda.empty_cache()
+        if size <= (64 << 10):
+            # small objects: 32 Reduces of 8 objects each requested together (shared waves, one wait)
+            mw = wl.Workload("reduce_x32", "multi_reduce", "f32", ("uniform",), size // 4, size, 2, n_objects=8, k=8,
+                             extra={"collectives": 32})
+            rr = Runner(mw, device)
+            m = measure_point(rr, n, 3, peak, k_steps=min(n, 5))
+            row["reduce_8_objects_x32_together"] = {"GBps": m["GBps"], "ms_per_step": m["ms_per_step"],
+                                                    "us_per_collective": m["ms_per_step"] * 1e3 / 32,
+                                                    "launches_per_step": m["launches_per_step"]}
+            rr.close()
+            del rr
+            torch.cuda.empty_cache()
         bw = wl.Workload("bcast16", "broadcast", "f32", ("uniform",), size // 4, min(1 << 20, size), 2, n_receivers=16,
                          extra={"join_window_ns": 1_000_000})
         rr = Runner(bw, device)

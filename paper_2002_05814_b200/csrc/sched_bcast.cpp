@@ -28,7 +28,46 @@ void BroadcastTreeSchedule::release(std::vector<int>& v, int x) {
     if (it != v.end()) v.erase(it);
 }
 
+// Chunks a receiver holds at time t in the closed form: those with b + (c + 1) tau <= t.
+int64_t BroadcastTreeSchedule::held_at(const BcastLocation& l, int64_t t) const {
+    if (l.complete) return C_;
+    if (t <= l.b) return 0;
+    return std::min<int64_t>(C_, (t - l.b) / tau_);
+}
+
+// Leaves the closed form: writes down, for the current time, what every receiver holds and which chunk is on
+// its way, exactly as the event simulation would have it, and goes on chunk by chunk.
+void BroadcastTreeSchedule::to_events() {
+    if (!closed_form_) return;
+    closed_form_ = false;
+    for (size_t i = 1; i < locs_.size(); ++i)
+        if (locs_[i].alive && !locs_[i].complete) locs_[i].have = held_at(locs_[i], now_);
+    for (size_t i = 1; i < locs_.size(); ++i) {
+        BcastLocation& r = locs_[i];
+        if (!r.alive || r.complete || r.sender < 0) continue;
+        if (locs_[r.sender].have > r.have) {   // its next chunk is on its way
+            r.landing = r.b + (r.have + 1) * tau_;
+            r.token = ++next_token_;
+            heap_.push(Landing{r.landing, (int)i, r.token});
+        }
+    }
+    while (!completions_.empty()) completions_.pop();
+}
+
+void BroadcastTreeSchedule::complete_location(int ri, int64_t t) {
+    locs_[ri].have = C_;
+    locs_[ri].complete = true;
+    locs_[ri].t_complete = t;
+    const int s = locs_[ri].sender;
+    if (s >= 0) {
+        release(locs_[s].receivers, ri);
+        if (locs_[s].alive) locs_[s].slots += 1;
+    }
+    locs_[ri].sender = -1;
+}
+
 void BroadcastTreeSchedule::source_progress(int64_t t, int64_t have) {
+    if (closed_form_ && locs_.size() > 1 && have < C_) to_events();   // (cannot happen: receivers only join a complete source here)
     advance(t);
     BcastLocation& s = locs_[0];
     s.have = std::max(s.have, have);
@@ -40,6 +79,15 @@ void BroadcastTreeSchedule::source_progress(int64_t t, int64_t have) {
 }
 
 void BroadcastTreeSchedule::advance(int64_t t) {
+    if (closed_form_) {
+        while (!completions_.empty() && completions_.top().first <= t) {
+            const Completion cmp = completions_.top();
+            completions_.pop();
+            complete_location(cmp.second, cmp.first);   // nobody waits in the closed form: a freed slot is just a count
+        }
+        now_ = std::max(now_, t);
+        return;
+    }
     while (!heap_.empty() && heap_.top().t <= t) {
         const Landing l = heap_.top();
         heap_.pop();
@@ -64,14 +112,7 @@ void BroadcastTreeSchedule::land(int ri, int64_t t) {
     locs_[ri].landing = -1;
     locs_[ri].have += 1;
     if (locs_[ri].have >= C_) {
-        locs_[ri].complete = true;
-        locs_[ri].t_complete = t;
-        const int s = locs_[ri].sender;
-        if (s >= 0) {
-            release(locs_[s].receivers, ri);
-            if (locs_[s].alive) locs_[s].slots += 1;
-        }
-        locs_[ri].sender = -1;
+        complete_location(ri, t);
         serve_waiting(t);
     } else {
         try_start(ri, t);
@@ -126,6 +167,7 @@ void BroadcastTreeSchedule::serve_waiting(int64_t t) {
 }
 
 void BroadcastTreeSchedule::join(int64_t t, int64_t dst_obj) {
+    if (closed_form_ && !locs_[0].complete) to_events();   // a source that is still being put: chunk by chunk
     advance(t);
     {
         auto it = index_.find(dst_obj);
@@ -140,6 +182,19 @@ void BroadcastTreeSchedule::join(int64_t t, int64_t dst_obj) {
     locs_.push_back(r);
     index_[dst_obj] = ri;
     const int s = choose(ri);
+    if (closed_form_ && s >= 0) {
+        // evenly spaced landings: chunk c at b + (c + 1) tau, complete at b + C tau
+        BcastLocation& r = locs_[ri];
+        r.first_sender_obj = locs_[s].obj;
+        locs_[s].slots -= 1;
+        locs_[s].receivers.push_back(ri);
+        r.sender = r.last_sender = s;
+        r.start_chunk = 0;
+        r.b = (s == 0 || locs_[s].complete) ? t : std::max(locs_[s].b + tau_, t);
+        completions_.push(Completion(r.b + C_ * tau_, ri));
+        return;
+    }
+    to_events();   // a receiver that has to wait: chunk by chunk from here on
     if (s < 0) {
         waiting_.push_back(ri);
     } else {
@@ -151,6 +206,7 @@ void BroadcastTreeSchedule::join(int64_t t, int64_t dst_obj) {
 
 void BroadcastTreeSchedule::fail(int64_t t, const std::vector<int64_t>& objs) {
     advance(t);
+    to_events();
     std::vector<int> gone;
     for (int64_t o : objs) {
         const int i = index_of(o);
@@ -202,6 +258,10 @@ void BroadcastTreeSchedule::fail(int64_t t, const std::vector<int64_t>& objs) {
 bool BroadcastTreeSchedule::run_until_complete(int64_t obj) {
     const int i = index_of(obj);
     if (i < 0) return false;
+    if (closed_form_) {
+        if (!locs_[i].complete && locs_[i].alive) advance(locs_[i].b + C_ * tau_);
+        return locs_[i].complete;
+    }
     while (!locs_[i].complete && !heap_.empty()) advance(heap_.top().t);
     return locs_[i].complete;
 }
@@ -212,7 +272,7 @@ void BroadcastTreeSchedule::dump(std::vector<int64_t>& w) const {
     for (size_t i = 1; i < locs_.size(); ++i) {
         const BcastLocation& r = locs_[i];
         w.insert(w.end(), {r.obj, r.first_sender_obj, r.sender >= 0 ? locs_[r.sender].obj : -1, r.start_chunk, r.t_join,
-                           r.have, r.alive ? 1 : 0, r.t_complete});
+                           closed_form_ ? held_at(r, now_) : r.have, r.alive ? 1 : 0, r.t_complete});
     }
     w.push_back((int64_t)edits_.size());
     for (auto& e : edits_) w.insert(w.end(), e.begin(), e.end());

@@ -8,6 +8,14 @@
 // as its sender holds it.  When a location fails, the receivers it was sending to ask again
 // (candidates that fetch, directly or not, from the asker are not eligible) and resume from
 // the chunks they hold.
+//
+// Two engines compute the same virtual-time model.  While the source was complete before the first
+// receiver joined and nothing has failed or had to wait, every receiver's chunks land at evenly spaced
+// times, L_r(c) = b_r + (c + 1) tau with b_r = max(b_sender + tau, t_join) (by induction over
+// avail_r(c) = max(avail_sender(c), avail_r(c - 1), t_join) + tau): only the completions are events, and
+// the chunks held at a time follow from b_r.  Anything else -- a source that is still being put, a
+// failure, a receiver without a sender -- first turns that state into the per-chunk event simulation
+// (chunks held, transfer in flight) and continues there.
 #pragma once
 #include <cstdint>
 #include <queue>
@@ -31,6 +39,7 @@ struct BcastLocation {
     int64_t t_join = -1, t_complete = -1;
     int64_t landing = -1;      // time the chunk in flight lands, -1 none
     uint64_t token = 0;        // identifies the transfer in flight
+    int64_t b = 0;             // closed form: chunk c lands at b + (c + 1) tau
     std::vector<int> receivers;
 };
 
@@ -65,6 +74,9 @@ private:
     void attach(int r, int s, int64_t t);
     void serve_waiting(int64_t t);
     void release(std::vector<int>& v, int x);
+    void complete_location(int r, int64_t t);
+    int64_t held_at(const BcastLocation& l, int64_t t) const;
+    void to_events();
 
     int64_t src_, C_, tau_, now_ = 0, epoch_ = 0;
     int d_;
@@ -74,6 +86,9 @@ private:
     std::vector<int> waiting_;
     std::vector<std::vector<int64_t>> edits_;
     std::priority_queue<Landing, std::vector<Landing>, std::greater<Landing>> heap_;
+    bool closed_form_ = true;                            // evenly spaced landings: only completions are events
+    typedef std::pair<int64_t, int> Completion;          // (time, location)
+    std::priority_queue<Completion, std::vector<Completion>, std::greater<Completion>> completions_;
 };
 
 }  // namespace hpl

@@ -152,7 +152,7 @@ def test_reduce_schedules_match_on_random_timelines(block):
         _reduce_timeline(seed)
 
 
-def _bcast_timeline(seed):
+def _bcast_timeline(seed, complete_source=False):
     rng = np.random.default_rng(seed)
     R = int(rng.integers(1, 14))
     d = int(rng.integers(1, 4))
@@ -165,8 +165,8 @@ def _bcast_timeline(seed):
         p.create(j, int(rng.integers(0, n_workers)), nbytes)
     t = 0
     src_pref = 0
-    if rng.random() < 0.5:
-        src_pref = nbytes if rng.random() < 0.6 else int(rng.integers(0, nbytes // 64 + 1)) * 64
+    if rng.random() < 0.5 or complete_source:
+        src_pref = nbytes if (rng.random() < 0.6 or complete_source) else int(rng.integers(0, nbytes // 64 + 1)) * 64
         if src_pref:
             p.put(0, src_pref)
     p.both("broadcast", 0, list(range(1, R + 1)))
@@ -205,6 +205,14 @@ def _bcast_timeline(seed):
 def test_broadcast_schedules_match_on_random_timelines(block):
     for seed in range(block * 150, (block + 1) * 150):
         _bcast_timeline(seed)
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_broadcasts_of_a_complete_source_match_through_failures(block):
+    """The library computes these in closed form (evenly spaced landings) until something fails or waits, then goes
+    on chunk by chunk; the oracle simulates every chunk throughout."""
+    for seed in range(10_000 + block * 150, 10_000 + (block + 1) * 150):
+        _bcast_timeline(seed, complete_source=True)
 
 
 def _composed_timeline(seed):
