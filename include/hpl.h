@@ -82,6 +82,9 @@ typedef struct hpl_config {
                                  from the reduce pass -- the output is written once to the target and once to each of
                                  them and is not read again; 0: the broadcast always reads the target */
     int32_t  reserved;
+    uint64_t debug_guard_bytes;   /* testing aid, 0 = off: every block the library takes from the arena is followed by this
+                                 many bytes of a canary pattern that no kernel may touch; checked when a block is
+                                 released and by hpl_check_guards */
 } hpl_config;
 
 /* Creates a context.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Nothing is
@@ -104,7 +107,11 @@ int hpl_create(hpl_ctx* ctx, int64_t object_id, int32_t worker, uint64_t total_b
  * the object's arrival (Section 3.2: the directory is told when Put is called, before the copy is done);
  * later calls extend the prefix (same `buf`, larger `bytes`); bytes == total marks it complete.  The store
  * borrows `buf`: the caller must not modify published bytes, nor free it before hpl_delete.  The bytes must
- * have been written by work enqueued earlier on the context's stream (or be visible before the call). */
+ * have been written by work enqueued earlier on the context's stream (or be visible before the call).
+ * With plan_ahead = 1 the rule is stricter: the prefix must be VISIBLE AT THE CALL (written and waited for, or
+ * produced on a stream the caller has synchronised).  The counter then goes out at once on a side stream, and a
+ * polling wave that is already running on the context's stream consumes the bytes as soon as it sees it -- it
+ * cannot be ordered behind producer work that sits after it on that stream. */
 int hpl_put(hpl_ctx* ctx, int64_t object_id, const void* buf, uint64_t bytes);
 
 /* Put (Table 1) with a HOST buffer: the store copies the prefix into its own device memory chunk by chunk,
@@ -210,8 +217,8 @@ int hpl_get_host(hpl_ctx* ctx, int64_t object_id, void* dst, uint64_t cap);
  * receivers it was sending to ask again and resume from what they hold. */
 int hpl_fail(hpl_ctx* ctx, int32_t worker);
 
-/* The task framework has reconstructed failed worker `worker` (Section 3.5: "we want to allow a recovered
- * task to rejoin"): the objects it owns are futures again -- not arrived, empty, to be Put again -- and the
+/* The task framework has reconstructed failed worker `worker` (Section 3.5 lets a rebuilt task take part
+ * again): the objects it owns are futures again -- not arrived, empty, to be Put again -- and the
  * receivers it owns may hpl_join again (a new location).  A Reduce counts a re-Put source as a new arrival:
  * it takes an open position or waits as a spare; a tree that shrank does not grow back.  A broadcast whose
  * SOURCE was lost is not revived.  Waits for enqueued work (directory rows are recycled). */
@@ -270,6 +277,11 @@ typedef struct hpl_stats_t {
 } hpl_stats_t;
 
 int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);
+
+/* With debug_guard_bytes set: waits for the device, checks the canary behind every live arena block and returns in
+ * *violations the number of canary bytes found changed so far (including those of blocks released earlier).
+ * Without it: 0. */
+int hpl_check_guards(hpl_ctx* ctx, uint64_t* violations);
 
 const char* hpl_strerror(int code);
 

@@ -227,6 +227,9 @@ struct hpl_ctx {
     uint64_t now = 0, tau = 1, seq = 0;
     int64_t next_internal = -1;  // ids of partial buffers: negative, never visible outside
     hpl::Arena arena;
+    uint64_t guard_bytes = 0;                                  // testing aid: canary after every arena block
+    std::map<void*, std::pair<uint64_t, uint64_t>> guards;     // block -> (offset of its canary, length)
+    uint64_t guard_violations = 0;
     DirRow* d_dir = nullptr;
     DirRow* h_dir = nullptr;
     DeviceStatus* d_status = nullptr;
@@ -297,6 +300,9 @@ DeviceStatus* next_wave_status(hpl_ctx* c);
 cudaEvent_t take_event(hpl_ctx* c);
 void collect_kernel_times(hpl_ctx* c);
 void release_object_memory(hpl_ctx* c, Object& o);
+void* arena_alloc(hpl_ctx* c, uint64_t n);
+void arena_release(hpl_ctx* c, void* p);
+uint64_t check_guard(hpl_ctx* c, void* block);
 
 // plan_reduce.cpp
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);

@@ -157,8 +157,47 @@ void collect_kernel_times(hpl_ctx* c) {   // call only after the stream has been
     c->timed.clear();
 }
 
+// Arena blocks.  With debug_guard_bytes set (a testing aid: compute-sanitizer is not always available) every
+// block is followed by a canary the library never writes; it is checked when the block is released and by
+// hpl_check_guards, so that a kernel that runs past a target, a partial result or a store copy is noticed.
+constexpr int kGuardPattern = 0xC5;
+
+void* arena_alloc(hpl_ctx* c, uint64_t n) {
+    if (!c->guard_bytes || !c->device) return c->arena.alloc(n);
+    const uint64_t body = (n + kAlign - 1) / kAlign * kAlign;
+    uint8_t* p = (uint8_t*)c->arena.alloc(body + c->guard_bytes);
+    if (!p) return nullptr;
+    // from the first byte behind the object (the padding up to the block's alignment is canary too)
+    if (cudaMemsetAsync(p + n, kGuardPattern, body - n + c->guard_bytes, c->stream) != cudaSuccess) {
+        c->arena.release(p);
+        return nullptr;
+    }
+    c->guards[p] = {n, body - n + c->guard_bytes};
+    return p;
+}
+
+// Bytes of the block's canary that no longer hold the pattern (waits for the device).
+uint64_t check_guard(hpl_ctx* c, void* block) {
+    auto g = c->guards.find(block);
+    if (g == c->guards.end()) return 0;
+    std::vector<uint8_t> host(g->second.second);
+    cudaStreamSynchronize(c->stream);
+    if (cudaMemcpy(host.data(), (uint8_t*)block + g->second.first, host.size(), cudaMemcpyDeviceToHost) != cudaSuccess) return 1;
+    uint64_t bad = 0;
+    for (uint8_t b : host) bad += b != kGuardPattern;
+    return bad;
+}
+
+void arena_release(hpl_ctx* c, void* p) {
+    if (c->guard_bytes && c->device) {
+        c->guard_violations += check_guard(c, p);
+        c->guards.erase(p);
+    }
+    c->arena.release(p);
+}
+
 void release_object_memory(hpl_ctx* c, Object& o) {
-    if (o.lib_owned && o.ptr) c->arena.release(o.ptr);
+    if (o.lib_owned && o.ptr) arena_release(c, o.ptr);
     o.ptr = nullptr;
     if (o.row >= 0) c->free_rows.push_back(o.row);
     o.row = -1;

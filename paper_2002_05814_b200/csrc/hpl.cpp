@@ -321,6 +321,7 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
             delete c;
             return HPL_ERR_CUDA;
         }
+        c->guard_bytes = (cfg->debug_guard_bytes + kAlign - 1) / kAlign * kAlign;
         for (uint32_t i = 0; i <= kMaxChunks; ++i) c->h_iota[i] = i;
         for (int r = (int)kMaxRows - 1; r >= 0; --r) c->free_rows.push_back(r);
         c->device = true;
@@ -442,14 +443,14 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
     const bool first = !o->arrived;
     if (!first && !o->from_host) return HPL_ERR_INVALID;
     if (first) {
-        o->ptr = c->arena.alloc(o->bytes);
+        o->ptr = arena_alloc(c, o->bytes);
         if (!o->ptr) return HPL_ERR_NOMEM;
         o->lib_owned = true;
         o->from_host = true;
         o->async_counter = true;
         rc = alloc_row(c, *o);
         if (rc != HPL_OK) {
-            c->arena.release(o->ptr);
+            arena_release(c, o->ptr);
             o->ptr = nullptr;
             o->lib_owned = false;
             return rc;
@@ -519,11 +520,11 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     t.ready_bytes = 0;
     t.seq = c->seq++;
     {
-        t.ptr = c->arena.alloc(t.bytes);
+        t.ptr = arena_alloc(c, t.bytes);
         if (!t.ptr) return HPL_ERR_NOMEM;
         int rc = alloc_row(c, t);
         if (rc != HPL_OK) {
-            c->arena.release(t.ptr);
+            arena_release(c, t.ptr);
             return rc;
         }
     }
@@ -535,7 +536,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     if (degree == 0)   // Section 4: picked per Reduce from the latency / bandwidth model and the object size
         degree = choose_reduce_degree(k, (double)bytes, (double)c->cfg.model_latency_ns * 1e-9, (double)c->cfg.model_bandwidth_bps);
     if (std::min<int64_t>(degree, k - 1) + 2 > (int64_t)kMaxStepsPerWave) {   // one node's operands must fit one task
-        if (t.ptr) c->arena.release(t.ptr);
+        if (t.ptr) arena_release(c, t.ptr);
         if (t.row >= 0) c->free_rows.push_back(t.row);
         c->objects.erase(target);
         return HPL_ERR_INVALID;
@@ -921,6 +922,14 @@ int hpl_schedule_dump(hpl_ctx* c, int64_t op_id, int64_t* words, uint64_t cap, u
     *len = w.size();
     if (!words || cap < w.size()) return HPL_ERR_INVALID;
     std::memcpy(words, w.data(), w.size() * sizeof(int64_t));
+    return HPL_OK;
+}
+
+int hpl_check_guards(hpl_ctx* c, uint64_t* violations) {
+    if (!c || !violations) return HPL_ERR_INVALID;
+    if (c->device)
+        for (auto& g : c->guards) c->guard_violations += check_guard(c, g.first);
+    *violations = c->guard_violations;
     return HPL_OK;
 }
 

@@ -34,12 +34,12 @@ int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out) {
     o.C = op.C;
     o.lib_owned = true;
     o.seq = c->seq++;
-    o.ptr = c->arena.alloc(o.bytes);
+    o.ptr = arena_alloc(c, o.bytes);
     if (!o.ptr) return HPL_ERR_NOMEM;
     o.ready_bytes = o.bytes;
     int rc = alloc_row(c, o);
     if (rc != HPL_OK) {
-        c->arena.release(o.ptr);
+        arena_release(c, o.ptr);
         return rc;
     }
     op.partial_key[pos] = o.id;

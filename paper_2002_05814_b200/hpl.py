@@ -32,7 +32,7 @@ class Config(C.Structure):
                 ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
                 ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64),
-                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32)]
+                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32), ("debug_guard_bytes", C.c_uint64)]
 
 
 class Stats(C.Structure):
@@ -123,6 +123,7 @@ def load_library():
         "hpl_sync": [VP],
         "hpl_schedule_dump": [VP, I64, P(I64), U64, P(U64)],
         "hpl_stats": [VP, P(Stats)],
+        "hpl_check_guards": [VP, P(U64)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -155,11 +156,12 @@ class Context:
     def __init__(self, chunk_bytes: int, reduce_degree: int = 2, bcast_degree: int = 2, *, arena=0,
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
                  eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False,
-                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0, fuse_fanout: bool = True):
+                 model_latency_ns: int = 0, model_bandwidth_bps: int = 0, fuse_fanout: bool = True,
+                 debug_guard_bytes: int = 0):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
                      int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes,
-                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0)
+                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0, debug_guard_bytes)
         self._h = C.c_void_p()
         self._p, self._n = C.c_void_p(), C.c_uint64()
         self._pref, self._nref = C.byref(self._p), C.byref(self._n)
@@ -300,6 +302,12 @@ class Context:
         buf = (C.c_int64 * n.value)()
         self._check(self._lib.hpl_schedule_dump(self._h, op_id, buf, n.value, C.byref(n)), "hpl_schedule_dump")
         return list(buf)
+
+    def check_guards(self) -> int:
+        """``hpl_check_guards``: canary bytes behind arena blocks found changed so far (0 without debug_guard_bytes)."""
+        n = C.c_uint64()
+        self._check(self._lib.hpl_check_guards(self._h, C.byref(n)), "hpl_check_guards")
+        return n.value
 
     def stats(self) -> dict:
         st = Stats()

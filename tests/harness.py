@@ -20,6 +20,7 @@ class Pair:
     def __init__(self, chunk_bytes, d_reduce=2, d_bcast=2, tau=0, arena_bytes=256 << 20, **flags):
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device="cuda")
         self.stream = torch.cuda.current_stream().cuda_stream
+        flags.setdefault("debug_guard_bytes", 256)      # canaries behind every block the library takes from the arena
         self.c = hpl.Context(chunk_bytes, d_reduce, d_bcast, arena=self.arena.data_ptr(), arena_bytes=arena_bytes,
                              stream=self.stream, virt_chunk_ns=tau, **flags)
         self.o = OracleStore(chunk_bytes, d_reduce, d_bcast, tau, flags.get("model_latency_ns", 0), flags.get("model_bandwidth_bps", 0))
@@ -31,7 +32,9 @@ class Pair:
 
     def close(self):
         """Shuts the context down and checks what no test may violate: objects are immutable (the bytes of every
-        put object are unchanged) and nothing was written outside a receiver's buffer."""
+        put object are unchanged) and nothing was written outside a receiver's buffer or behind a block of the
+        library's arena (targets, partial results, store copies of host objects)."""
+        assert self.c.check_guards() == 0, "write behind an arena block"
         self.c.shutdown()
         torch.cuda.synchronize()
         for oid, a in self.host.items():

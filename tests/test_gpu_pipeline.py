@@ -84,7 +84,7 @@ def test_host_source_is_broadcast_while_it_is_copied_in():
 
 def test_polling_kernel_picks_up_chunks_published_while_it_runs():
     k, elems, chunk = 4, 16 * 4096, 16 << 10                 # 16 chunks of 4096 elements
-    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=5_000_000_000)
+    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=500_000_000)
     for i in range(k):
         p.create(i, i, gen(("uniform",), 72, i, elems))
     p.reduce(100, list(range(k)), k)
@@ -166,7 +166,7 @@ def test_delete_returns_memory_and_rows_for_the_next_round():
 
 
 def test_waits_are_counted():
-    p = Pair(16 << 10, 2, plan_ahead=True, poll_budget_ns=5_000_000_000)
+    p = Pair(16 << 10, 2, plan_ahead=True, poll_budget_ns=500_000_000)
     for i in range(2):
         p.create(i, i, gen(("uniform",), 76, i, 8 * 4096))
     p.reduce(100, [0, 1], 2)
@@ -206,3 +206,73 @@ def test_pageable_host_memory_and_get_host_of_every_kind_of_object():
         p.c.get_host(2, out.ctypes.data, 16)                         # destination too small
     assert ei.value.code == hpl.HPL_ERR_INVALID
     p.close()
+
+
+def test_many_device_puts_then_a_host_object_with_plan_ahead():
+    """The control stream is busy with the rows of many device objects when a host object is put: its row must reach
+    the directory with a zero counter (a snapshot taken at the Put), so that the polling wave never sees chunks that
+    have not landed."""
+    elems, chunk, k = 24 * 4096 + 9, 16 << 10, 41
+    for rnd in range(3):
+        p = Pair(chunk, 4, plan_ahead=True, poll_budget_ns=500_000_000, arena_bytes=64 << 20)
+        for i in range(k):
+            p.create(i, i, gen(("uniform",), 78 + rnd, i, elems))
+        p.reduce(100, list(range(k)), k)
+        for i in range(k - 1):
+            p.put(i)                                         # device objects: rows and counters on the control stream
+        host = torch.from_numpy(p.host[k - 1]).pin_memory()
+        p.c.put_host(k - 1, host.data_ptr(), host.numel() * 4)   # copied in chunk by chunk behind them
+        p.o.put(k - 1, p.host[k - 1], p.host[k - 1].nbytes)
+        p.progress()
+        p.check_target_bits(100)
+        assert p.c.stats()["device_timeouts"] == 0
+        p.close()
+
+
+def test_plan_ahead_put_publishes_what_is_visible_at_the_call():
+    """The documented contract of hpl_put with plan_ahead = 1: the prefix must be valid when the call is made.  A
+    producer that fills the object on another stream synchronises before each Put; the polling wave, launched before
+    any byte existed, then consumes each piece as its counter arrives."""
+    elems, chunk = 32 * 4096, 16 << 10
+    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=500_000_000)
+    src = gen(("uniform",), 79, 0, elems)
+    other = gen(("uniform",), 79, 1, elems)
+    p.create(1, 1, other)
+    p.put(1)
+    p.host[0] = src
+    buf = torch.zeros(elems, dtype=torch.float32, device="cuda")
+    p.dev[0] = buf
+    p.c.create(0, 0, elems * 4, DT_F32)
+    p.o.create(0, 0, elems * 4, DT_F32)
+    p.reduce(100, [0, 1], 2)
+    whole = torch.from_numpy(src).cuda()
+    side = torch.cuda.Stream()
+    p.c.put(0, buf.data_ptr(), 0)                            # published with nothing valid yet: the arrival
+    p.o.put(0, src, 0)
+    p.progress()                                             # the wave polls for chunk 0 of object 0
+    for step in (8, 20, 32):
+        with torch.cuda.stream(side):
+            buf[: step * 4096].copy_(whole[: step * 4096])
+        side.synchronize()                                   # visible at the call
+        p.c.put(0, buf.data_ptr(), step * chunk)
+        p.o.put(0, src, step * chunk)
+    p.check_target_bits(100)
+    assert p.c.stats()["device_timeouts"] == 0
+    p.close()
+
+
+def test_arena_canaries_notice_a_write_behind_a_block():
+    """The overrun detector of the test harness itself: the test (not a kernel) changes one byte behind a reduce target
+    inside the arena it owns; hpl_check_guards reports it."""
+    p = Pair(16 << 10, 2)
+    for i in range(2):
+        p.create(i, i, gen(("uniform",), 80, i, 1000))
+        p.put(i)
+    p.reduce(100, [0, 1], 2)
+    ptr, n = p.c.get(100)
+    assert p.c.check_guards() == 0
+    off = ptr - p.arena.data_ptr()
+    p.arena[off + n + 3] = 0x11
+    torch.cuda.synchronize()
+    assert p.c.check_guards() == 1
+    p.c.shutdown()
