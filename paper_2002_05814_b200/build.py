@@ -7,7 +7,8 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.path.join(HERE, "libhpl.so")
+DEBUG = os.environ.get("HPL_DEBUG_BOUNDS") == "1"      # the bounds-checking build, selected like in hpl.lib_path()
+LIB = os.path.join(HERE, "libhpl_debug.so" if DEBUG else "libhpl.so")
 SOURCES = ["hpl.cpp", "directory.cpp", "plan_reduce.cpp", "plan_bcast.cpp", "sched_reduce.cpp", "sched_bcast.cpp",
            "kernels.cu", "noalloc.cu"]
 HEADERS = ["context.h", "device_types.h", "sched_reduce.h", "sched_bcast.h", os.path.join("..", "..", "include", "hpl.h")]
@@ -27,6 +28,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-shared", "-Xcompiler", "-fPIC", "-std=c++17", "-O3", "-lineinfo",
            "-gencode", "arch=compute_100a,code=sm_100a", "-x", "cu"]
+    if DEBUG:
+        cmd += ["-DHPL_DEBUG_BOUNDS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, f) for f in SOURCES] + ["-o", LIB]

@@ -181,6 +181,7 @@ struct PlannedReduceTask {
     bool poll;
     std::vector<ReduceStep> steps;
     std::vector<unsigned long long> fan;   // buffers of broadcast receivers that take the result from this task (root tasks only)
+    std::vector<uint32_t> fan_rows;        // their directory rows
 };
 
 struct ReduceOp {
@@ -259,6 +260,12 @@ struct hpl_ctx {
 };
 
 namespace hpl {
+
+#ifdef HPL_DEBUG_BOUNDS
+constexpr bool kDebugBounds = true;    // kernels look every buffer up in the directory and record accesses outside it
+#else
+constexpr bool kDebugBounds = false;
+#endif
 
 #define CUDA_TRY(x)                                  \
     do {                                             \

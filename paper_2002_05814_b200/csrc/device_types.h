@@ -19,7 +19,7 @@ static_assert(sizeof(DirRow) == 32, "directory row layout");
 
 // Error record the kernels write when a bounded wait runs out.
 struct DeviceStatus {
-    unsigned int error;      // 0, or 1 = a wait on a progress counter expired
+    unsigned int error;      // 0, 1 = a wait on a progress counter expired, 2 = (bounds-checking build) an access outside its object
     unsigned int row;        // directory row that was waited for
     unsigned int chunk;      // chunk index that was waited for
     unsigned int abort;      // set together with error: other CTAs stop waiting
@@ -69,7 +69,7 @@ struct ReduceTask {
     uint32_t poll;                // 1: operands' progress counters must be polled before each chunk
     uint32_t fan_begin, n_fan;    // receivers of a broadcast of this result that take each tile straight from the
                                   // reduce (indices into ReduceWave::fan_ptrs); 0 = the result goes to out_ptr only
-    uint32_t pad;
+    uint32_t out_row;             // directory row of the result buffer (read by the bounds-checking build only)
 };
 
 constexpr int kMaxTasksPerWave = 24;
@@ -86,6 +86,7 @@ struct ReduceWave {
     unsigned long long recs[kMaxStepsPerWave];   // packed steps (pack_step)
     uint32_t rows[kMaxStepsPerWave];             // directory row of each load step's operand
     unsigned long long fan_ptrs[kMaxFusedDst];   // device addresses of receivers' buffers (fused reduce -> fan-out)
+    uint32_t fan_rows[kMaxFusedDst];             // their directory rows (bounds-checking build)
 };
 
 struct FanoutTask {
@@ -111,6 +112,7 @@ struct FanoutWave {
     uint32_t total_tiles;
     FanoutTask tasks[kMaxFanoutTasks];
     unsigned long long dst_ptrs[kMaxFanoutDst];   // device addresses of the receivers' buffers
+    uint32_t dst_rows[kMaxFanoutDst];             // their directory rows (bounds-checking build)
 };
 
 // Launchers (kernels.cu).  Return a cudaError_t as int.

@@ -189,6 +189,7 @@ int sync_and_check(hpl_ctx* c) {
     for (uint32_t i = 0; i < used; ++i) {
         c->stats.device_waits += c->h_status[i].waits;
         if (!c->h_status[i].error) continue;
+        if (c->h_status[i].error == 2) c->stats.bounds_errors++;   // (bounds-checking build) a tile was outside its object and was skipped
         failed = true;
         // the record in the last slot may stand for several waves: the earliest of them decides
         const uint64_t tag = c->wave_tag[i];

@@ -58,6 +58,22 @@ __device__ bool wait_chunk(const DirRow* dir, DeviceStatus* status, unsigned int
     return false;
 }
 
+#ifdef HPL_DEBUG_BOUNDS
+// Bounds-checking build: every buffer a tile touches is looked up in the device directory; the address the wave
+// carries must be the row's, and the bytes touched must lie inside the object.  A violation is recorded (error 2)
+// and the tile is skipped instead of being accessed.
+__device__ bool range_ok(const DirRow* dir, DeviceStatus* status, unsigned int row, unsigned long long ptr, unsigned long long lo,
+                         unsigned long long hi, unsigned int chunk) {
+    const DirRow r = dir[row];
+    if ((r.ptr & ((1ull << kRecShift) - 1)) == (ptr & ((1ull << kRecShift) - 1)) && lo <= hi && hi <= r.bytes) return true;
+    if (atomicCAS(&status->error, 0u, 2u) == 0u) {
+        status->row = row;
+        status->chunk = chunk;
+    }
+    return false;
+}
+#endif
+
 __device__ __forceinline__ float combine(float a, float b, unsigned int red_op) {
     if (red_op == 0) return __fadd_rn(a, b);
     if (red_op == 1) return (b < a) ? b : a;
@@ -399,6 +415,22 @@ __global__ void __launch_bounds__(kReduceThreads, StagesFor<A, FAN>::min_ctas) r
         }
 
         const unsigned int count = (unsigned int)(e1 - e0);
+#ifdef HPL_DEBUG_BOUNDS
+        if (task.out_row != 0xFFFFFFFFu) {   // (a task without directory rows of its own is not checked)
+            int ok = 1;
+            for (unsigned int i = t; i < task.n_steps; i += kReduceThreads) {
+                const unsigned long long rec = w.recs[task.step_begin + i];
+                const unsigned int m = rec_meta(rec);
+                if (meta_code(m) == OPC_ADD_ACC) continue;
+                const unsigned long long es = (BF16 && meta_is_bf16(m)) ? 2ull : 4ull;
+                ok &= range_ok(w.dir, w.status, w.rows[task.step_begin + i], s_rec[i], e0 * es, e1 * es, c) ? 1 : 0;
+            }
+            if (t == 0) ok &= range_ok(w.dir, w.status, task.out_row, task.out_ptr, e0 * 4ull, e1 * 4ull, c) ? 1 : 0;
+            for (unsigned int i = t; i < task.n_fan; i += kReduceThreads)
+                ok &= range_ok(w.dir, w.status, w.fan_rows[task.fan_begin + i], w.fan_ptrs[task.fan_begin + i], e0 * 4ull, e1 * 4ull, c) ? 1 : 0;
+            if (!__syncthreads_and(ok)) continue;
+        }
+#endif
         run_tile<A, BF16, FAN>(rec_base, stage_base, task, e0, count, t, w.fan_ptrs);
     }
     if constexpr (FAN) {
@@ -452,6 +484,15 @@ __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __gri
             if (!__syncthreads_and(ok)) break;
         }
 
+#ifdef HPL_DEBUG_BOUNDS
+        {
+            int ok = 1;
+            if (t == 0) ok = range_ok(w.dir, w.status, task.src_row, task.src_ptr, b0, b1, c) ? 1 : 0;
+            for (unsigned int i = t; i < task.n_dst; i += kFanoutThreads)
+                ok &= range_ok(w.dir, w.status, w.dst_rows[task.dst_begin + i], w.dst_ptrs[task.dst_begin + i], b0, b1, c) ? 1 : 0;
+            if (!__syncthreads_and(ok)) continue;
+        }
+#endif
         // the bulk copies that read this buffer two tiles ago must have finished reading it
         if (t < kFanoutIssuers) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
         __syncthreads();

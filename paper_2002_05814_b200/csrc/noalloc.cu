@@ -173,7 +173,7 @@ extern "C" int hpl_reduce_noalloc(const void* const* src_bufs, int32_t n, int32_
     t.red_op = (uint32_t)op;
     t.poll = 0;
     t.fan_begin = t.n_fan = 0;
-    t.pad = 0;
+    t.out_row = 0xFFFFFFFFu;   // the output has no directory row: the bounds-checking build leaves this task alone
     for (size_t i = 0; i < steps.size(); ++i) {
         w.recs[i] = pack_step(steps[i]);   // address 0: the kernel takes it from the row in the scratch array
         w.rows[i] = steps[i].row;

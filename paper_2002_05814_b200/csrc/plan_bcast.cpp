@@ -126,7 +126,11 @@ int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanou
             if (tt.poll) c->polling_in_flight = true;
             d.bytes = src->bytes;
             d.chunk_bytes = chunk_bytes;
-            for (int r : tt.dst) w.dst_ptrs[n_dst++] = (unsigned long long)(uintptr_t)find(c, locs[r].obj)->ptr;
+            for (int r : tt.dst) {
+                const Object* ro = find(c, locs[r].obj);
+                w.dst_rows[n_dst] = (uint32_t)ro->row;
+                w.dst_ptrs[n_dst++] = (unsigned long long)(uintptr_t)ro->ptr;
+            }
             w.total_tiles += (tt.b - tt.a) * tpc;
             const uint64_t b_lo = (uint64_t)tt.a * chunk_bytes, b_hi = std::min<uint64_t>((uint64_t)tt.b * chunk_bytes, src->bytes);
             c->stats.bytes_read_planned += b_hi - b_lo;
@@ -145,9 +149,10 @@ int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanou
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
         if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
-        bool polls = false;
+        bool polls = kDebugBounds;   // (the bounds-checking build reads the directory in every wave, and may record an error)
         for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
         if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counter it waits on is a row of the directory
+        if (kDebugBounds) c->polling_in_flight = true;
         w.status = next_wave_status(c);
         {
             LaunchTimer timer(c, 1);

@@ -192,6 +192,7 @@ static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, PlannedReduceTask& t
     std::vector<unsigned long long>& out = t.fan;
     const size_t room = kMaxFusedDst;
     out.clear();
+    t.fan_rows.clear();
     if (!c->cfg.fuse_fanout || t.pos != 0 || t.end != op.n_ops(0)) return;
     auto bi = c->bcast_of_src.find(op.target);
     if (bi == c->bcast_of_src.end()) return;
@@ -212,6 +213,7 @@ static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, PlannedReduceTask& t
         c->journal.b.push_back({b.src, (int)r, b.phys_have[r], c->batch_tag});
         b.phys_have[r] = b_b;
         out.push_back((unsigned long long)(uintptr_t)o->ptr);
+        t.fan_rows.push_back((uint32_t)o->row);
     }
 }
 
@@ -343,8 +345,11 @@ int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedRedu
             const std::vector<unsigned long long>& fan = t.fan;
             d.fan_begin = n_fan;
             d.n_fan = (uint32_t)fan.size();
-            for (unsigned long long p : fan) w.fan_ptrs[n_fan++] = p;
-            d.pad = 0;
+            for (size_t q = 0; q < fan.size(); ++q) {
+                w.fan_rows[n_fan] = t.fan_rows[q];
+                w.fan_ptrs[n_fan++] = fan[q];
+            }
+            d.out_row = (uint32_t)out->row;
             for (size_t q = 0; q < t.steps.size(); ++q) {
                 w.recs[n_steps + q] = pack_step(t.steps[q]);
                 w.rows[n_steps + q] = t.steps[q].row;
@@ -374,9 +379,10 @@ int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedRedu
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * occ);
         if (grid < 1) grid = 1;
         if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;   // rows of partial results created while planning
-        bool polls = false;
+        bool polls = kDebugBounds;   // (the bounds-checking build reads the directory in every wave, and may record an error)
         for (uint32_t q = 0; q < w.n_tasks; ++q) polls = polls || w.tasks[q].poll;
         if (polls && order_main_after_control(c) != HPL_OK) return HPL_ERR_CUDA;   // the counters it waits on are rows of the directory
+        if (kDebugBounds) c->polling_in_flight = true;
         w.status = next_wave_status(c);
         {
             LaunchTimer timer(c, 0);

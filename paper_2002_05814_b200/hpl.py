@@ -22,7 +22,9 @@ _LIB = None
 
 
 def lib_path() -> str:
-    return os.path.join(_HERE, "libhpl.so")
+    """The library this process uses: ``libhpl.so``, or with ``HPL_DEBUG_BOUNDS=1`` in the environment the
+    bounds-checking build ``libhpl_debug.so`` (same code, kernels check every tile against the directory)."""
+    return os.path.join(_HERE, "libhpl_debug.so" if os.environ.get("HPL_DEBUG_BOUNDS") == "1" else "libhpl.so")
 
 
 class Config(C.Structure):
@@ -41,7 +43,7 @@ class Stats(C.Structure):
                                           "bytes_read_planned", "bytes_written_planned", "device_timeouts",
                                           "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
                                           "reduce_launches", "fanout_launches", "reduce_kernel_ns",
-                                          "fanout_kernel_ns", "device_waits", "fused_fanout_tasks")]
+                                          "fanout_kernel_ns", "device_waits", "fused_fanout_tasks", "bounds_errors")]
 
 
 class Event(C.Structure):

@@ -35,6 +35,7 @@ class Pair:
         put object are unchanged) and nothing was written outside a receiver's buffer or behind a block of the
         library's arena (targets, partial results, store copies of host objects)."""
         assert self.c.check_guards() == 0, "write behind an arena block"
+        assert self.c.stats()["bounds_errors"] == 0, "a tile outside its object (bounds-checking build)"
         self.c.shutdown()
         torch.cuda.synchronize()
         for oid, a in self.host.items():
