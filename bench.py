@@ -165,9 +165,11 @@ class Runner:
         arena_bytes = 64 * MiB + 2 * w.elems * 4 + (n_src + 2) * S * (1 if host_buffers else 0)
         if w.kind == "ft_reduce":
             arena_bytes += 8 * w.elems * 4       # partial results of the subtrees beside the failing worker's root path
+        arena_bytes += w.extra.get("partials", 0) * w.elems * 4
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
         self.plan_ahead = plan_ahead
         self.fuse_fanout = fuse_fanout
+        self.ctx_flags = {}          # further context settings (degree sweep: fuse, the Eq. 1 model)
         self.ctx = None
         self.open_context(time_kernels=False)
         self.src = [wl.values_torch(w.dist, w.seed + i, i, 0, w.elems, w.dtype, device=device) for i in range(n_src)]
@@ -197,9 +199,9 @@ class Runner:
         torch, w = self.torch, self.w
         if self.ctx is not None:
             self.ctx.shutdown()
-        self.ctx = self.hpl.Context(w.chunk_bytes, w.degree, w.degree, arena=self.arena.data_ptr(), arena_bytes=self.arena.numel(),
+        self.ctx = self.hpl.Context(w.chunk_bytes, w.degree, max(1, w.degree), arena=self.arena.data_ptr(), arena_bytes=self.arena.numel(),
                                     stream=torch.cuda.current_stream().cuda_stream, time_kernels=time_kernels,
-                                    plan_ahead=self.plan_ahead, fuse_fanout=self.fuse_fanout)
+                                    plan_ahead=self.plan_ahead, fuse_fanout=self.fuse_fanout, **self.ctx_flags)
         self.prepared = {}
 
     def close(self):
@@ -664,6 +666,61 @@ def size_sweep(device, peak: float):
     return rows
 
 
+def degree_sweep(device, peak: float):
+    """Section 3.4.2 / Appendix B on one GPU: reduce time against the tree degree d in {1, 2, k}, for k in {8, 32} objects
+    of several sizes, (a) as the paper executes a tree -- every node writes its reduced object, one wave per tree level
+    (fuse = 0) -- and (b) with ready subtrees fused in registers (fuse = 1, where the degree only changes the
+    association order).  L and B of Eq. 1 are calibrated from the measurements themselves: L = time per tree level
+    (chain against star on the smallest objects), B = bytes per second of the largest fused pass; the degree Eq. 1
+    picks from them (reduce_degree = 0) is then run and compared with the best measured one."""
+    import torch
+    import paper_2002_05814_b200 as hpl
+    sizes = [64 << 10, 1 << 20, 16 << 20, 64 << 20]
+    rows, cal = [], {}
+    for k in (8, 32):
+        for size in sizes:
+            w = wl.Workload("degree", "reduce", "f32", ("uniform",), size // 4, min(4 * MiB, size), 2, n_objects=k, k=k,
+                            extra={"partials": k})
+            rr = Runner(w, device)
+            n = 20 if size <= (1 << 20) else 6
+            cell = {"k": k, "object_bytes": size}
+            for fuse in (0, 1):
+                for d in (1, 2, k):
+                    w.degree = d
+                    rr.ctx_flags = {"fuse": bool(fuse)}
+                    rr.open_context(time_kernels=False)
+                    r = time_steps(rr, n, 3)
+                    cell[f"fuse{fuse}_d{d}_ms"] = float(np.mean(r["total_ms"]))
+            rows.append((cell, rr, w, n))
+    # calibration: per-level latency from the smallest objects (k = 32: the chain has 31 levels, the star one), bandwidth
+    # from the largest fused pass
+    small = next(c for c, _, _, _ in rows if c["k"] == 32 and c["object_bytes"] == sizes[0])
+    big = next(c for c, _, _, _ in rows if c["k"] == 32 and c["object_bytes"] == sizes[-1])
+    L = max(1e-7, (small["fuse0_d1_ms"] - small["fuse0_d32_ms"]) * 1e-3 / 30.0)
+    B = (33 * sizes[-1]) / (big["fuse1_d2_ms"] * 1e-3)
+    out = []
+    for cell, rr, w, n in rows:
+        k, size = cell["k"], cell["object_bytes"]
+        w.degree = 0
+        rr.ctx_flags = {"fuse": False, "model_latency_ns": max(1, int(L * 1e9)), "model_bandwidth_bps": int(B)}
+        rr.open_context(time_kernels=False)
+        r = time_steps(rr, n, 3)
+        chosen = hpl.choose_degree(k, size, L, B)
+        best0 = min((1, 2, k), key=lambda d: cell[f"fuse0_d{d}_ms"])
+        cell.update({"eq1_degree": chosen, "eq1_degree_ms_fuse0": float(np.mean(r["total_ms"])), "best_degree_fuse0": best0,
+                     "best_ms_fuse0": cell[f"fuse0_d{best0}_ms"],
+                     "fuse1_spread": max(cell[f"fuse1_d{d}_ms"] for d in (1, 2, k)) / min(cell[f"fuse1_d{d}_ms"] for d in (1, 2, k))})
+        out.append(cell)
+        rr.close()
+    del rows
+    torch.cuda.empty_cache()
+    return {"L_s_per_level": L, "B_bytes_per_s": B, "cells": out,
+            "note": ("Eq. 1 models nodes with links of their own: a larger d costs d S / B at one node while the others work in "
+                     "parallel.  On one GPU every node shares the same HBM: a tree that writes every partial result moves "
+                     "(k + 2 (I - 1) + 1) S bytes for I internal nodes, so the star (d = k) is best whenever it fits, and the "
+                     "fused path makes the degree irrelevant (fuse1_spread is about 1).")}
+
+
 # ----------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -815,6 +872,9 @@ def main():
             "max_ms_per_step_up_to_4MiB": max(max(r["reduce_lazy"]["ms_per_step"], r["broadcast16"]["ms_per_step"])
                                               for r in rows if r["object_bytes"] <= (4 << 20)),
             "of": "measured copy bandwidth; reduce = fault-tolerant reduce of 32 objects planned at the Get"}
+
+    if rank == 0 and world == 1 and not args.no_sweep and args.shrink == 1:
+        line["degree_sweep"] = degree_sweep(device, peak)
 
     if rank == 0 and world == 1 and not args.no_realtime and args.shrink == 1:
         line["realtime"] = realtime_rounds(device)
