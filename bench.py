@@ -666,6 +666,128 @@ def size_sweep(device, peak: float):
     return rows
 
 
+def worker_per_gpu_round(dist, device, rank: int, world: int, steps: int = 5):
+    """The paper's own setting on N GPUs of one node: worker = rank, one 64 MiB fp32 object per GPU, a Reduce of all of
+    them through a binary tree whose edges cross NVLink (every node's result materialised on its own GPU, remote
+    operands pulled from peer memory; levels separated by a barrier).  Reported beside the replicas headline; every
+    rank takes part in every collective step even after a local error, so a refused peer mapping ends the round with a
+    message instead of a hang."""
+    import torch
+    import paper_2002_05814_b200 as hpl
+
+    state = {"ok": True, "err": ""}
+
+    def fail(e):
+        state["ok"] = False
+        state["err"] = state["err"] or repr(e)
+
+    def agree():
+        """All ranks learn whether all are still fine (doubles as the barrier between levels)."""
+        t = torch.tensor([1 if state["ok"] else 0], device=device, dtype=torch.int32)
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        return bool(t.item())
+
+    S = 64 * MiB
+    arena_bytes = 64 * MiB + 4 * S
+    ctx, mapped = None, []
+    out = {"objects": world, "object_bytes": S, "degree": 2}
+    try:
+        arena = torch.empty(arena_bytes, dtype=torch.uint8, device=device)
+        obj = wl.values_torch(("uniform",), wl.BASE_SEED + rank, rank, 0, S // 4, "f32", device=device)
+        mine = (hpl.ipc_export(arena.data_ptr()), hpl.ipc_export(obj.data_ptr()))
+    except Exception as e:      # noqa: BLE001
+        fail(e)
+        mine = None
+    handles = [None] * world
+    dist.all_gather_object(handles, mine)
+    peer_arena, peer_obj = {}, {}
+    if agree():
+        try:
+            for r in range(world):
+                if r == rank:
+                    peer_arena[r], peer_obj[r] = arena.data_ptr(), obj.data_ptr()
+                else:
+                    (ha, oa), (ho, oo) = handles[r]
+                    peer_arena[r] = hpl.ipc_import(ha, oa)
+                    peer_obj[r] = hpl.ipc_import(ho, oo)
+                    mapped += [peer_arena[r], peer_obj[r]]
+            ctx = hpl.Context(4 * MiB, 2, 2, arena=arena.data_ptr(), arena_bytes=arena_bytes,
+                              stream=torch.cuda.current_stream().cuda_stream, fuse=False, rank=rank, world_size=world)
+            for r in range(world):
+                if r != rank:
+                    ctx.set_peer_arena(r, peer_arena[r])
+        except Exception as e:  # noqa: BLE001
+            fail(e)
+    times = []
+    if agree():
+        t = 0
+        for step in range(steps + 2):
+            dist.barrier()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            try:
+                t += 1_000_000_000
+                ctx.advance(t)
+                ids = list(range(world))
+                ctx.create_batch(ids, ids, S)
+                ctx.put_batch(ids, [peer_obj[r] for r in ids], S)
+                ctx.reduce(1000, ids, world)
+            except Exception as e:  # noqa: BLE001
+                fail(e)
+            while True:                       # Context.drive, with `agree` as the barrier and a way out after an error
+                n = 0
+                try:
+                    if state["ok"]:
+                        ctx.progress()
+                        n = ctx.pending_levels()
+                except Exception as e:  # noqa: BLE001
+                    fail(e)
+                if not agree() or n == 0:
+                    break
+                for _ in range(n):
+                    try:
+                        if state["ok"]:
+                            ctx.run_level()
+                            ctx.sync()
+                    except Exception as e:  # noqa: BLE001
+                        fail(e)
+                    if not agree():
+                        break
+                if not state["ok"]:
+                    break
+            if not agree():
+                break
+            torch.cuda.synchronize()
+            dt = (time.perf_counter() - t0) * 1e3
+            if step >= 2:
+                times.append(max_over_ranks([dt], dist, device)[0])
+            try:
+                ctx.get(1000)
+                for i in [1000] + ids:
+                    ctx.delete(i)
+            except Exception as e:  # noqa: BLE001
+                fail(e)
+    agree()
+    try:
+        if ctx is not None:
+            ctx.shutdown()
+        dist.barrier()
+        for p in mapped:
+            hpl.ipc_close(p)
+    except Exception as e:      # noqa: BLE001
+        fail(e)
+    errs = [None] * world
+    dist.all_gather_object(errs, state["err"])
+    if any(errs):
+        out["error"] = next(e for e in errs if e)
+    if times:
+        ms = float(np.mean(times))
+        out.update({"ms_per_reduce": ms, "GBps_algorithmic": gbs((world + 1) * S, ms),
+                    "how": "wall clock from the Puts to the last level's barrier, maximum over ranks; levels = tree height, "
+                           "one NCCL all-reduce of a flag between levels"})
+    return out
+
+
 def degree_sweep(device, peak: float):
     """Section 3.4.2 / Appendix B on one GPU: reduce time against the tree degree d in {1, 2, k}, for k in {8, 32} objects
     of several sizes, (a) as the paper executes a tree -- every node writes its reduced object, one wave per tree level
@@ -738,6 +860,9 @@ def main():
     ap.add_argument("--no-sweep", action="store_true",
                     help="skip GB/s against object size: the fault-tolerant reduce (32 objects, both modes) and a "
                          "broadcast to 16 receivers, for 1 KiB ... 1 GiB in powers of 4")
+    ap.add_argument("--worker-per-gpu", action="store_true",
+                    help="with --gpus N > 1: also run a Reduce whose objects live one per GPU and whose tree edges cross NVLink "
+                         "(peer memory through CUDA IPC); off by default: this path has never run on more than one GPU")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--also", default="cfg2,cfg3", help="extra workloads reported under 'also' (cfg3 for its 50 rounds); 'none' skips them")
@@ -878,6 +1003,12 @@ def main():
 
     if rank == 0 and world == 1 and not args.no_realtime and args.shrink == 1:
         line["realtime"] = realtime_rounds(device)
+
+    if world > 1 and args.worker_per_gpu:
+        try:
+            line["worker_per_gpu"] = worker_per_gpu_round(dist, device, rank, world)
+        except Exception as e:  # noqa: BLE001
+            line["worker_per_gpu"] = {"error": repr(e)}
 
     if not args.no_e2e:
         e_steps = max(1, min(args.steps, 3))

@@ -85,6 +85,8 @@ typedef struct hpl_config {
     uint64_t debug_guard_bytes;   /* testing aid, 0 = off: every block the library takes from the arena is followed by this
                                  many bytes of a canary pattern that no kernel may touch; checked when a block is
                                  released and by hpl_check_guards */
+    int32_t  rank;            /* worker-per-GPU mode (below): this process' rank, 0 <= rank < world_size */
+    int32_t  world_size;      /* 0 or 1: everything lives on this GPU.  > 1: see "Worker-per-GPU mode" */
 } hpl_config;
 
 /* Creates a context.  `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Nothing is
@@ -286,6 +288,40 @@ int hpl_stats(hpl_ctx* ctx, hpl_stats_t* out);
 int hpl_check_guards(hpl_ctx* ctx, uint64_t* violations);
 
 const char* hpl_strerror(int code);
+
+/* ---- Worker-per-GPU mode (world_size > 1): the paper's own setting -- one process and one GPU per node, objects live
+ * where their worker runs, tree edges cross the interconnect (Sections 3.4 and 4; here NVLink peer memory).
+ *
+ * Every rank makes the SAME calls in the same order (the directory and the schedules are replicated; they are a pure
+ * function of the timeline), and every rank executes only the tasks whose output lives on its GPU:
+ *   - object `id` of worker w lives on rank w % world_size; a Reduce output lives on rank target_id % world_size; the
+ *     partial result of a tree node lives with the node's object;
+ *   - hpl_put / hpl_join take, on every rank, the address of the buffer IN THAT RANK'S address space: the owner its own
+ *     allocation, the others a peer mapping of it (CUDA IPC; hpl_ipc_export / hpl_ipc_import);
+ *   - every rank's arena has the same size and is peer-mapped by all others (hpl_set_peer_arena); allocation is
+ *     replicated, so each rank knows where a remote partial result sits without asking;
+ *   - a reduce task is run by the rank that owns its output and pulls remote operands over the link; a fan-out task is
+ *     run by the rank that holds the copy being read and pushes to its receivers (one sender, at most d receivers:
+ *     the tree edges of Section 3.4.1, followed strictly);
+ *   - kernels never wait on another GPU.  Work is released in LEVELS: hpl_progress only plans; hpl_pending_levels
+ *     says how many levels the plan has; hpl_run_level launches this rank's tasks of the next one.  Between two
+ *     levels the caller waits for its own stream (hpl_sync) and runs a barrier over the live ranks.  When no level is
+ *     left, hpl_progress is called again (receivers further down a broadcast tree are served by the next plan) until
+ *     it plans nothing.  hpl_get does not drive this loop: it returns HPL_ERR_TIMEOUT until the object is done.
+ * plan_ahead, eager and hpl_put_host are not available in this mode (HPL_ERR_INVALID).  A rank that is lost is taken
+ * out with hpl_fail_rank on every survivor: its workers fail (Section 3.5), and what lived on it is re-made
+ * elsewhere; a Reduce whose output lived there is lost (HPL_ERR_FAILED_WORKER). */
+int hpl_set_peer_arena(hpl_ctx* ctx, int32_t rank, void* arena_base /* DEVICE address, in this process, of that rank's arena */);
+int hpl_pending_levels(hpl_ctx* ctx, int32_t* levels);
+int hpl_run_level(hpl_ctx* ctx);
+int hpl_fail_rank(hpl_ctx* ctx, int32_t rank);
+/* Thin wrappers of CUDA IPC for the plumbing above.  Export: the 64-byte handle of the device ALLOCATION that holds
+ * dev_ptr and the offset of dev_ptr inside it (a pointer handed out by a caching allocator need not be the start of
+ * an allocation).  Import: maps another process' allocation and returns the address of the same byte in this
+ * process.  Close: unmaps what hpl_ipc_import returned (before the owner frees the memory). */
+int hpl_ipc_export(const void* dev_ptr, uint8_t handle[64], uint64_t* offset);
+int hpl_ipc_import(const uint8_t handle[64], uint64_t offset, void** dev_ptr);
+int hpl_ipc_close(void* dev_ptr);
 
 /* Reduce for callers that cannot allocate device memory.  The paper has no counterpart: this is an
  * addition for users of this library who run where cudaMalloc is off limits -- allocator callbacks,

@@ -5,7 +5,7 @@ is its thin ctypes binding.  Importing the package does not load the library; th
 does, and fails loudly if it has not been built (``python -m paper_2002_05814_b200.build``).
 """
 from .hpl import (  # noqa: F401
-    HplError, Context, Config, load_library, lib_path, reduce_noalloc, choose_degree,
+    HplError, Context, Config, load_library, lib_path, reduce_noalloc, choose_degree, ipc_export, ipc_import, ipc_close,
     HPL_F32, HPL_BF16, HPL_SUM, HPL_MIN, HPL_MAX,
     HPL_OK, HPL_ERR_INVALID, HPL_ERR_NOT_FOUND, HPL_ERR_EXISTS, HPL_ERR_TIMEOUT,
     HPL_ERR_INSUFFICIENT, HPL_ERR_FAILED_WORKER, HPL_ERR_CUDA, HPL_ERR_NOMEM,

@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd += ["-DHPL_DEBUG_BOUNDS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, f) for f in SOURCES] + ["-o", LIB]
+    cmd += [os.path.join(CSRC, f) for f in SOURCES] + ["-ldl", "-o", LIB]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

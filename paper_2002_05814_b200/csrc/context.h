@@ -161,6 +161,7 @@ struct Object {
     int64_t t_arrival = -1;
     uint64_t seq = 0;          // creation order
     int row = -1;
+    int home = 0;              // rank whose GPU holds the bytes (worker-per-GPU mode)
 };
 
 struct Journal {  // what was planned since the last successful wait (undone if a device wait expires)
@@ -194,6 +195,7 @@ struct ReduceOp {
     std::vector<IntervalMap> merged;        // per position: chunks -> leading operands merged into its buffer (valid ones only)
     int n_ops(int pos) const { return sched->n_children(pos) + 1; }
     std::vector<int64_t> partial_key;       // per position: internal object id of its partial buffer (0 none)
+    bool lost = false;                      // worker-per-GPU mode: the rank that held the output is gone
 };
 
 struct BcastOp {
@@ -227,7 +229,15 @@ struct hpl_ctx {
     int n_sm = 0;
     uint64_t now = 0, tau = 1, seq = 0;
     int64_t next_internal = -1;  // ids of partial buffers: negative, never visible outside
-    hpl::Arena arena;
+    hpl::Arena arena;                          // this rank's arena
+    int rank = 0, world = 1;
+    std::vector<hpl::Arena> peer_arenas;       // worker-per-GPU mode: replicas of the other ranks' allocators (index = rank)
+    std::vector<char> rank_alive;
+    struct Level {                             // tasks of one dependency level of the current plan, all ranks'
+        std::vector<std::pair<ReduceOp*, PlannedReduceTask>> r;
+        std::vector<std::pair<BcastOp*, PlannedFanout>> f;
+    };
+    std::vector<Level> levels;                 // planned, not yet released (worker-per-GPU mode)
     uint64_t guard_bytes = 0;                                  // testing aid: canary after every arena block
     std::map<void*, std::pair<uint64_t, uint64_t>> guards;     // block -> (offset of its canary, length)
     uint64_t guard_violations = 0;
@@ -307,12 +317,14 @@ DeviceStatus* next_wave_status(hpl_ctx* c);
 cudaEvent_t take_event(hpl_ctx* c);
 void collect_kernel_times(hpl_ctx* c);
 void release_object_memory(hpl_ctx* c, Object& o);
-void* arena_alloc(hpl_ctx* c, uint64_t n);
+void* arena_alloc(hpl_ctx* c, uint64_t n, int home = -1);
+hpl::Arena& arena_of_rank(hpl_ctx* c, int home);
 void arena_release(hpl_ctx* c, void* p);
 uint64_t check_guard(hpl_ctx* c, void* block);
 
 // plan_reduce.cpp
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);
+int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out);
 int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);
 int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedReduceTask*>>& group, bool bf16);
 void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv);

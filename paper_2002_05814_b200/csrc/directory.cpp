@@ -162,14 +162,20 @@ void collect_kernel_times(hpl_ctx* c) {   // call only after the stream has been
 // hpl_check_guards, so that a kernel that runs past a target, a partial result or a store copy is noticed.
 constexpr int kGuardPattern = 0xC5;
 
-void* arena_alloc(hpl_ctx* c, uint64_t n) {
-    if (!c->guard_bytes || !c->device) return c->arena.alloc(n);
+Arena& arena_of_rank(hpl_ctx* c, int home) { return (home < 0 || home == c->rank || c->world <= 1) ? c->arena : c->peer_arenas[home]; }
+
+// `home`: the rank on whose GPU the block lives (worker-per-GPU mode; every rank makes the same allocations in the same
+// order in its replica of that rank's allocator, so the offset is known everywhere).  -1 = this rank.
+void* arena_alloc(hpl_ctx* c, uint64_t n, int home) {
+    Arena& ar = arena_of_rank(c, home);
+    const bool local = &ar == &c->arena;
+    if (!c->guard_bytes || !c->device) return ar.alloc(n);
     const uint64_t body = (n + kAlign - 1) / kAlign * kAlign;
-    uint8_t* p = (uint8_t*)c->arena.alloc(body + c->guard_bytes);
-    if (!p) return nullptr;
+    uint8_t* p = (uint8_t*)ar.alloc(body + c->guard_bytes);
+    if (!p || !local) return p;      // (a remote block's canary is its owner's to write and check)
     // from the first byte behind the object (the padding up to the block's alignment is canary too)
     if (cudaMemsetAsync(p + n, kGuardPattern, body - n + c->guard_bytes, c->stream) != cudaSuccess) {
-        c->arena.release(p);
+        ar.release(p);
         return nullptr;
     }
     c->guards[p] = {n, body - n + c->guard_bytes};
@@ -189,9 +195,18 @@ uint64_t check_guard(hpl_ctx* c, void* block) {
 }
 
 void arena_release(hpl_ctx* c, void* p) {
-    if (c->guard_bytes && c->device) {
+    if (c->guard_bytes && c->device && c->guards.count(p)) {
         c->guard_violations += check_guard(c, p);
         c->guards.erase(p);
+    }
+    if (c->world > 1) {   // the block belongs to the allocator whose range holds it
+        for (int r = 0; r < c->world; ++r) {
+            Arena& ar = arena_of_rank(c, r);
+            if ((uint8_t*)p >= ar.base && (uint8_t*)p < ar.base + ar.size) {
+                ar.release(p);
+                return;
+            }
+        }
     }
     c->arena.release(p);
 }

@@ -11,12 +11,17 @@
 // kept, so the bits do not depend on it.
 #include "context.h"
 
+#include <dlfcn.h>
+
+#include <mutex>
+
 using namespace hpl;
 
 namespace {
 
 int sync_and_check(hpl_ctx* c);
 int progress(hpl_ctx* c);
+int plan_levels(hpl_ctx* c);
 
 // Small objects (Section 3.2 treats objects under 64 KB apart: for them latency, not bandwidth, is the cost).
 // Their collectives do not get launches of their own: the tasks planned for them in one pass are gathered and
@@ -59,6 +64,77 @@ int flush_small(hpl_ctx* c, SmallBatch& sb) {
     return HPL_OK;
 }
 
+// Worker-per-GPU mode: the plan of one pass, identical on every rank, is kept as dependency levels; nothing is
+// launched here.  A task sits in the level after everything it reads: the levels of its own tree below it, the
+// collectives whose output it consumes.  hpl_run_level releases one level at a time, each rank launching the tasks
+// whose output (reduce) or source copy (fan-out) lives on its GPU; the caller puts a barrier between levels.
+int plan_levels(hpl_ctx* c) {
+    if (!c->levels.empty()) return HPL_OK;   // the previous plan has not been run to its end yet
+    std::unordered_map<int64_t, int> end_level;   // output id -> last level that writes it in this plan
+    auto level_at = [c](int l) -> hpl_ctx::Level& {
+        if ((int)c->levels.size() < l) c->levels.resize(l);
+        return c->levels[l - 1];
+    };
+    auto ri = c->reduces.begin();
+    auto bi = c->bcasts.begin();
+    while (ri != c->reduces.end() || bi != c->bcasts.end()) {
+        const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
+        c->batch_tag = c->launch_seq;
+        if (take_reduce) {
+            ReduceOp& op = ri->second;
+            std::vector<PlannedReduceTask> tasks;
+            int rc = plan_reduce(c, op, tasks);
+            if (rc != HPL_OK) return rc;
+            int base = 0, top = 0;
+            for (int p = 0; p < op.sched->k(); ++p) {
+                auto e = end_level.find(op.sched->object_at(p));
+                if (e != end_level.end()) base = std::max(base, e->second);
+            }
+            for (auto& t : tasks) {
+                top = std::max(top, t.level);
+                level_at(base + t.level).r.push_back({&op, std::move(t)});
+            }
+            if (top) end_level[op.target] = base + top;
+            ++ri;
+        } else {
+            BcastOp& op = bi->second;
+            std::vector<PlannedFanout> tasks;
+            int rc = plan_bcast(c, op, tasks);
+            if (rc != HPL_OK) return rc;
+            auto e = end_level.find(op.src);
+            const int lvl = (e == end_level.end() ? 0 : e->second) + 1;
+            for (auto& t : tasks) level_at(lvl).f.push_back({&op, std::move(t)});
+            ++bi;
+        }
+    }
+    return HPL_OK;
+}
+
+int run_level(hpl_ctx* c) {
+    if (c->levels.empty()) return HPL_OK;
+    hpl_ctx::Level lv = std::move(c->levels.front());
+    c->levels.erase(c->levels.begin());
+    for (int bf = 0; bf < 2; ++bf) {
+        std::vector<std::pair<ReduceOp*, PlannedReduceTask*>> g;
+        for (auto& x : lv.r) {
+            if ((x.first->in_dtype == HPL_BF16) != (bf == 1)) continue;
+            Object* out = nullptr;
+            int rc = ensure_partial_buffer(c, *x.first, x.second.pos, &out);
+            if (rc != HPL_OK) return rc;
+            if (out->home == c->rank) g.push_back({x.first, &x.second});   // owner computes
+        }
+        int rc = launch_reduce_group(c, g, bf == 1);
+        if (rc != HPL_OK) return rc;
+    }
+    std::vector<std::pair<BcastOp*, PlannedFanout>> g;
+    for (auto& x : lv.f) {
+        const auto& locs = x.first->sched->locations();
+        Object* from = x.second.loc == 0 ? find(c, x.first->src) : find(c, locs[x.second.loc].obj);
+        if (from && from->home == c->rank) g.push_back(std::move(x));   // the holder of the copy pushes it to its receivers
+    }
+    return launch_fanout_group(c, g);
+}
+
 int progress(hpl_ctx* c) {
     // (a schedule-only context plans as well -- its planned tasks are counted, nothing is launched)
     {
@@ -73,6 +149,7 @@ int progress(hpl_ctx* c) {
         for (auto& kv : c->objects)
             if (kv.second.async_counter) kv.second.landed = published_chunks(c, kv.second);
     }
+    if (c->world > 1) return plan_levels(c);
     // collectives in creation order, so that one that consumes another's output (composed Reduce, reduce
     // followed by broadcast) is planned after its producer and launched behind it on the stream
     SmallBatch sb;
@@ -276,9 +353,15 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
     if (!cfg || !out) return HPL_ERR_INVALID;
     if (cfg->chunk_bytes == 0 || cfg->chunk_bytes % 16 || cfg->reduce_degree < 0 || cfg->bcast_degree < 1) return HPL_ERR_INVALID;
     if (cfg->reduce_degree == 0 && (cfg->model_latency_ns == 0 || cfg->model_bandwidth_bps == 0)) return HPL_ERR_INVALID;
+    if (cfg->world_size > 1 && (cfg->rank < 0 || cfg->rank >= cfg->world_size || cfg->plan_ahead || cfg->eager)) return HPL_ERR_INVALID;
     hpl_ctx* c = new (std::nothrow) hpl_ctx();
     if (!c) return HPL_ERR_NOMEM;
     c->cfg = *cfg;
+    if (cfg->world_size > 1) {
+        c->rank = cfg->rank;
+        c->world = cfg->world_size;
+        c->rank_alive.assign(c->world, 1);
+    }
     if (c->cfg.poll_budget_ns == 0) c->cfg.poll_budget_ns = 2000000000ull;
     c->tau = cfg->virt_chunk_ns ? cfg->virt_chunk_ns : std::max<uint64_t>(1, cfg->chunk_bytes * 1000000000ull / (64ull << 30));
     c->stream = (cudaStream_t)cuda_stream;
@@ -337,6 +420,22 @@ int hpl_init(const hpl_config* cfg, void* cuda_stream, hpl_ctx** out) {
         }
         for (int r = (int)kMaxRows - 1; r >= 0; --r) c->free_rows.push_back(r);
         c->n_sm = 148;
+    }
+    if (c->world > 1) {
+        // replicas of the other ranks' allocators: same size, same first allocations (directory, error records), so
+        // that every later allocation lands at the same offset everywhere.  Their base addresses are set by
+        // hpl_set_peer_arena; until then (and in a schedule-only context) a range that is never dereferenced stands in.
+        c->peer_arenas.resize(c->world);
+        for (int r = 0; r < c->world; ++r) {
+            if (r == c->rank) continue;
+            c->peer_arenas[r].init((void*)(uintptr_t)((1ull << 45) + ((uint64_t)r << 40)), c->arena.size);
+            c->peer_arenas[r].alloc(sizeof(DirRow) * kMaxRows);
+            c->peer_arenas[r].alloc(sizeof(DeviceStatus) * kStatusSlots);
+        }
+        if (!c->device) {   // the schedule-only arena takes the same two blocks, like a device one
+            c->arena.alloc(sizeof(DirRow) * kMaxRows);
+            c->arena.alloc(sizeof(DeviceStatus) * kStatusSlots);
+        }
     }
     *out = c;
     return HPL_OK;
@@ -408,6 +507,7 @@ int hpl_put(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
     if (!first && (o->ptr != buf || o->from_host)) return HPL_ERR_INVALID;
     if (first) {
         o->ptr = const_cast<void*>(buf);
+        o->home = c->world > 1 ? o->worker % c->world : 0;
         rc = alloc_row(c, *o);
         if (rc != HPL_OK) {
             o->ptr = nullptr;
@@ -441,6 +541,7 @@ int hpl_put_host(hpl_ctx* c, int64_t id, const void* buf, uint64_t bytes) {
     int rc = put_checks(c, id, buf, bytes, &o);
     if (rc != HPL_OK) return rc;
     if (!c->device) return HPL_ERR_CUDA;
+    if (c->world > 1) return HPL_ERR_INVALID;   // host objects are copied into THIS rank's store: not in worker-per-GPU mode
     const bool first = !o->arrived;
     if (!first && !o->from_host) return HPL_ERR_INVALID;
     if (first) {
@@ -521,7 +622,9 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     t.ready_bytes = 0;
     t.seq = c->seq++;
     {
-        t.ptr = arena_alloc(c, t.bytes);
+        t.home = c->world > 1 ? (int)(target % c->world) : 0;
+        if (c->world > 1 && !c->rank_alive[t.home]) return HPL_ERR_FAILED_WORKER;
+        t.ptr = arena_alloc(c, t.bytes, t.home);
         if (!t.ptr) return HPL_ERR_NOMEM;
         int rc = alloc_row(c, t);
         if (rc != HPL_OK) {
@@ -612,6 +715,7 @@ int hpl_join(hpl_ctx* c, int64_t dst_id, void* dst_buf) {
     const int li = b.sched->index_of(dst_id);
     if (li < 0 || !b.sched->locations()[li].alive) {   // first join, or again after its worker was rebuilt
         d->ptr = dst_buf;
+        d->home = c->world > 1 ? d->worker % c->world : 0;
         d->ready_bytes = 0;
         int rc = alloc_row(c, *d);
         if (rc != HPL_OK) return rc;
@@ -733,8 +837,10 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
             if (bytes) *bytes = o->bytes;
             return HPL_OK;
         }
-        int rc = progress(c);   // whatever can run now runs, even if the target cannot complete yet
+        if (op.lost) return HPL_ERR_FAILED_WORKER;
+        int rc = c->world > 1 ? HPL_OK : progress(c);   // whatever can run now runs, even if the target cannot complete yet
         if (rc != HPL_OK) return rc;
+        if (c->world > 1 && !c->levels.empty()) return HPL_ERR_TIMEOUT;   // the caller drives the levels (hpl_run_level)
         if (!op.sched->full()) return HPL_ERR_TIMEOUT;
         for (int p = 0; p < op.sched->k(); ++p) {
             Object* m = find(c, op.sched->object_at(p));
@@ -751,6 +857,8 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
         const int li = op.sched->index_of(id);
         if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
+        if (c->world > 1 && (!c->levels.empty() || li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C))
+            return HPL_ERR_TIMEOUT;   // the caller drives the levels (hpl_run_level)
         if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) {
             // start the copies first: the GPU works while the host lets the virtual clock run below
             int rc = progress(c);
@@ -774,7 +882,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
             if (bytes) *bytes = o->bytes;
             return HPL_OK;
         }
-        int rc = progress(c);
+        int rc = c->world > 1 ? HPL_OK : progress(c);
         if (rc != HPL_OK) return rc;
         if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) return HPL_ERR_TIMEOUT;
         rc = sync_and_check(c);
@@ -923,6 +1031,122 @@ int hpl_schedule_dump(hpl_ctx* c, int64_t op_id, int64_t* words, uint64_t cap, u
     *len = w.size();
     if (!words || cap < w.size()) return HPL_ERR_INVALID;
     std::memcpy(words, w.data(), w.size() * sizeof(int64_t));
+    return HPL_OK;
+}
+
+int hpl_set_peer_arena(hpl_ctx* c, int32_t rank, void* base) {
+    if (!c || c->world <= 1 || rank < 0 || rank >= c->world || rank == c->rank || !base || (uintptr_t)base % kAlign) return HPL_ERR_INVALID;
+    Arena& ar = c->peer_arenas[rank];
+    if (ar.sizes_.size() != 2) return HPL_ERR_INVALID;   // addresses in it have been handed out already
+    ar.base = (uint8_t*)base;
+    return HPL_OK;
+}
+
+int hpl_pending_levels(hpl_ctx* c, int32_t* levels) {
+    if (!c || !levels) return HPL_ERR_INVALID;
+    *levels = (int32_t)c->levels.size();
+    return HPL_OK;
+}
+
+int hpl_run_level(hpl_ctx* c) {
+    if (!c || c->world <= 1) return HPL_ERR_INVALID;
+    return run_level(c);
+}
+
+int hpl_fail_rank(hpl_ctx* c, int32_t rank) {
+    if (!c || c->world <= 1 || rank < 0 || rank >= c->world) return HPL_ERR_INVALID;
+    if (!c->levels.empty()) return HPL_ERR_INVALID;   // a rank leaves between plans, with no level pending
+    if (!c->rank_alive[rank]) return HPL_OK;
+    if (c->device) {
+        cudaStreamSynchronize(c->ctl_stream);
+        cudaStreamSynchronize(c->stream);
+    }
+    c->rank_alive[rank] = 0;
+    // what the library itself kept on that GPU: outputs are lost with it, partial results are made again elsewhere
+    for (auto& kv : c->reduces) {
+        ReduceOp& op = kv.second;
+        Object* tgt = find(c, op.target);
+        if (tgt && tgt->home == rank) {
+            op.lost = true;
+            invalidate_consumers(c, op.target);
+        }
+        ReduceInvalidation inv;
+        for (int p = 0; p < (int)op.partial_key.size(); ++p) {
+            if (op.partial_key[p] == 0) continue;
+            Object* po = find(c, op.partial_key[p]);
+            if (!po || po->home != rank) continue;
+            release_object_memory(c, *po);
+            c->objects.erase(op.partial_key[p]);
+            op.partial_key[p] = 0;
+            inv.touched.push_back(p);
+        }
+        if (!inv.touched.empty()) {
+            apply_invalidation(op, inv);
+            invalidate_consumers(c, op.target);
+        }
+    }
+    // its task workers fail (Section 3.5)
+    std::vector<int32_t> workers;
+    for (auto& kv : c->objects)
+        if (kv.second.alive && kv.second.worker >= 0 && kv.second.worker % c->world == rank) workers.push_back(kv.second.worker);
+    std::sort(workers.begin(), workers.end());
+    workers.erase(std::unique(workers.begin(), workers.end()), workers.end());
+    for (int32_t w : workers) {
+        int rc = hpl_fail(c, w);
+        if (rc != HPL_OK) return rc;
+    }
+    return HPL_OK;
+}
+
+int hpl_ipc_export(const void* dev_ptr, uint8_t handle[64], uint64_t* offset) {
+    static_assert(sizeof(cudaIpcMemHandle_t) == 64, "IPC handle size");
+    if (!dev_ptr || !handle || !offset) return HPL_ERR_INVALID;
+    // the start of the allocation: asked of the driver, which is looked up at run time (the library itself links
+    // the runtime only, so that it loads on a machine without a GPU)
+    typedef int (*range_fn)(unsigned long long*, size_t*, unsigned long long);
+    static range_fn get_range = nullptr;
+    if (!get_range) {
+        void* drv = dlopen("libcuda.so.1", RTLD_NOW | RTLD_GLOBAL);
+        if (drv) get_range = (range_fn)dlsym(drv, "cuMemGetAddressRange_v2");
+    }
+    unsigned long long base = 0;
+    size_t size = 0;
+    if (!get_range || get_range(&base, &size, (unsigned long long)(uintptr_t)dev_ptr) != 0) return HPL_ERR_CUDA;
+    cudaIpcMemHandle_t h;
+    CUDA_TRY(cudaIpcGetMemHandle(&h, (void*)(uintptr_t)base));
+    std::memcpy(handle, &h, 64);
+    *offset = (uint64_t)((uintptr_t)dev_ptr - base);
+    return HPL_OK;
+}
+
+namespace {
+std::mutex g_ipc_mu;
+std::map<void*, void*> g_ipc_base_of;   // address handed out by hpl_ipc_import -> start of the mapping
+}
+
+int hpl_ipc_import(const uint8_t handle[64], uint64_t offset, void** dev_ptr) {
+    if (!handle || !dev_ptr) return HPL_ERR_INVALID;
+    cudaIpcMemHandle_t h;
+    std::memcpy(&h, handle, 64);
+    void* base = nullptr;
+    CUDA_TRY(cudaIpcOpenMemHandle(&base, h, cudaIpcMemLazyEnablePeerAccess));
+    *dev_ptr = (uint8_t*)base + offset;
+    std::lock_guard<std::mutex> lock(g_ipc_mu);
+    g_ipc_base_of[*dev_ptr] = base;
+    return HPL_OK;
+}
+
+int hpl_ipc_close(void* dev_ptr) {
+    if (!dev_ptr) return HPL_ERR_INVALID;
+    void* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_ipc_mu);
+        auto it = g_ipc_base_of.find(dev_ptr);
+        if (it == g_ipc_base_of.end()) return HPL_ERR_NOT_FOUND;
+        base = it->second;
+        g_ipc_base_of.erase(it);
+    }
+    CUDA_TRY(cudaIpcCloseMemHandle(base));
     return HPL_OK;
 }
 

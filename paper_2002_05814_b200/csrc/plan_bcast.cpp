@@ -46,6 +46,20 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
             if (stuck[r] || !usable(r) || locs[r].last_sender < 0) continue;
             if (op.phys_have[r] != (int64_t)a) continue;  // needs this interval next
             int loc = -1;
+            if (c->world > 1) {
+                // worker-per-GPU mode: bytes cross the interconnect along the tree's edges only -- a receiver is
+                // served by its own sender, once that copy holds the interval (its rank pushes it)
+                const int x = locs[r].last_sender;
+                if (usable(x) && pre[x] >= (int64_t)b) loc = x;
+                if (loc < 0) {
+                    stuck[r] = 1;
+                    continue;
+                }
+                groups[loc].push_back(r);
+                c->journal.b.push_back({op.src, r, op.phys_have[r], c->batch_tag});
+                op.phys_have[r] = b;
+                continue;
+            }
             for (int x = locs[r].last_sender, hops = 0; x >= 0 && hops <= (int)locs.size(); x = locs[x].last_sender, ++hops) {
                 if (usable(x) && pre[x] >= (int64_t)b) {
                     loc = x;

@@ -34,7 +34,13 @@ int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out) {
     o.C = op.C;
     o.lib_owned = true;
     o.seq = c->seq++;
-    o.ptr = arena_alloc(c, o.bytes);
+    if (c->world > 1) {   // the partial result of a tree node lives with the node's object (else with the output)
+        Object* own = find(c, op.sched->object_at(pos));
+        Object* tgt = find(c, op.target);
+        o.home = own ? own->home : (tgt ? tgt->home : c->rank);
+        if (!c->rank_alive[o.home] && tgt) o.home = tgt->home;
+    }
+    o.ptr = arena_alloc(c, o.bytes, c->world > 1 ? o.home : -1);
     if (!o.ptr) return HPL_ERR_NOMEM;
     o.ready_bytes = o.bytes;
     int rc = alloc_row(c, o);
@@ -220,7 +226,7 @@ static void claim_fused_receivers(hpl_ctx* c, ReduceOp& op, PlannedReduceTask& t
 int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks) {
     ReduceTreeSchedule& s = *op.sched;
     const int k = s.k();
-    if (k <= 0) return HPL_OK;
+    if (k <= 0 || op.lost) return HPL_OK;
     std::vector<uint32_t> ready(k, 0), landed(k, 0);
     std::vector<uint32_t> bp = {0u, op.C};
     for (int p = 0; p < k; ++p) {

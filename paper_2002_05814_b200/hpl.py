@@ -34,7 +34,8 @@ class Config(C.Structure):
                 ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
                 ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64),
-                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32), ("debug_guard_bytes", C.c_uint64)]
+                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32), ("debug_guard_bytes", C.c_uint64),
+                ("rank", C.c_int32), ("world_size", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -126,6 +127,13 @@ def load_library():
         "hpl_schedule_dump": [VP, I64, P(I64), U64, P(U64)],
         "hpl_stats": [VP, P(Stats)],
         "hpl_check_guards": [VP, P(U64)],
+        "hpl_set_peer_arena": [VP, I32, VP],
+        "hpl_pending_levels": [VP, P(I32)],
+        "hpl_run_level": [VP],
+        "hpl_fail_rank": [VP, I32],
+        "hpl_ipc_export": [VP, P(C.c_uint8), P(U64)],
+        "hpl_ipc_import": [P(C.c_uint8), U64, P(VP)],
+        "hpl_ipc_close": [VP],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -159,11 +167,11 @@ class Context:
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
                  eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False,
                  model_latency_ns: int = 0, model_bandwidth_bps: int = 0, fuse_fanout: bool = True,
-                 debug_guard_bytes: int = 0):
+                 debug_guard_bytes: int = 0, rank: int = 0, world_size: int = 1):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
                      int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes,
-                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0, debug_guard_bytes)
+                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0, debug_guard_bytes, rank, world_size)
         self._h = C.c_void_p()
         self._p, self._n = C.c_void_p(), C.c_uint64()
         self._pref, self._nref = C.byref(self._p), C.byref(self._n)
@@ -305,6 +313,34 @@ class Context:
         self._check(self._lib.hpl_schedule_dump(self._h, op_id, buf, n.value, C.byref(n)), "hpl_schedule_dump")
         return list(buf)
 
+    # ---- worker-per-GPU mode (world_size > 1): every rank makes the same calls; see include/hpl.h
+    def set_peer_arena(self, rank: int, arena_base: int):
+        self._check(self._lib.hpl_set_peer_arena(self._h, rank, C.c_void_p(arena_base)), "hpl_set_peer_arena")
+
+    def pending_levels(self) -> int:
+        n = C.c_int32()
+        self._check(self._lib.hpl_pending_levels(self._h, C.byref(n)), "hpl_pending_levels")
+        return n.value
+
+    def run_level(self):
+        self._check(self._lib.hpl_run_level(self._h), "hpl_run_level")
+
+    def fail_rank(self, rank: int):
+        self._check(self._lib.hpl_fail_rank(self._h, rank), "hpl_fail_rank")
+
+    def drive(self, barrier):
+        """Called by every live rank together: plans, then releases the plan level by level -- own tasks of the level,
+        wait for the own stream, ``barrier()`` over the live ranks -- and plans again until nothing is left to do."""
+        while True:
+            self.progress()
+            n = self.pending_levels()
+            if n == 0:
+                return
+            for _ in range(n):
+                self.run_level()
+                self.sync()
+                barrier()
+
     def check_guards(self) -> int:
         """``hpl_check_guards``: canary bytes behind arena blocks found changed so far (0 without debug_guard_bytes)."""
         n = C.c_uint64()
@@ -324,6 +360,33 @@ def reduce_noalloc(src_ptrs, degree: int, op: int, dtype: int, elems: int, out_p
     lib = load_library()
     arr = (C.c_void_p * len(src_ptrs))(*src_ptrs)
     return lib.hpl_reduce_noalloc(arr, len(src_ptrs), degree, op, dtype, elems, C.c_void_p(out_ptr), C.c_void_p(stream or None))
+
+
+def ipc_export(dev_ptr: int):
+    """``hpl_ipc_export``: ``(handle, offset)`` -- the 64-byte CUDA IPC handle of the allocation that holds ``dev_ptr``
+    and the pointer's offset inside it."""
+    h = (C.c_uint8 * 64)()
+    off = C.c_uint64()
+    rc = load_library().hpl_ipc_export(C.c_void_p(dev_ptr), h, C.byref(off))
+    if rc:
+        raise HplError(rc, "hpl_ipc_export")
+    return bytes(h), off.value
+
+
+def ipc_import(handle: bytes, offset: int = 0) -> int:
+    """``hpl_ipc_import``: maps another process' allocation; returns the address of the exported byte in this process."""
+    h = (C.c_uint8 * 64)(*handle)
+    p = C.c_void_p()
+    rc = load_library().hpl_ipc_import(h, offset, C.byref(p))
+    if rc:
+        raise HplError(rc, "hpl_ipc_import")
+    return p.value
+
+
+def ipc_close(dev_ptr: int):
+    rc = load_library().hpl_ipc_close(C.c_void_p(dev_ptr))
+    if rc:
+        raise HplError(rc, "hpl_ipc_close")
 
 
 def choose_degree(n: int, object_bytes: int, latency_s: float, bandwidth_bytes_per_s: float) -> int:

@@ -1,0 +1,190 @@
+"""Worker-per-GPU mode, values: the ranks are emulated as several contexts in ONE process on one GPU -- each with an
+arena of its own, "peer" addresses being ordinary device addresses -- and driven level by level in turn, so no kernel
+ever waits for another one.  Every rank runs only the tasks it owns; the results must equal the oracle's bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_05814_b200 as hpl
+from oracle.store import OracleStore, DT_F32, DT_BF16
+from tests.harness import to_device, gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2002_05814_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+class Ranks:
+    def __init__(self, world, chunk, d, fuse, arena_bytes=48 << 20):
+        self.world = world
+        self.arenas = [torch.empty(arena_bytes, dtype=torch.uint8, device="cuda") for _ in range(world)]
+        stream = torch.cuda.current_stream().cuda_stream
+        self.c = [hpl.Context(chunk, d, d, arena=self.arenas[r].data_ptr(), arena_bytes=arena_bytes, stream=stream, fuse=fuse,
+                              rank=r, world_size=world, debug_guard_bytes=256) for r in range(world)]
+        for r in range(world):
+            for q in range(world):
+                if q != r:
+                    self.c[r].set_peer_arena(q, self.arenas[q].data_ptr())
+        self.live = list(range(world))
+        self.o = OracleStore(chunk, d, d)
+        self.host, self.dev = {}, {}
+        self.launches = [0] * world
+
+    def each(self, name, *args):
+        for r in self.live:
+            getattr(self.c[r], name)(*args)
+
+    def advance(self, t):
+        self.each("advance", t)
+        self.o.advance(t)
+
+    def create(self, oid, worker, data=None, nbytes=None, dtype=DT_F32):
+        if data is not None:
+            self.host[oid] = data
+            self.dev[oid] = to_device(data)
+            nbytes, dtype = data.nbytes, (DT_BF16 if data.dtype == np.uint16 else DT_F32)
+        else:
+            self.dev[oid] = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")
+        self.each("create", oid, worker, nbytes, dtype)
+        self.o.create(oid, worker, nbytes, dtype)
+
+    def put(self, oid, nbytes=None):
+        nbytes = self.host[oid].nbytes if nbytes is None else nbytes
+        self.each("put", oid, self.dev[oid].data_ptr(), nbytes)
+        self.o.put(oid, self.host[oid], nbytes)
+
+    def reduce(self, target, srcs, k, dtype=DT_F32):
+        self.each("reduce", target, srcs, k, 0, dtype)
+        self.o.reduce(target, srcs, k, 0, dtype)
+
+    def broadcast(self, src, dsts):
+        self.each("broadcast", src, dsts)
+        self.o.broadcast(src, dsts)
+
+    def join(self, dst):
+        self.each("join", dst, self.dev[dst].data_ptr())
+        self.o.join(dst)
+
+    def fail_rank(self, rank):
+        self.live.remove(rank)
+        self.each("fail_rank", rank)
+        for w in sorted({e.worker for e in self.o.objects.values() if e.alive and e.worker >= 0 and e.worker % self.world == rank}):
+            self.o.fail(w)
+
+    def drive(self):
+        while True:
+            self.each("progress")
+            n = {self.c[r].pending_levels() for r in self.live}
+            assert len(n) == 1, "the ranks' plans differ"
+            n = n.pop()
+            if n == 0:
+                return
+            for _ in range(n):
+                self.each("run_level")
+                for r in self.live:
+                    assert self.c[r].sync() == hpl.HPL_OK
+                # (here every rank would run its barrier)
+
+    def target_bits(self, target):
+        ptrs = {self.c[r].get(target) for r in self.live}
+        assert len(ptrs) == 1                                # peer addresses are plain addresses in this emulation
+        ptr, n = ptrs.pop()
+        home = target % self.world
+        off = ptr - self.arenas[home].data_ptr()
+        assert 0 <= off < self.arenas[home].numel(), "the output does not live on rank target % world"
+        return self.arenas[home][off:off + n].cpu().numpy().view(np.uint32)
+
+    def close(self):
+        for r in range(self.world):
+            if r in self.live:
+                assert self.c[r].check_guards() == 0
+            self.c[r].shutdown()
+        for oid, a in self.host.items():
+            assert self.dev[oid].view(torch.uint8).cpu().numpy().tobytes() == a.tobytes()
+
+
+@pytest.mark.parametrize("world,fuse,dtype", [(2, False, "f32"), (4, False, "f32"), (4, True, "f32"), (3, False, "bf16"), (8, False, "f32")])
+def test_tree_reduce_across_ranks_matches_the_oracle(world, fuse, dtype):
+    elems, chunk, k = 9 * 4096 + 11, 16 << 10, 8
+    p = Ranks(world, chunk, 2, fuse)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",) if dtype == "f32" else ("normal", 0.02), 400, i, elems, dtype))
+    p.reduce(100, list(range(k)), k, DT_BF16 if dtype == "bf16" else DT_F32)
+    for i in range(k):
+        p.advance(i + 1)
+        p.put(i, None if i != 3 else 2 * chunk)              # a member that is only partly there at first
+    p.drive()
+    p.advance(50)
+    p.put(3)
+    p.drive()
+    assert np.array_equal(p.target_bits(100), p.o.get(100).view(np.uint32))
+    for r in p.live:
+        assert p.c[r].schedule_dump(100) == p.o.dump(100)
+    st = [p.c[r].stats() for r in range(world)]
+    assert sum(s["reduce_tasks"] > 0 for s in st) >= min(2, world)        # the work is spread over the ranks
+    if not fuse:
+        assert sum(s["bytes_written_planned"] for s in st) >= 4 * elems * 4   # every internal node wrote its result
+    p.close()
+
+
+def test_broadcast_follows_the_tree_across_ranks_and_allreduce_is_fused_at_the_root():
+    elems, chunk, R = 6 * 4096 + 5, 16 << 10, 6
+    p = Ranks(4, chunk, 2, False)
+    for i in range(4):
+        p.create(i, i, gen(("uniform",), 401, i, elems))
+    src = gen(("uniform",), 402, 9, elems)
+    p.create(9, 2, src)
+    for j in range(R):
+        p.create(50 + j, 10 + j, nbytes=elems * 4)
+        p.create(70 + j, 20 + j, nbytes=elems * 4)
+    p.reduce(100, [0, 1, 2, 3], 4)
+    p.broadcast(100, [50 + j for j in range(R)])               # reduce followed by broadcast
+    p.broadcast(9, [70 + j for j in range(R)])                 # a plain object: two send slots per copy, depth > 1
+    p.put(9)
+    for j in range(R):
+        p.advance(j + 1)
+        p.join(50 + j)
+        p.join(70 + j)
+    p.advance(20)
+    for i in range(4):
+        p.put(i)
+    p.drive()
+    want = p.o.get(100)
+    assert np.array_equal(p.target_bits(100), want.view(np.uint32))
+    for j in range(R):
+        for r in p.live:
+            p.c[r].get(50 + j)
+            p.c[r].get(70 + j)
+        assert p.dev[50 + j].cpu().numpy().tobytes() == p.o.get(50 + j).tobytes() == want.tobytes()
+        assert p.dev[70 + j].cpu().numpy().tobytes() == src.tobytes()
+    assert p.c[0].schedule_dump(9) == p.o.dump(9)
+    p.close()
+
+
+def test_a_rank_is_lost_between_plans_and_the_survivors_sum_is_exact():
+    elems, chunk, k = 5 * 4096 + 3, 16 << 10, 8
+    p = Ranks(4, chunk, 2, False)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 403, i, elems))
+    p.reduce(100, list(range(k)), k)
+    for i in range(k):
+        p.advance(i + 1)
+        p.put(i, None if i != 6 else chunk)
+    p.drive()                                                 # partial results exist on every rank
+    p.advance(30)
+    p.fail_rank(3)                                            # workers 3 and 7 and what the library kept on that GPU
+    p.advance(40)
+    p.put(6)
+    p.drive()
+    got = p.target_bits(100)
+    assert np.array_equal(got, p.o.get(100).view(np.uint32))
+    ref = sum(p.host[i].astype(np.float64) for i in (0, 1, 2, 4, 5, 6))
+    assert np.max(np.abs(got.view(np.float32) - ref)) / np.max(np.abs(ref)) <= 3e-5
+    for r in p.live:
+        assert p.c[r].schedule_dump(100) == p.o.dump(100)
+    p.close()
