@@ -871,7 +871,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    w = wl.cfg5_at(args.size) if args.workload == "cfg5" else wl.workload(args.workload)
+    if args.workload == "allreduce":     # reduce followed by broadcast, 8 x 64 MiB fp32 to 8 receivers (Section 5.1's allreduce shape)
+        w = wl.Workload("allreduce", "allreduce", "f32", ("uniform",), 16 * MiB, 4 * MiB, 2, n_objects=8, k=8, n_receivers=8)
+    else:
+        w = wl.cfg5_at(args.size) if args.workload == "cfg5" else wl.workload(args.workload)
     if args.shrink > 1:
         w.elems = max(8, w.elems // args.shrink // 8 * 8)
     ab = algorithmic_bytes(w)
@@ -879,7 +882,8 @@ def main():
     name = {"cfg1": "cfg1 reduce 8 x 1 MiB fp32", "cfg2": "cfg2 broadcast 64 MiB fp32 to 16 receivers",
             "cfg3": "cfg3 async-SGD reduce, first 8 of 16 x 97.5 MiB fp32",
             "cfg4": "cfg4 policy round: broadcast 64 MiB bf16 to 64 receivers + fp32 sum of 64 x 64 MiB bf16",
-            "cfg5": f"cfg5 fault-tolerant reduce of 32 x {args.size} B fp32, worker 7 fails at 40%"}[w.name]
+            "cfg5": f"cfg5 fault-tolerant reduce of 32 x {args.size} B fp32, worker 7 fails at 40%",
+            "allreduce": "allreduce: fp32 sum of 8 x 64 MiB broadcast to 8 receivers, fused into one pass"}[w.name]
     if args.shrink > 1:
         name += f" [objects shrunk {args.shrink}x]"
     config = {"workload": name, "chunk_bytes": w.chunk_bytes, "degree": w.degree, "object_bytes": w.object_bytes,
@@ -967,7 +971,7 @@ def main():
         line["broadcast"] = {"GBps": gbs(ab["broadcast"] * args.steps, float(np.sum(res["bcast_ms"]))), "ms": float(np.mean(res["bcast_ms"])),
                              "ms_std": float(np.std(res["bcast_ms"]))}
 
-    if rank == 0 and world == 1 and args.also:
+    if rank == 0 and world == 1 and args.also and args.also != "none":
         also = {}
         for nm in [x for x in args.also.split(",") if x and x != "none" and x != w.name]:
             ww = wl.workload(nm)
