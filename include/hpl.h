@@ -276,6 +276,7 @@ typedef struct hpl_stats_t {
     uint64_t fanout_kernel_ns;
     uint64_t device_waits;         /* polls of a progress counter that did not succeed at the first look (updated by waits) */
     uint64_t fused_fanout_tasks;   /* reduce tasks that also wrote their result to broadcast receivers */
+    uint64_t evictions;            /* partial results dropped, least recently used first, because the arena was full */
     uint64_t bounds_errors;        /* bounds-checking build of the library only: waves in which a tile lay outside its
                                       object (the tile is skipped and the wait reports HPL_ERR_TIMEOUT) */
 } hpl_stats_t;

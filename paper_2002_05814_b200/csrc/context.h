@@ -162,6 +162,9 @@ struct Object {
     uint64_t seq = 0;          // creation order
     int row = -1;
     int home = 0;              // rank whose GPU holds the bytes (worker-per-GPU mode)
+    int pos = -1;              // partial result: its tree position (op_key = the Reduce's target)
+    uint64_t last_use = 0;     // partial result: when a planning pass last wrote or read it (eviction order)
+    uint64_t last_pass = 0;    //                 and which pass that was
 };
 
 struct Journal {  // what was planned since the last successful wait (undone if a device wait expires)
@@ -238,6 +241,8 @@ struct hpl_ctx {
         std::vector<std::pair<BcastOp*, PlannedFanout>> f;
     };
     std::vector<Level> levels;                 // planned, not yet released (worker-per-GPU mode)
+    uint64_t use_tick = 0, plan_pass = 0;                      // eviction clock of partial results; planning passes so far
+    int64_t planning_target = -1;                              // the Reduce being planned right now (-1 none)
     uint64_t guard_bytes = 0;                                  // testing aid: canary after every arena block
     std::map<void*, std::pair<uint64_t, uint64_t>> guards;     // block -> (offset of its canary, length)
     uint64_t guard_violations = 0;

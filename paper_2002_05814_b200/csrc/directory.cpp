@@ -162,6 +162,45 @@ void collect_kernel_times(hpl_ctx* c) {   // call only after the stream has been
 // hpl_check_guards, so that a kernel that runs past a target, a partial result or a store copy is noticed.
 constexpr int kGuardPattern = 0xC5;
 
+// Memory pressure (Section 6 of the paper: the copy made by Put is pinned until Delete, other copies may be evicted
+// least recently used first).  What this store keeps beyond the pinned copies -- sources, Reduce outputs -- are the
+// partial results of tree nodes: they can always be made again from the pinned sources.  When the arena is full the
+// least recently used ones are dropped, except those of the Reduce that is being planned and those the current
+// planning pass has already put into a task.  Returns whether anything was freed.
+static bool evict_partial_results(hpl_ctx* c, uint64_t need) {
+    if (c->world > 1) return false;
+    std::vector<Object*> cand;
+    for (auto& kv : c->objects) {
+        Object& o = kv.second;
+        if (o.kind == OBJ_PARTIAL && o.ptr && o.op_key != c->planning_target && o.last_pass != c->plan_pass) cand.push_back(&o);
+    }
+    if (cand.empty()) return false;
+    std::sort(cand.begin(), cand.end(), [](Object* a, Object* b) { return a->last_use < b->last_use; });
+    if (c->device) {   // enqueued work may still read them
+        cudaStreamSynchronize(c->ctl_stream);
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamSynchronize(c->stream);
+    }
+    uint64_t freed = 0;
+    for (Object* o : cand) {
+        auto it = c->reduce_of_target.find(o->op_key);
+        if (it != c->reduce_of_target.end()) {
+            ReduceOp& op = c->reduces.at(it->second);
+            if (o->pos >= 0 && o->pos < (int)op.partial_key.size() && op.partial_key[o->pos] == o->id) {
+                op.partial_key[o->pos] = 0;
+                op.merged[o->pos].clear();    // what the buffer held is gone; what ancestors merged from it stands
+            }
+        }
+        freed += o->bytes;
+        const int64_t id = o->id;
+        release_object_memory(c, *o);
+        c->objects.erase(id);
+        c->stats.evictions++;
+        if (freed >= need) break;
+    }
+    return true;
+}
+
 Arena& arena_of_rank(hpl_ctx* c, int home) { return (home < 0 || home == c->rank || c->world <= 1) ? c->arena : c->peer_arenas[home]; }
 
 // `home`: the rank on whose GPU the block lives (worker-per-GPU mode; every rank makes the same allocations in the same
@@ -169,9 +208,14 @@ Arena& arena_of_rank(hpl_ctx* c, int home) { return (home < 0 || home == c->rank
 void* arena_alloc(hpl_ctx* c, uint64_t n, int home) {
     Arena& ar = arena_of_rank(c, home);
     const bool local = &ar == &c->arena;
-    if (!c->guard_bytes || !c->device) return ar.alloc(n);
+    if (!c->guard_bytes || !c->device) {
+        void* q = ar.alloc(n);
+        while (!q && local && evict_partial_results(c, n)) q = ar.alloc(n);
+        return q;
+    }
     const uint64_t body = (n + kAlign - 1) / kAlign * kAlign;
     uint8_t* p = (uint8_t*)ar.alloc(body + c->guard_bytes);
+    while (!p && local && evict_partial_results(c, body + c->guard_bytes)) p = (uint8_t*)ar.alloc(body + c->guard_bytes);
     if (!p || !local) return p;      // (a remote block's canary is its owner's to write and check)
     // from the first byte behind the object (the padding up to the block's alignment is canary too)
     if (cudaMemsetAsync(p + n, kGuardPattern, body - n + c->guard_bytes, c->stream) != cudaSuccess) {

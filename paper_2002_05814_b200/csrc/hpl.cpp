@@ -136,6 +136,7 @@ int run_level(hpl_ctx* c) {
 }
 
 int progress(hpl_ctx* c) {
+    ++c->plan_pass;
     // (a schedule-only context plans as well -- its planned tasks are counted, nothing is launched)
     {
         int rc = flush_directory(c);

@@ -24,11 +24,17 @@ int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out) {
     }
     if (op.partial_key[pos] != 0) {
         *out = find(c, op.partial_key[pos]);
+        (*out)->last_use = ++c->use_tick;
+        (*out)->last_pass = c->plan_pass;
         return HPL_OK;
     }
     Object o;
     o.id = c->next_internal--;
     o.kind = OBJ_PARTIAL;
+    o.op_key = op.target;
+    o.pos = pos;
+    o.last_use = ++c->use_tick;
+    o.last_pass = c->plan_pass;
     o.bytes = op.elems * 4;
     o.dtype = HPL_F32;
     o.C = op.C;
@@ -64,7 +70,9 @@ void emit_operand(ReducePlanCtx& p, PlannedReduceTask& task, int q, bool partial
     st.a = (uint8_t)acc;
     if (partial) {
         st.kind = SRC_F32;
-        const Object* o = find(p.c, q == 0 ? op.target : op.partial_key[q]);
+        Object* o = find(p.c, q == 0 ? op.target : op.partial_key[q]);
+        o->last_use = ++p.c->use_tick;
+        o->last_pass = p.c->plan_pass;
         st.row = (uint32_t)o->row;
         st.ptr = (unsigned long long)(uintptr_t)o->ptr;
     } else {
@@ -227,6 +235,11 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
     ReduceTreeSchedule& s = *op.sched;
     const int k = s.k();
     if (k <= 0 || op.lost) return HPL_OK;
+    struct Planning {   // partial results of the Reduce being planned are not evicted under its feet
+        hpl_ctx* c;
+        Planning(hpl_ctx* ctx, int64_t t) : c(ctx) { c->planning_target = t; }
+        ~Planning() { c->planning_target = -1; }
+    } planning(c, op.target);
     std::vector<uint32_t> ready(k, 0), landed(k, 0);
     std::vector<uint32_t> bp = {0u, op.C};
     for (int p = 0; p < k; ++p) {

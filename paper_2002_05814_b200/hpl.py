@@ -44,7 +44,7 @@ class Stats(C.Structure):
                                           "bytes_read_planned", "bytes_written_planned", "device_timeouts",
                                           "arena_used", "h2d_bytes", "d2h_bytes", "last_kernel_grid",
                                           "reduce_launches", "fanout_launches", "reduce_kernel_ns",
-                                          "fanout_kernel_ns", "device_waits", "fused_fanout_tasks", "bounds_errors")]
+                                          "fanout_kernel_ns", "device_waits", "fused_fanout_tasks", "evictions", "bounds_errors")]
 
 
 class Event(C.Structure):

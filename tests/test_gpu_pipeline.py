@@ -276,3 +276,30 @@ def test_arena_canaries_notice_a_write_behind_a_block():
     torch.cuda.synchronize()
     assert p.c.check_guards() == 1
     p.c.shutdown()
+
+
+def test_partial_results_are_evicted_least_recently_used_when_the_arena_is_full():
+    """Section 6: pinned copies (sources, outputs) stay, other copies go under memory pressure.  Two Reduces whose tree
+    nodes each keep their reduced object do not fit the arena together: the second one's buffers take the place of the
+    first one's partial results, and after a failure the first one makes its own again."""
+    elems, chunk, k = 64 * 1024, 64 << 10, 8
+    S = elems * 4
+    fixed = 4096 * 32 + 256 * 32 + (64 << 10)              # directory, error records, slack
+    p = Pair(chunk, 2, fuse=False, arena_bytes=fixed + 7 * (S + 512))   # room for 7 buffers; the two trees want 2 x 4
+    for i in range(2 * k + 1):
+        p.create(i, i, gen(("uniform",), 81, i, elems))
+        p.put(i)
+    p.reduce(100, list(range(k)) + [2 * k], k)              # object 16 is a spare
+    p.check_target_bits(100)
+    assert p.c.stats()["evictions"] == 0
+    p.reduce(200, list(range(k, 2 * k)), k)
+    p.check_target_bits(200)
+    ev = p.c.stats()["evictions"]
+    assert ev >= 1
+    p.advance(10)
+    p.fail(3)                                               # the first tree has to redo the path above object 3
+    p.check_target_bits(100)
+    p.check_schedule(100)
+    assert p.c.stats()["evictions"] > ev
+    p.check_target_bits(200)                                # outputs were never touched
+    p.close()
