@@ -727,6 +727,7 @@ int hpl_join(hpl_ctx* c, int64_t dst_id, void* dst_buf) {
 
 int hpl_fail(hpl_ctx* c, int32_t worker) {
     if (!c || worker < 0) return HPL_ERR_INVALID;
+    if (!c->levels.empty()) return HPL_ERR_INVALID;   // worker-per-GPU mode: trees change between plans, not inside one
     std::vector<Object*> lost;
     for (auto& kv : c->objects)
         if (kv.second.worker == worker && kv.second.alive) lost.push_back(&kv.second);
@@ -756,6 +757,7 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
 
 int hpl_rejoin(hpl_ctx* c, int32_t worker) {
     if (!c || worker < 0) return HPL_ERR_INVALID;
+    if (!c->levels.empty()) return HPL_ERR_INVALID;
     bool any = false;
     for (auto& kv : c->objects) {
         Object& o = kv.second;
@@ -969,6 +971,7 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
     if (!c) return HPL_ERR_INVALID;
     Object* o = find(c, id);
     if (!o || id < 0) return HPL_ERR_NOT_FOUND;
+    if (!c->levels.empty()) return HPL_ERR_INVALID;       // worker-per-GPU mode: a planned level may still name it
     if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
     for (auto& kv : c->reduces)
         if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
@@ -1106,10 +1109,11 @@ int hpl_ipc_export(const void* dev_ptr, uint8_t handle[64], uint64_t* offset) {
     // the runtime only, so that it loads on a machine without a GPU)
     typedef int (*range_fn)(unsigned long long*, size_t*, unsigned long long);
     static range_fn get_range = nullptr;
-    if (!get_range) {
+    static std::once_flag looked_up;
+    std::call_once(looked_up, [] {
         void* drv = dlopen("libcuda.so.1", RTLD_NOW | RTLD_GLOBAL);
         if (drv) get_range = (range_fn)dlsym(drv, "cuMemGetAddressRange_v2");
-    }
+    });
     unsigned long long base = 0;
     size_t size = 0;
     if (!get_range || get_range(&base, &size, (unsigned long long)(uintptr_t)dev_ptr) != 0) return HPL_ERR_CUDA;
