@@ -666,7 +666,7 @@ def size_sweep(device, peak: float):
     return rows
 
 
-def worker_per_gpu_round(dist, device, rank: int, world: int, steps: int = 5):
+def worker_per_gpu_round(dist, device, rank: int, world: int, steps: int = 5, object_bytes: int = 64 * MiB):
     """The paper's own setting on N GPUs of one node: worker = rank, one 64 MiB fp32 object per GPU, a Reduce of all of
     them through a binary tree whose edges cross NVLink (every node's result materialised on its own GPU, remote
     operands pulled from peer memory; levels separated by a barrier).  Reported beside the replicas headline; every
@@ -681,13 +681,16 @@ def worker_per_gpu_round(dist, device, rank: int, world: int, steps: int = 5):
         state["ok"] = False
         state["err"] = state["err"] or repr(e)
 
+    # (with the gloo backend -- ranks that share one GPU in a test -- collectives take host tensors)
+    coll_device = device if dist.get_backend() == "nccl" else torch.device("cpu")
+
     def agree():
         """All ranks learn whether all are still fine (doubles as the barrier between levels)."""
-        t = torch.tensor([1 if state["ok"] else 0], device=device, dtype=torch.int32)
+        t = torch.tensor([1 if state["ok"] else 0], device=coll_device, dtype=torch.int32)
         dist.all_reduce(t, op=dist.ReduceOp.MIN)
         return bool(t.item())
 
-    S = 64 * MiB
+    S = object_bytes
     arena_bytes = 64 * MiB + 4 * S
     ctx, mapped = None, []
     out = {"objects": world, "object_bytes": S, "degree": 2}
@@ -760,7 +763,7 @@ def worker_per_gpu_round(dist, device, rank: int, world: int, steps: int = 5):
             torch.cuda.synchronize()
             dt = (time.perf_counter() - t0) * 1e3
             if step >= 2:
-                times.append(max_over_ranks([dt], dist, device)[0])
+                times.append(max_over_ranks([dt], dist, coll_device)[0])
             try:
                 ctx.get(1000)
                 for i in [1000] + ids:
@@ -893,7 +896,7 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        value, sample, ms = oracle_sample(w, budget_s=max(5.0, 4.0 * (args.steps + args.warmup)))
+        value, sample, ms = oracle_sample(w, budget_s=min(60.0, max(5.0, 4.0 * (args.steps + args.warmup))))
         line = {"impl": "reference", "metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value,
                 "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
