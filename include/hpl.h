@@ -81,7 +81,10 @@ typedef struct hpl_config {
                                  allreduce of Section 3.4.3), receivers that have joined take each result tile straight
                                  from the reduce pass -- the output is written once to the target and once to each of
                                  them and is not read again; 0: the broadcast always reads the target */
-    int32_t  reserved;
+    int32_t  pipeline_chunks; /* worker-per-GPU mode: > 0 releases a task's chunk range in pieces of this many chunks, piece j
+                                 one level after piece j-1, so that a tree level (or a broadcast hop) works on piece j
+                                 while the next one works on piece j-1 -- Section 3.3's pipelining across the levels of a
+                                 tree; 0: whole ranges, one level per tree level */
     uint64_t debug_guard_bytes;   /* testing aid, 0 = off: every block the library takes from the arena is followed by this
                                  many bytes of a canary pattern that no kernel may touch; checked when a block is
                                  released and by hpl_check_guards */

@@ -214,6 +214,7 @@ struct PlannedFanout {
     int loc;  // location index read from
     uint32_t a, b;
     bool poll;
+    int level = 1;  // worker-per-GPU mode: 1 + number of hops of this plan the copy that is read is away from one that holds the interval already
     std::vector<int> dst;  // location indices written
 };
 

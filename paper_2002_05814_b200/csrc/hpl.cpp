@@ -90,9 +90,20 @@ int plan_levels(hpl_ctx* c) {
                 auto e = end_level.find(op.sched->object_at(p));
                 if (e != end_level.end()) base = std::max(base, e->second);
             }
+            // a task's chunk range is released in pieces, piece j one level after piece j - 1: while a tree level
+            // works on piece j, the level above it works on piece j - 1 (pipelining across the levels, Section 3.3)
+            const uint32_t g = c->cfg.pipeline_chunks > 0 ? (uint32_t)c->cfg.pipeline_chunks : ~0u;
             for (auto& t : tasks) {
-                top = std::max(top, t.level);
-                level_at(base + t.level).r.push_back({&op, std::move(t)});
+                int j = 0;
+                for (uint32_t a = t.a; a < t.b; ++j) {
+                    const uint32_t b = (t.b - a > g) ? a + g : t.b;
+                    PlannedReduceTask piece = t;
+                    piece.a = a;
+                    piece.b = b;
+                    top = std::max(top, t.level + j);
+                    level_at(base + t.level + j).r.push_back({&op, std::move(piece)});
+                    a = b;
+                }
             }
             if (top) end_level[op.target] = base + top;
             ++ri;
@@ -102,8 +113,19 @@ int plan_levels(hpl_ctx* c) {
             int rc = plan_bcast(c, op, tasks);
             if (rc != HPL_OK) return rc;
             auto e = end_level.find(op.src);
-            const int lvl = (e == end_level.end() ? 0 : e->second) + 1;
-            for (auto& t : tasks) level_at(lvl).f.push_back({&op, std::move(t)});
+            const int lvl = (e == end_level.end() ? 0 : e->second);
+            const uint32_t g = c->cfg.pipeline_chunks > 0 ? (uint32_t)c->cfg.pipeline_chunks : ~0u;
+            for (auto& t : tasks) {   // hop h of the plan one level after hop h - 1, piece j one level after piece j - 1
+                int j = 0;
+                for (uint32_t a = t.a; a < t.b; ++j) {
+                    const uint32_t b = (t.b - a > g) ? a + g : t.b;
+                    PlannedFanout piece = t;
+                    piece.a = a;
+                    piece.b = b;
+                    level_at(lvl + t.level + j).f.push_back({&op, std::move(piece)});
+                    a = b;
+                }
+            }
             ++bi;
         }
     }

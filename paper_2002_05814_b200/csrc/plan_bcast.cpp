@@ -41,25 +41,36 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
     std::vector<char> stuck(locs.size(), 0);
     for (size_t bi = 0; bi + 1 < bp.size(); ++bi) {
         const uint32_t a = bp[bi], b = bp[bi + 1];
-        std::map<int, std::vector<int>> groups;  // read location -> receivers
-        for (int r = 1; r < (int)locs.size(); ++r) {
+        std::map<int, std::vector<int>> groups;  // read location (and, in worker-per-GPU mode, hop depth) -> receivers
+        if (c->world > 1) {
+            // worker-per-GPU mode: bytes cross the interconnect along the tree's edges only -- a receiver is served by
+            // its own sender (whose rank pushes), from a copy that holds the interval already or that is itself
+            // served in this plan, one hop (level) earlier
+            std::vector<int> depth(locs.size(), -1);   // hops of this plan after which the location holds [a, b)
+            for (size_t x = 0; x < locs.size(); ++x)
+                if (usable((int)x) && pre[x] >= (int64_t)b) depth[x] = 0;
+            bool progressed = true;
+            while (progressed) {
+                progressed = false;
+                for (int r = 1; r < (int)locs.size(); ++r) {
+                    if (stuck[r] || !usable(r) || locs[r].last_sender < 0 || depth[r] >= 0) continue;
+                    if (op.phys_have[r] != (int64_t)a) continue;
+                    const int x = locs[r].last_sender;
+                    if (!usable(x) || depth[x] < 0) continue;
+                    depth[r] = depth[x] + 1;
+                    groups[x * 4096 + depth[r]].push_back(r);
+                    c->journal.b.push_back({op.src, r, op.phys_have[r], c->batch_tag});
+                    op.phys_have[r] = b;
+                    progressed = true;
+                }
+            }
+            for (int r = 1; r < (int)locs.size(); ++r)
+                if (usable(r) && op.phys_have[r] == (int64_t)a && depth[r] < 0) stuck[r] = 1;
+        }
+        for (int r = 1; r < (int)locs.size() && c->world <= 1; ++r) {
             if (stuck[r] || !usable(r) || locs[r].last_sender < 0) continue;
             if (op.phys_have[r] != (int64_t)a) continue;  // needs this interval next
             int loc = -1;
-            if (c->world > 1) {
-                // worker-per-GPU mode: bytes cross the interconnect along the tree's edges only -- a receiver is
-                // served by its own sender, once that copy holds the interval (its rank pushes it)
-                const int x = locs[r].last_sender;
-                if (usable(x) && pre[x] >= (int64_t)b) loc = x;
-                if (loc < 0) {
-                    stuck[r] = 1;
-                    continue;
-                }
-                groups[loc].push_back(r);
-                c->journal.b.push_back({op.src, r, op.phys_have[r], c->batch_tag});
-                op.phys_have[r] = b;
-                continue;
-            }
             for (int x = locs[r].last_sender, hops = 0; x >= 0 && hops <= (int)locs.size(); x = locs[x].last_sender, ++hops) {
                 if (usable(x) && pre[x] >= (int64_t)b) {
                     loc = x;
@@ -83,16 +94,23 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
             op.phys_have[r] = b;
         }
         for (auto& g : groups) {
-            const bool poll = (g.first == 0) && (src_landed < b);
+            const int loc = c->world > 1 ? g.first / 4096 : g.first;
+            const int level = c->world > 1 ? g.first % 4096 : 1;
+            const bool poll = (loc == 0) && (src_landed < b);
             bool merged = false;
             for (auto& prev : tasks) {
-                if (prev.loc == g.first && prev.b == a && prev.poll == poll && prev.dst == g.second) {
+                if (prev.loc == loc && prev.level == level && prev.b == a && prev.poll == poll && prev.dst == g.second) {
                     prev.b = b;
                     merged = true;
                     break;
                 }
             }
-            if (!merged) tasks.push_back(PlannedFanout{g.first, a, b, poll, g.second});
+            if (!merged) {
+                PlannedFanout t{loc, a, b, poll};
+                t.level = level;
+                t.dst = g.second;
+                tasks.push_back(std::move(t));
+            }
         }
     }
     return HPL_OK;

@@ -34,7 +34,7 @@ class Config(C.Structure):
                 ("plan_ahead", C.c_int32), ("fuse", C.c_int32), ("time_kernels", C.c_int32),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_uint64),
                 ("model_latency_ns", C.c_uint64), ("model_bandwidth_bps", C.c_uint64),
-                ("fuse_fanout", C.c_int32), ("reserved", C.c_int32), ("debug_guard_bytes", C.c_uint64),
+                ("fuse_fanout", C.c_int32), ("pipeline_chunks", C.c_int32), ("debug_guard_bytes", C.c_uint64),
                 ("rank", C.c_int32), ("world_size", C.c_int32)]
 
 
@@ -167,11 +167,11 @@ class Context:
                  arena_bytes: int = 0, stream=0, virt_chunk_ns: int = 0, poll_budget_ns: int = 0,
                  eager: bool = False, plan_ahead: bool = False, fuse: bool = True, time_kernels: bool = False,
                  model_latency_ns: int = 0, model_bandwidth_bps: int = 0, fuse_fanout: bool = True,
-                 debug_guard_bytes: int = 0, rank: int = 0, world_size: int = 1):
+                 debug_guard_bytes: int = 0, rank: int = 0, world_size: int = 1, pipeline_chunks: int = 0):
         self._lib = load_library()
         cfg = Config(chunk_bytes, reduce_degree, bcast_degree, virt_chunk_ns, poll_budget_ns, int(eager),
                      int(plan_ahead), int(fuse), int(time_kernels), _addr(arena) if arena else None, arena_bytes,
-                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), 0, debug_guard_bytes, rank, world_size)
+                     model_latency_ns, model_bandwidth_bps, int(fuse_fanout), pipeline_chunks, debug_guard_bytes, rank, world_size)
         self._h = C.c_void_p()
         self._p, self._n = C.c_void_p(), C.c_uint64()
         self._pref, self._nref = C.byref(self._p), C.byref(self._n)

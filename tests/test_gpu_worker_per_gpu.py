@@ -20,12 +20,12 @@ def _lib():
 
 
 class Ranks:
-    def __init__(self, world, chunk, d, fuse, arena_bytes=48 << 20):
+    def __init__(self, world, chunk, d, fuse, arena_bytes=48 << 20, pipeline_chunks=0):
         self.world = world
         self.arenas = [torch.empty(arena_bytes, dtype=torch.uint8, device="cuda") for _ in range(world)]
         stream = torch.cuda.current_stream().cuda_stream
         self.c = [hpl.Context(chunk, d, d, arena=self.arenas[r].data_ptr(), arena_bytes=arena_bytes, stream=stream, fuse=fuse,
-                              rank=r, world_size=world, debug_guard_bytes=256) for r in range(world)]
+                              rank=r, world_size=world, debug_guard_bytes=256, pipeline_chunks=pipeline_chunks) for r in range(world)]
         for r in range(world):
             for q in range(world):
                 if q != r:
@@ -33,7 +33,7 @@ class Ranks:
         self.live = list(range(world))
         self.o = OracleStore(chunk, d, d)
         self.host, self.dev = {}, {}
-        self.launches = [0] * world
+        self.plans = []              # levels of every plan that had any
 
     def each(self, name, *args):
         for r in self.live:
@@ -84,6 +84,7 @@ class Ranks:
             n = n.pop()
             if n == 0:
                 return
+            self.plans.append(n)
             for _ in range(n):
                 self.each("run_level")
                 for r in self.live:
@@ -187,4 +188,45 @@ def test_a_rank_is_lost_between_plans_and_the_survivors_sum_is_exact():
     assert np.max(np.abs(got.view(np.float32) - ref)) / np.max(np.abs(ref)) <= 3e-5
     for r in p.live:
         assert p.c[r].schedule_dump(100) == p.o.dump(100)
+    p.close()
+
+
+@pytest.mark.parametrize("world,pieces", [(4, 2), (2, 1), (8, 3)])
+def test_pieces_of_a_chunk_range_move_up_the_tree_one_level_apart(world, pieces):
+    """pipeline_chunks: while a tree level reduces piece j, the level above it reduces piece j - 1 (Section 3.3).  The plan
+    has tree height + pieces - 1 levels instead of tree height; the bits are the same."""
+    elems, chunk, k = 12 * 4096, 16 << 10, 8                   # 12 chunks
+    p = Ranks(world, chunk, 2, False, pipeline_chunks=pieces)
+    for i in range(k):
+        p.create(i, i, gen(("uniform",), 410, i, elems))
+    p.reduce(100, list(range(k)), k)
+    for i in range(k):
+        p.advance(i + 1)
+        p.put(i)
+    p.drive()
+    assert np.array_equal(p.target_bits(100), p.o.get(100).view(np.uint32))
+    n_pieces = -(-12 // pieces)
+    assert p.plans == [3 + n_pieces - 1]                        # the tree of 8 has three levels of internal nodes
+    p.close()
+
+
+def test_a_broadcast_chain_is_pipelined_hop_by_hop_within_one_plan():
+    elems, chunk, R = 6 * 4096, 16 << 10, 5                     # 6 chunks, one send slot per copy: a chain of 5 hops
+    p = Ranks(3, chunk, 1, False, pipeline_chunks=1)
+    src = gen(("uniform",), 411, 0, elems)
+    p.create(0, 0, src)
+    for j in range(R):
+        p.create(10 + j, 1 + j, nbytes=elems * 4)
+    p.put(0)
+    p.broadcast(0, [10 + j for j in range(R)])
+    for j in range(R):
+        p.advance(j + 1)                                        # each joins while its predecessor is still receiving
+        p.join(10 + j)
+    p.drive()
+    for j in range(R):
+        for r in p.live:
+            p.c[r].get(10 + j)
+        assert p.dev[10 + j].cpu().numpy().tobytes() == src.tobytes() == p.o.get(10 + j).tobytes()
+    assert p.c[0].schedule_dump(0) == p.o.dump(0)
+    assert p.plans == [R + 6 - 1]                               # hop h works on piece j while hop h + 1 works on piece j - 1
     p.close()
