@@ -260,6 +260,7 @@ struct hpl_ctx {
     std::map<uint64_t, ReduceOp> reduces;  // by creation order
     std::map<uint64_t, BcastOp> bcasts;
     std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
+    std::unordered_map<int64_t, std::vector<uint64_t>> reduces_of_source;   // source id -> the Reduces that name it (keys of `reduces`)
     Journal journal;
     bool work_in_flight = false;
     bool polling_in_flight = false;   // some wave in flight polls progress counters (only those can record an error)

@@ -335,8 +335,12 @@ void invalidate_consumers(hpl_ctx* c, int64_t target) {
 }
 
 void notify_arrival(hpl_ctx* c, Object& o) {
-    for (auto& kv : c->reduces)
-        if (kv.second.sched->has_source(o.id)) kv.second.sched->arrive(o.id);
+    auto it = c->reduces_of_source.find(o.id);
+    if (it == c->reduces_of_source.end()) return;
+    for (uint64_t key : it->second) {   // in creation order
+        auto r = c->reduces.find(key);
+        if (r != c->reduces.end()) r->second.sched->arrive(o.id);
+    }
 }
 
 int do_put_common(hpl_ctx* c, Object& o, uint64_t bytes, bool first) {
@@ -690,6 +694,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     r.merged.assign(r.sched->k(), IntervalMap());
     r.partial_key.assign(r.sched->k(), 0);
     const uint64_t key = r.seq;
+    for (int64_t sid : srcs) c->reduces_of_source[sid].push_back(key);
     c->reduce_of_target[target] = key;
     c->reduces.emplace(key, std::move(r));
     refresh_composed(c);
@@ -995,8 +1000,10 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
     if (!o || id < 0) return HPL_ERR_NOT_FOUND;
     if (!c->levels.empty()) return HPL_ERR_INVALID;       // worker-per-GPU mode: a planned level may still name it
     if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
-    for (auto& kv : c->reduces)
-        if (kv.second.sched->has_source(id)) return HPL_ERR_INVALID;  // still referenced by a Reduce
+    {
+        auto it = c->reduces_of_source.find(id);
+        if (it != c->reduces_of_source.end() && !it->second.empty()) return HPL_ERR_INVALID;  // still referenced by a Reduce
+    }
     if (c->device && (c->work_in_flight || c->copy_pending || c->ctl_unconfirmed)) {
         // rows and arena memory are recycled only when nothing enqueued can still read them (nothing of the
         // library's is in flight after a Get or a wait, so a round's Deletes cost no device wait)
@@ -1015,6 +1022,12 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
                     c->objects.erase(pk);
                 }
             }
+        for (int64_t sid : op.sched->sources()) {
+            auto it = c->reduces_of_source.find(sid);
+            if (it == c->reduces_of_source.end()) continue;
+            it->second.erase(std::remove(it->second.begin(), it->second.end(), key), it->second.end());
+            if (it->second.empty()) c->reduces_of_source.erase(it);
+        }
         c->reduces.erase(key);
         c->reduce_of_target.erase(id);
     }

@@ -85,8 +85,13 @@ std::vector<int> ReduceTreeSchedule::strict_ancestors(int p) const {
 }
 
 int ReduceTreeSchedule::first_open() const {
-    for (int p : generalised_inorder(k_, d_))
-        if (at_[p] < 0) return p;
+    if (order_k_ != k_) {
+        order_ = generalised_inorder(k_, d_);
+        order_k_ = k_;
+        filled_prefix_ = 0;
+    }
+    for (; filled_prefix_ < order_.size(); ++filled_prefix_)
+        if (at_[order_[filled_prefix_]] < 0) return order_[filled_prefix_];
     return -1;
 }
 
@@ -117,6 +122,7 @@ void ReduceTreeSchedule::rejoin(int64_t obj) {
 ReduceInvalidation ReduceTreeSchedule::fail(int64_t obj, int64_t delivered,
                                             const std::function<int64_t(int64_t)>& delivered_of) {
     ReduceInvalidation inv;
+    filled_prefix_ = 0;   // a position may open anywhere
     auto it = alive_.find(obj);
     if (it == alive_.end() || !it->second) return inv;
     it->second = false;

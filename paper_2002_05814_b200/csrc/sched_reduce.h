@@ -73,6 +73,11 @@ private:
     std::vector<int64_t> spares_;
     std::vector<std::pair<int64_t, int>> placements_;
     std::vector<ReduceEdit> edits_;
+    // the in-order of the current tree, kept between arrivals, and how far it is known to be filled (reset by every
+    // event that can open a position)
+    mutable std::vector<int> order_;
+    mutable int order_k_ = -1;
+    mutable size_t filled_prefix_ = 0;
 };
 
 // Eq. 1 / Section 4: the degree among 1, 2 and n with the smallest estimated reduce time (ties: the smaller).
