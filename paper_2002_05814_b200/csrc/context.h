@@ -168,7 +168,7 @@ struct Object {
 };
 
 struct Journal {  // what was planned since the last successful wait (undone if a device wait expires)
-    // tag: number of waves launched before the planning pass that made the entry (its waves have seq >= tag)
+    // tag: the planning pass that made the entry; the waves that pass launches carry the same tag
     struct R { int64_t target; int pos; uint32_t a, b; int old_v; uint64_t tag; };
     struct B { int64_t src; int loc; int64_t old_have; uint64_t tag; };
     std::vector<R> r;
@@ -266,7 +266,8 @@ struct hpl_ctx {
     bool polling_in_flight = false;   // some wave in flight polls progress counters (only those can record an error)
     uint64_t launch_seq = 0;       // waves launched so far
     uint64_t first_unchecked = 0;  // the first wave whose error record has not been read back
-    uint64_t batch_tag = 0;        // launch_seq when the current planning pass began
+    uint64_t batch_tag = 0;        // tag of the current planning pass (one per collective and call of progress)
+    uint64_t tag_counter = 0;      // tags handed out so far: later passes have larger tags, whether or not anything was launched in between
     std::vector<uint64_t> wave_tag;  // for the waves in flight (seq - first_unchecked): the tag of their planning pass
     hpl_stats_t stats{};
     int occ_reduce[2][2][3] = {};   // [bf16][fan][accumulator class]

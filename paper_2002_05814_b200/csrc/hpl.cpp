@@ -79,7 +79,7 @@ int plan_levels(hpl_ctx* c) {
     auto bi = c->bcasts.begin();
     while (ri != c->reduces.end() || bi != c->bcasts.end()) {
         const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
-        c->batch_tag = c->launch_seq;
+        c->batch_tag = ++c->tag_counter;
         if (take_reduce) {
             ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
@@ -180,7 +180,7 @@ int progress(hpl_ctx* c) {
     auto bi = c->bcasts.begin();
     while (ri != c->reduces.end() || bi != c->bcasts.end()) {
         const bool take_reduce = bi == c->bcasts.end() || (ri != c->reduces.end() && ri->first < bi->first);
-        c->batch_tag = c->launch_seq;
+        c->batch_tag = ++c->tag_counter;
         if (take_reduce) {
             ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
@@ -198,9 +198,11 @@ int progress(hpl_ctx* c) {
                 sb.end_stage[op.target] = base + top;
                 sb.r.push_back({&op, std::move(tasks), base});
             } else if (!tasks.empty()) {
-                rc = flush_small(c, sb);     // what was planned earlier is launched earlier
+                // what was planned earlier is launched earlier.  (The tag of this planning pass stays as it was set
+                // before planning: the journal entries made above carry it, and the waves launched below must too, or a
+                // wait that runs out in one of them would not void them.)
+                rc = flush_small(c, sb);
                 if (rc != HPL_OK) return rc;
-                c->batch_tag = c->launch_seq;
                 rc = launch_reduce_tasks(c, op, tasks);
                 if (rc != HPL_OK) return rc;
             }
@@ -219,7 +221,6 @@ int progress(hpl_ctx* c) {
             } else if (!tasks.empty()) {
                 rc = flush_small(c, sb);
                 if (rc != HPL_OK) return rc;
-                c->batch_tag = c->launch_seq;
                 rc = launch_fanout_tasks(c, op, tasks);
                 if (rc != HPL_OK) return rc;
             }

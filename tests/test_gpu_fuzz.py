@@ -139,3 +139,11 @@ def test_random_timelines_match_the_oracle(block):
             _timeline(seed)
         except AssertionError as e:
             raise AssertionError(f"seed {seed}: {e}") from e
+
+
+@pytest.mark.parametrize("seed", [639, 1088, 1166, 1199, 1221, 1471])
+def test_small_collectives_beside_a_polling_one_whose_wait_runs_out(seed):
+    """Timelines in which a small collective (its tasks wait for a shared wave) is planned in the same pass as one whose
+    polling wave gives up: the wait that ran out must void exactly the pass that launched it and the later ones -- not
+    the small collective planned before it, whose wave completed -- and must void all of its own pass."""
+    _timeline(seed)
