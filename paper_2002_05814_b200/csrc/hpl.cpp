@@ -90,18 +90,23 @@ int plan_levels(hpl_ctx* c) {
                 auto e = end_level.find(op.sched->object_at(p));
                 if (e != end_level.end()) base = std::max(base, e->second);
             }
-            // a task's chunk range is released in pieces, piece j one level after piece j - 1: while a tree level
-            // works on piece j, the level above it works on piece j - 1 (pipelining across the levels, Section 3.3)
+            // a task's chunk range is released in pieces, one level apart: while a tree level works on a piece, the
+            // level above it works on the piece before (pipelining across the levels, Section 3.3).  Pieces are the
+            // groups of `pipeline_chunks` chunks counted from chunk 0 of the OBJECT, not from the task's first chunk:
+            // tasks of one tree cover different ranges, and a parent's piece must come after the child's same piece.
             const uint32_t g = c->cfg.pipeline_chunks > 0 ? (uint32_t)c->cfg.pipeline_chunks : ~0u;
+            uint32_t first_group = ~0u;
+            for (auto& t : tasks) first_group = std::min(first_group, t.a / g);
             for (auto& t : tasks) {
-                int j = 0;
-                for (uint32_t a = t.a; a < t.b; ++j) {
-                    const uint32_t b = (t.b - a > g) ? a + g : t.b;
+                for (uint32_t a = t.a; a < t.b;) {
+                    const uint32_t group = a / g;
+                    const uint32_t b = (g == ~0u || (uint64_t)(group + 1) * g >= t.b) ? t.b : (group + 1) * g;
                     PlannedReduceTask piece = t;
                     piece.a = a;
                     piece.b = b;
-                    top = std::max(top, t.level + j);
-                    level_at(base + t.level + j).r.push_back({&op, std::move(piece)});
+                    const int lvl = t.level + (int)(group - first_group);
+                    top = std::max(top, lvl);
+                    level_at(base + lvl).r.push_back({&op, std::move(piece)});
                     a = b;
                 }
             }
@@ -115,14 +120,16 @@ int plan_levels(hpl_ctx* c) {
             auto e = end_level.find(op.src);
             const int lvl = (e == end_level.end() ? 0 : e->second);
             const uint32_t g = c->cfg.pipeline_chunks > 0 ? (uint32_t)c->cfg.pipeline_chunks : ~0u;
-            for (auto& t : tasks) {   // hop h of the plan one level after hop h - 1, piece j one level after piece j - 1
-                int j = 0;
-                for (uint32_t a = t.a; a < t.b; ++j) {
-                    const uint32_t b = (t.b - a > g) ? a + g : t.b;
+            uint32_t first_group = ~0u;
+            for (auto& t : tasks) first_group = std::min(first_group, t.a / g);
+            for (auto& t : tasks) {   // hop h of the plan one level after hop h - 1, a piece one level after the piece before
+                for (uint32_t a = t.a; a < t.b;) {
+                    const uint32_t group = a / g;
+                    const uint32_t b = (g == ~0u || (uint64_t)(group + 1) * g >= t.b) ? t.b : (group + 1) * g;
                     PlannedFanout piece = t;
                     piece.a = a;
                     piece.b = b;
-                    level_at(lvl + t.level + j).f.push_back({&op, std::move(piece)});
+                    level_at(lvl + t.level + (int)(group - first_group)).f.push_back({&op, std::move(piece)});
                     a = b;
                 }
             }
@@ -888,9 +895,7 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
         const int li = op.sched->index_of(id);
         if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
-        if (c->world > 1 && (!c->levels.empty() || li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C))
-            return HPL_ERR_TIMEOUT;   // the caller drives the levels (hpl_run_level)
-        if (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C) {
+        if (c->world <= 1 && (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C)) {
             // start the copies first: the GPU works while the host lets the virtual clock run below
             int rc = progress(c);
             if (rc != HPL_OK) return rc;
@@ -907,6 +912,8 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
                 if (logical_delivered(c, op.src) < (int64_t)so->C) return HPL_ERR_TIMEOUT;
             }
         }
+        if (c->world > 1 && (!c->levels.empty() || li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C))
+            return HPL_ERR_TIMEOUT;   // worker-per-GPU mode: the caller drives the levels (hpl_run_level)
         if (!c->device) return HPL_ERR_CUDA;
         if (li < (int)op.phys_have.size() && op.phys_have[li] >= (int64_t)o->C && !c->work_in_flight && !c->copy_pending) {
             if (dev_ptr) *dev_ptr = o->ptr;   // already copied and waited for

@@ -37,12 +37,12 @@ def _get_both(p: Pair, oid, plan_ahead):
         p.c.sync()
 
 
-def _timeline(seed):
+def _timeline(seed, chunks=(4096, 16384)):
     rng = np.random.default_rng(seed)
     na, nb, R = int(rng.integers(2, 9)), int(rng.integers(1, 5)), int(rng.integers(1, 5))
     ka, kb = int(rng.integers(1, na + 1)), int(rng.integers(1, nb + 2))
     d = int(rng.integers(1, 5))
-    chunk = int(rng.choice([4096, 16384]))
+    chunk = int(rng.choice(list(chunks)))
     elems = int(rng.integers(1, 6)) * (chunk // 4) + int(rng.choice([0, 0, 3, 1000]))
     plan_ahead = bool(rng.random() < 0.3)
     flags = dict(fuse=bool(rng.random() < 0.6), eager=bool(rng.random() < 0.4), plan_ahead=plan_ahead,
@@ -137,6 +137,17 @@ def test_random_timelines_match_the_oracle(block):
     for seed in range(block * 40, (block + 1) * 40):
         try:
             _timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_timelines_with_objects_above_the_small_object_threshold(block):
+    """The same timelines with chunks of 32 and 64 KiB: objects of 32 KiB to 320 KiB, most of them above the 64 KiB
+    under which collectives share their waves."""
+    for seed in range(5000 + block * 40, 5000 + (block + 1) * 40):
+        try:
+            _timeline(seed, chunks=(32768, 65536))
         except AssertionError as e:
             raise AssertionError(f"seed {seed}: {e}") from e
 

@@ -230,3 +230,86 @@ def test_a_broadcast_chain_is_pipelined_hop_by_hop_within_one_plan():
     assert p.c[0].schedule_dump(0) == p.o.dump(0)
     assert p.plans == [R + 6 - 1]                               # hop h works on piece j while hop h + 1 works on piece j - 1
     p.close()
+
+
+def _rank_timeline(seed):
+    """A random timeline on emulated ranks: instalment Puts, joins, worker failures, a lost rank, drives in between."""
+    from oracle.store import StoreError, OK
+    rng = np.random.default_rng(seed)
+    world = int(rng.integers(2, 5))
+    k, R = int(rng.integers(2, 9)), int(rng.integers(1, 5))
+    kk = int(rng.integers(1, k + 1))
+    d = int(rng.integers(1, 4))
+    chunk = int(rng.choice([4096, 16384]))
+    elems = int(rng.integers(1, 6)) * (chunk // 4) + int(rng.choice([0, 0, 3, 1000]))
+    p = Ranks(world, chunk, d, bool(rng.random() < 0.5), arena_bytes=16 << 20, pipeline_chunks=int(rng.choice([0, 0, 1, 2])))
+    T = 1000 - 1000 % world                                     # the output lives on rank 0, which is never lost here
+    nbytes = elems * 4
+    for i in range(k):
+        p.create(i, int(rng.integers(0, 2 * world)), gen(("smallint", 30) if seed % 2 else ("uniform",), 600 + seed, i, elems))
+    for j in range(R):
+        p.create(500 + j, int(rng.integers(0, 2 * world)), nbytes=nbytes)
+    p.reduce(T, list(range(k)), kk)
+    p.broadcast(T, [500 + j for j in range(R)])
+    prefix = {i: 0 for i in range(k)}
+    joiners = [500 + j for j in range(R)]
+    lost_rank = False
+    t = 0
+    for _ in range(int(rng.integers(2 * k, 5 * k + 6))):
+        t = max(t + int(rng.integers(0, 40)), p.o.now)
+        p.advance(t)
+        r = rng.random()
+        if r < 0.5:
+            i = int(rng.integers(0, k))
+            if p.o.objects[i].alive:
+                nb_ = nbytes if rng.random() < 0.5 else min(nbytes, prefix[i] + chunk)
+                p.put(i, nb_)
+                prefix[i] = nb_
+        elif r < 0.58:
+            w = int(rng.integers(0, 2 * world))
+            p.each("fail", w)
+            p.o.fail(w)
+        elif r < 0.63 and not lost_rank and world > 2:
+            p.fail_rank(int(rng.integers(1, world)))             # never rank 0, where the output lives
+            lost_rank = True
+        elif r < 0.75 and joiners:
+            j = joiners.pop(0)
+            if p.o.objects[j].alive:
+                p.join(j)
+        else:
+            p.drive()
+        for rk in p.live:
+            assert p.c[rk].schedule_dump(T) == p.o.dump(T), "schedules differ"
+    for i in range(k):
+        if p.o.objects[i].alive:
+            t = max(t + 5, p.o.now)
+            p.advance(t)
+            p.put(i)
+    p.drive()
+    for oid in [T] + [500 + j for j in range(R)]:
+        ro, want = OK, None
+        try:
+            want = p.o.get(oid)
+        except StoreError as e:
+            ro = e.code
+        codes = {p.c[rk].try_get(oid)[0] for rk in p.live}
+        assert codes == {ro}, (oid, ro, codes)
+        if ro == OK:
+            got = p.target_bits(T).tobytes() if oid == T else p.dev[oid].cpu().numpy().tobytes()
+            assert got == want.tobytes(), f"object {oid} differs"
+    p.close()
+
+
+def test_pieces_are_counted_from_the_objects_first_chunk_not_the_tasks():
+    """A timeline that once gave wrong bits: tasks of one tree covered different chunk ranges, and a parent's piece was
+    released in the same level as the child's."""
+    _rank_timeline(1111)
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_random_timelines_on_emulated_ranks_match_the_oracle(block):
+    for seed in range(block * 30, (block + 1) * 30):
+        try:
+            _rank_timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
