@@ -158,3 +158,86 @@ def test_small_collectives_beside_a_polling_one_whose_wait_runs_out(seed):
     polling wave gives up: the wait that ran out must void exactly the pass that launched it and the later ones -- not
     the small collective planned before it, whose wave completed -- and must void all of its own pass."""
     _timeline(seed)
+
+
+def _tight_arena_timeline(seed):
+    """Several Reduces whose tree nodes keep their reduced objects, in an arena that holds the outputs and only a few
+    partial results: buffers are evicted and made again all the time.  Returns the number of evictions, or None when
+    even the pinned copies did not fit."""
+    rng = np.random.default_rng(seed)
+    n_ops = int(rng.integers(2, 6))
+    chunk = int(rng.choice([4096, 16384, 65536]))
+    elems = int(rng.integers(1, 5)) * (chunk // 4) + int(rng.choice([0, 3]))
+    S = elems * 4
+    fixed = 4096 * 32 + 256 * 32 + (64 << 10)
+    ks = [int(rng.integers(2, 9)) for _ in range(n_ops)]
+    room = n_ops + int(rng.integers(1, 6))                  # the outputs are pinned; a few more buffers for partial results
+    p = Pair(chunk, int(rng.integers(1, 4)), fuse=bool(rng.random() < 0.3), eager=bool(rng.random() < 0.3),
+             arena_bytes=fixed + room * (((S + 255) // 256) * 256 + 512))
+    oid, ops = 0, []
+    for q in range(n_ops):
+        ids = list(range(oid, oid + ks[q] + 1))
+        oid += ks[q] + 1
+        for i in ids:
+            p.create(i, i, gen(("smallint", 20) if seed % 2 else ("uniform",), 700 + seed, i, elems))
+        ops.append((1000 + q, ids))
+
+    def check(tgt, final):
+        ro, want = OK, None
+        try:
+            want = p.o.get(tgt)
+        except StoreError as e:
+            ro = e.code
+        rl, ptr, nb = p.c.try_get(tgt)
+        if rl == hpl.HPL_ERR_NOMEM:
+            raise hpl.HplError(rl, "hpl_get")
+        assert rl == ro, (tgt, ro, rl)
+        if ro == OK:
+            assert p.view(ptr, nb).cpu().numpy().tobytes() == want.tobytes(), f"target {tgt} differs"
+            if final:
+                p.check_schedule(tgt)
+
+    try:
+        for tgt, ids in ops:
+            p.reduce(tgt, ids, len(ids) - 1)                # one spare each
+        pend = [i for _, ids in ops for i in ids]
+        t = 0
+        for idx in rng.permutation(len(pend)):
+            i = pend[idx]
+            t += int(rng.integers(0, 10))
+            p.advance(t)
+            if rng.random() < 0.85:
+                p.put(i, S if rng.random() < 0.7 else min(S, chunk))
+            r = rng.random()
+            if r < 0.3:
+                p.progress()
+            elif r < 0.38 and p.o.objects[i].alive:
+                p.fail(i)
+            elif r < 0.5:
+                check(ops[int(rng.integers(0, n_ops))][0], False)
+        for _, ids in ops:
+            for i in ids:
+                if p.o.objects[i].alive:
+                    t += 1
+                    p.advance(t)
+                    p.put(i)
+        for tgt, _ in ops:
+            check(tgt, True)
+    except hpl.HplError as e:
+        if e.code != hpl.HPL_ERR_NOMEM:
+            raise
+        p.c.shutdown()
+        return None
+    ev = p.c.stats()["evictions"]
+    p.close()
+    return ev
+
+
+def test_random_timelines_in_arenas_too_small_for_all_partial_results():
+    evictions = 0
+    for seed in range(120):
+        try:
+            evictions += _tight_arena_timeline(seed) or 0
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
+    assert evictions > 50
