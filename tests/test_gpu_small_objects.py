@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import paper_2002_05814_b200 as hpl
-from oracle.store import DT_F32, DT_BF16
+from oracle.store import StoreError, OK, DT_F32, DT_BF16
 from tests.harness import Pair, gen
 
 pytestmark = pytest.mark.gpu
@@ -103,3 +103,81 @@ def test_small_reduce_with_a_failure_and_a_spare():
     p.check_target_bits(100)
     p.check_schedule(100)
     p.close()
+
+
+def _dag_timeline(seed):
+    """Up to a dozen collectives, most on small objects, some consuming others' outputs, some broadcast, requested before
+    any object exists; objects then arrive in random order (some partly, some never, some workers fail)."""
+    rng = np.random.default_rng(seed)
+    chunk = int(rng.choice([1024, 4096, 16384]))
+    elems = int(rng.integers(1, 4)) * (chunk // 4) + int(rng.choice([0, 0, 8]))
+    elems -= elems % 8
+    big = rng.random() < 0.25                      # sometimes above the threshold: mixes shared and own launches
+    if big:
+        elems = 24 * 1024
+    p = Pair(chunk, int(rng.integers(1, 5)), int(rng.integers(1, 3)), eager=bool(rng.random() < 0.25), fuse=bool(rng.random() < 0.7))
+    n_ops = int(rng.integers(3, 12))
+    oid, recv_id = 0, 5000
+    outputs, plain, receivers = [], [], []
+    def new_obj(bf):
+        nonlocal oid
+        i = oid
+        oid += 1
+        p.create(i, i, gen(("normal", 0.02), 800 + seed, i, elems, "bf16") if bf else gen(("uniform",), 800 + seed, i, elems))
+        plain.append(i)
+        return i
+    for q in range(n_ops):
+        bf = rng.random() < 0.3
+        n_src = int(rng.integers(1, 6))
+        srcs = [new_obj(bf) for _ in range(n_src)]
+        if not bf and outputs and rng.random() < 0.6:       # consume earlier outputs (fp32)
+            for o_ in rng.choice(outputs, size=min(len(outputs), int(rng.integers(1, 3))), replace=False):
+                if int(o_) not in srcs:
+                    srcs.append(int(o_))
+        tgt = 1000 + q
+        k = len(srcs) if rng.random() < 0.7 else int(rng.integers(1, len(srcs) + 1))
+        p.reduce(tgt, srcs, k, 0, DT_BF16 if bf else DT_F32)
+        outputs.append(tgt)
+        if rng.random() < 0.4:
+            dst = []
+            for _ in range(int(rng.integers(1, 4))):
+                p.create(recv_id, 900 + recv_id, nbytes=elems * 4, dtype=DT_F32)
+                dst.append(recv_id)
+                recv_id += 1
+            p.broadcast(tgt, dst)
+            receivers += dst
+            for d_ in dst:
+                if rng.random() < 0.8:
+                    p.join(d_)
+    t = 0
+    for i in rng.permutation(plain):
+        t += int(rng.integers(0, 5))
+        p.advance(t)
+        if rng.random() < 0.9 and p.o.objects[int(i)].alive:
+            p.put(int(i), None if rng.random() < 0.8 else min(chunk, p.host[int(i)].nbytes))
+        if rng.random() < 0.1:
+            p.progress()
+        if rng.random() < 0.05:
+            p.fail(int(rng.choice(plain)))
+    for oid_ in outputs + receivers:
+        ro = OK
+        try:
+            want = p.o.get(oid_)
+        except StoreError as e:
+            ro = e.code
+        rl, ptr, nb = p.c.try_get(oid_)
+        assert rl == ro, (oid_, ro, rl)
+        if ro == OK:
+            assert p.view(ptr, nb).cpu().numpy().tobytes() == want.tobytes(), f"object {oid_} differs"
+        t = max(t, p.o.now)
+        p.advance(t)
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_dags_of_small_collectives_match_the_oracle(block):
+    for seed in range(block * 40, (block + 1) * 40):
+        try:
+            _dag_timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
