@@ -217,7 +217,8 @@ int hpl_get(hpl_ctx* ctx, int64_t object_id, const void** dev_ptr, uint64_t* byt
 int hpl_get_host(hpl_ctx* ctx, int64_t object_id, void* dst, uint64_t cap);
 
 /* Takes a task worker out (Section 3.5): every object and receiver copy it owns leaves all trees at once;
- * its buffers are never read by work enqueued after the call.  Reduce: the next ready source takes the
+ * its buffers are never read by work enqueued after the call (what a broadcast copy of the worker can still serve
+ * to receivers that have joined is copied by work the call itself enqueues first).  Reduce: the next ready source takes the
  * position, ancestors' partial results are cleared; with no spare left the tree shrinks.  Broadcast: the
  * receivers it was sending to ask again and resume from what they hold. */
 int hpl_fail(hpl_ctx* ctx, int32_t worker);

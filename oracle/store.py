@@ -233,8 +233,10 @@ class OracleStore:
             src = self.dst_of[oid]
             sched: BroadcastSchedule = self.bcasts[src]["sched"]
             loc = sched.by_obj.get(oid)
-            if loc is None:
-                raise StoreError(ERR_TIMEOUT, "never joined")
+            if loc is None or not loc.alive:
+                # never asked, or its worker was rebuilt and has not asked again (Section 3.5.1: a rebuilt receiver
+                # fetches the object again as a new location; until then it holds no copy)
+                raise StoreError(ERR_TIMEOUT, "has not joined")
             # blocking on the copy = letting virtual time run until it has landed
             while not loc.complete and sched._heap:
                 sched.advance(sched._heap[0][0])

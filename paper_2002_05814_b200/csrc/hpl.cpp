@@ -767,6 +767,37 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
     for (auto& kv : c->objects)
         if (kv.second.worker == worker && kv.second.alive) lost.push_back(&kv.second);
     std::sort(lost.begin(), lost.end(), [](Object* a, Object* b) { return a->seq < b->seq; });
+    if (c->world <= 1 && !lost.empty()) {
+        // Copies are made lazily (at a Get, or at every event when eager), while in the schedule a receiver may already
+        // hold chunks it was sent before this instant.  What a copy that is about to disappear can still serve is
+        // therefore copied NOW, by work enqueued before the call returns: afterwards its buffer is never read again.
+        bool any = false;
+        for (auto& kv : c->bcasts) {
+            BcastOp& op = kv.second;
+            bool concerned = false;
+            for (Object* o : lost) concerned = concerned || o->id == op.src || (o->kind == OBJ_RECEIVER && o->op_key == op.src);
+            if (!concerned) continue;
+            if (!any) {
+                ++c->plan_pass;
+                int rc = flush_directory(c);
+                if (rc != HPL_OK) return rc;
+                if (c->device && c->copy_pending && !c->cfg.plan_ahead) {
+                    CUDA_TRY(cudaEventRecord(c->copy_ev, c->copy_stream));
+                    CUDA_TRY(cudaStreamWaitEvent(c->stream, c->copy_ev, 0));
+                    c->copy_pending = false;
+                    for (auto& ob : c->objects)
+                        if (ob.second.async_counter) ob.second.landed = published_chunks(c, ob.second);
+                }
+                any = true;
+            }
+            c->batch_tag = ++c->tag_counter;
+            std::vector<PlannedFanout> tasks;
+            int rc = plan_bcast(c, op, tasks);
+            if (rc != HPL_OK) return rc;
+            rc = launch_fanout_tasks(c, op, tasks);
+            if (rc != HPL_OK) return rc;
+        }
+    }
     for (Object* o : lost) o->alive = false;
     for (auto& kv : c->reduces) {
         ReduceOp& op = kv.second;
@@ -894,7 +925,9 @@ int hpl_get(hpl_ctx* c, int64_t id, const void** dev_ptr, uint64_t* bytes) {
         if (!o->alive) return HPL_ERR_FAILED_WORKER;
         BcastOp& op = c->bcasts.at(c->bcast_of_src.at(o->op_key));
         const int li = op.sched->index_of(id);
-        if (li < 0) return HPL_ERR_TIMEOUT;  // never joined
+        // never asked, or its worker was rebuilt and has not asked again (a rebuilt receiver holds no copy until it joins
+        // again as a new location, Section 3.5.1)
+        if (li < 0 || !op.sched->locations()[li].alive) return HPL_ERR_TIMEOUT;
         if (c->world <= 1 && (li >= (int)op.phys_have.size() || op.phys_have[li] < (int64_t)o->C)) {
             // start the copies first: the GPU works while the host lets the virtual clock run below
             int rc = progress(c);

@@ -5,7 +5,7 @@ import torch
 
 import paper_2002_05814_b200 as hpl
 import workloads as wl
-from oracle.store import DT_F32, DT_BF16
+from oracle.store import StoreError, OK, DT_F32, DT_BF16
 from tests.harness import Pair, gen
 
 pytestmark = pytest.mark.gpu
@@ -144,12 +144,141 @@ def test_rebuilt_receiver_asks_again():
     p.advance(1500)
     p.c.rejoin(2)
     p.o.rejoin(2)
+    # rebuilt, but it has not asked again: it holds no copy, although the copy it held before it failed was complete
+    from oracle.store import StoreError, ERR_TIMEOUT
+    with pytest.raises(StoreError) as ei:
+        p.o.get(2)
+    assert ei.value.code == ERR_TIMEOUT and p.c.try_get(2)[0] == hpl.HPL_ERR_TIMEOUT
     p.dev[2] = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     p.advance(1600)
     p.join(2)
     p.join(4)
     p.check_schedule(0)
     for j in (1, 2, 3, 4):
+        p.check_receiver_bytes(j)
+    p.check_schedule(0)
+    p.close()
+
+
+def _bcast_timeline(seed):
+    """One broadcast under random events: a source that is put in instalments (from the device or from host memory), staggered
+    joins, worker failures (the source's too), rebuilt workers that ask again or not, explicit progress, Gets in between."""
+    rng = np.random.default_rng(seed)
+    R, d, tau = int(rng.integers(1, 14)), int(rng.integers(1, 4)), int(rng.integers(1, 60))
+    chunk = int(rng.choice([4096, 16384, 65536]))
+    nbytes = int(rng.integers(1, 9)) * chunk + int(rng.choice([0, 0, 4, 1000, 4097]))
+    nbytes -= nbytes % 4
+    plan_ahead = bool(rng.random() < 0.3)
+    p = Pair(chunk, 2, d, tau=tau, eager=bool(rng.random() < 0.4), plan_ahead=plan_ahead, poll_budget_ns=3_000_000 if plan_ahead else 0)
+    nw = int(rng.integers(1, R + 2))
+    host_src = rng.random() < 0.3
+    data = gen(("uniform",), 900 + seed, 0, nbytes // 4)
+    srcw = int(rng.integers(0, nw)) if rng.random() < 0.2 else 99
+    if host_src:
+        p.host[0] = data
+        p.c.create(0, srcw, nbytes, DT_F32)
+        p.o.create(0, srcw, nbytes, DT_F32)
+    else:
+        p.create(0, srcw, data)
+    for j in range(1, R + 1):
+        p.create(j, int(rng.integers(0, nw)), nbytes=nbytes, dtype=DT_F32)
+    pref = 0
+
+    def put(nb):
+        if host_src:
+            p.c.put_host(0, p.host[0].ctypes.data, nb)
+            p.o.put(0, p.host[0], nb)
+        else:
+            p.put(0, nb)
+
+    if rng.random() < 0.5:
+        pref = nbytes if rng.random() < 0.6 else min(nbytes, int(rng.integers(0, nbytes // chunk + 1)) * chunk)
+        if pref:
+            put(pref)
+    p.broadcast(0, list(range(1, R + 1)))
+    joiners = list(rng.permutation(np.arange(1, R + 1)))
+    t = 0
+
+    def get(j):
+        nonlocal t
+        ro = OK
+        try:
+            want = p.o.get(j)
+        except StoreError as e:
+            ro = e.code
+        rl, ptr, nb = p.c.try_get(j)
+        if plan_ahead and ro == OK and rl == hpl.HPL_ERR_TIMEOUT:
+            p.c.sync()
+            rl, ptr, nb = p.c.try_get(j)
+        assert rl == ro, (j, ro, rl)
+        if ro == OK:
+            assert p.view(ptr, nb).cpu().numpy().tobytes() == want.tobytes(), f"receiver {j} differs"
+        t = max(t, p.o.now)
+        if plan_ahead:
+            p.c.sync()
+
+    for s in range(int(rng.integers(R, 4 * R + 6))):
+        t = max(t + int(rng.integers(0, 3 * tau)), p.o.now)
+        p.advance(t)
+        r = rng.random()
+        if r < 0.4 and joiners:
+            j = int(joiners.pop(0))
+            if p.o.objects[j].alive:
+                p.join(j)
+        elif r < 0.55 and pref < nbytes and p.o.objects[0].alive:
+            pref = nbytes if rng.random() < 0.5 else min(nbytes, pref + chunk)
+            put(pref)
+        elif r < 0.67:
+            p.fail(int(rng.integers(0, nw)))
+        elif r < 0.75:
+            wk = int(rng.integers(0, nw))
+            p.c.rejoin(wk)
+            p.o.rejoin(wk)
+            for j in range(1, R + 1):
+                if p.o.objects[j].worker == wk and j not in joiners and rng.random() < 0.7:
+                    joiners.append(j)
+        elif r < 0.85:
+            p.progress()
+        else:
+            get(int(rng.integers(1, R + 1)))
+        p.check_schedule(0)
+    if pref < nbytes and p.o.objects[0].alive:
+        t = max(t + 1, p.o.now)
+        p.advance(t)
+        put(nbytes)
+    for j in range(1, R + 1):
+        get(j)
+        p.check_schedule(0)
+    if plan_ahead:
+        p.c.sync()
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_broadcast_timelines_match_the_oracle(block):
+    for seed in range(block * 40, (block + 1) * 40):
+        try:
+            _bcast_timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
+
+
+def test_receivers_keep_what_the_schedule_gave_them_when_the_source_is_lost_before_any_copy_ran():
+    """Copies are made lazily; in the schedule the receivers had the whole object when the source's worker failed.  The
+    failure itself enqueues the copies that copy can still serve."""
+    nbytes, chunk = 5 * 4096 + 8, 4096
+    p = Pair(chunk, 2, 2, tau=10)
+    p.create(0, 7, gen(("uniform",), 12, 0, nbytes // 4))
+    for j in (1, 2, 3):
+        p.create(j, 10 + j, nbytes=nbytes, dtype=DT_F32)
+    p.put(0)
+    p.broadcast(0, [1, 2, 3])
+    for j in (1, 2, 3):
+        p.join(j)
+    p.advance(100_000)                                  # every transfer of the schedule has landed; nothing has run yet
+    assert p.c.stats()["kernel_launches"] == 0
+    p.fail(7)
+    for j in (1, 2, 3):
         p.check_receiver_bytes(j)
     p.check_schedule(0)
     p.close()

@@ -181,3 +181,29 @@ def test_store_broadcast_bytes_and_blocking_get():
         assert got.tobytes() == data.tobytes()
     w = st.dump(0)
     assert w[0] == 0x48504C42 and w[6] == 3
+
+
+def test_a_rebuilt_receiver_holds_nothing_until_it_asks_again():
+    """Section 3.5.1: a receiver whose worker failed and was rebuilt fetches the object again, as a new location.  Between
+    the rebuild and that second request it holds no copy -- even if the copy it had before the failure was complete."""
+    from oracle.store import OracleStore, StoreError, ERR_TIMEOUT, ERR_FAILED_WORKER, DT_F32
+    st = OracleStore(64, 2, 1, 10)
+    data = np.arange(64, dtype=np.float32)                 # 256 bytes = 4 chunks
+    st.create(0, 9, 256, DT_F32)
+    st.create(1, 1, 256, DT_F32)
+    st.put(0, data, 256)
+    st.broadcast(0, [1])
+    st.join(1)
+    assert st.get(1).tobytes() == data.tobytes()           # complete (the Get lets virtual time run)
+    st.advance(st.now + 5)
+    st.fail(1)
+    with pytest.raises(StoreError) as ei:
+        st.get(1)
+    assert ei.value.code == ERR_FAILED_WORKER
+    st.rejoin(1)
+    with pytest.raises(StoreError) as ei:
+        st.get(1)
+    assert ei.value.code == ERR_TIMEOUT                    # rebuilt, not asked again
+    st.join(1)
+    assert st.get(1).tobytes() == data.tobytes()           # a new location, fetched again from the start
+    assert [l.obj for l in st.bcasts[0]["sched"].locs] == [0, 1, 1]
