@@ -207,8 +207,9 @@ class OracleStore:
             self.reduces.pop(oid)
         if oid in self.bcasts:
             b = self.bcasts.pop(oid)
-            for dd in b["dsts"]:
+            for dd in b["dsts"]:      # Delete removes every copy of the object (Table 1): the receivers' copies go with it
                 self.dst_of.pop(dd, None)
+                self.objects.pop(dd, None)
 
     def get(self, oid: int) -> np.ndarray:
         """The complete object (read-only), or StoreError(ERR_TIMEOUT) if it cannot complete yet."""

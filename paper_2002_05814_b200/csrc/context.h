@@ -335,7 +335,7 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
 int ensure_partial_buffer(hpl_ctx* c, ReduceOp& op, int pos, Object** out);
 int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks);
 int launch_reduce_group(hpl_ctx* c, std::vector<std::pair<ReduceOp*, PlannedReduceTask*>>& group, bool bf16);
-void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv);
+void apply_invalidation(hpl_ctx* c, ReduceOp& op, const ReduceInvalidation& inv);
 
 // plan_bcast.cpp
 int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks);

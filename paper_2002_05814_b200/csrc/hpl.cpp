@@ -806,7 +806,7 @@ int hpl_fail(hpl_ctx* c, int32_t worker) {
         for (Object* o : lost) {
             if (!op.sched->has_source(o->id)) continue;
             ReduceInvalidation inv = op.sched->fail(o->id, logical_delivered_in(c, o->id, op), dl);
-            apply_invalidation(op, inv);
+            apply_invalidation(c, op, inv);
             if (!inv.positions.empty() || inv.shrank) invalidate_consumers(c, op.target);
         }
     }
@@ -1161,7 +1161,7 @@ int hpl_fail_rank(hpl_ctx* c, int32_t rank) {
             inv.touched.push_back(p);
         }
         if (!inv.touched.empty()) {
-            apply_invalidation(op, inv);
+            apply_invalidation(c, op, inv);
             invalidate_consumers(c, op.target);
         }
     }

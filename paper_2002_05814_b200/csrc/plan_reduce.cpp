@@ -433,10 +433,24 @@ int launch_reduce_tasks(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>
 // A position's own object changed, or the position disappeared: its buffer is void, and so is, in every
 // ancestor, whatever was merged from the child on that path onwards.  What an ancestor had merged BEFORE that
 // child (its earlier operands) is untouched and kept -- healthy chunks are not redone.
-void apply_invalidation(ReduceOp& op, const ReduceInvalidation& inv) {
+void apply_invalidation(hpl_ctx* c, ReduceOp& op, const ReduceInvalidation& inv) {
     const int k = op.sched->k();
     ReduceTreeSchedule& s = *op.sched;
     if (inv.shrank) {
+        // the positions that disappeared give their buffers back (once nothing enqueued can still read them)
+        bool waited = false;
+        for (int q = k; q < (int)op.partial_key.size(); ++q) {
+            if (op.partial_key[q] == 0) continue;
+            Object* po = find(c, op.partial_key[q]);
+            if (!po) continue;
+            if (!waited && c->device && (c->work_in_flight || c->copy_pending)) {
+                cudaStreamSynchronize(c->copy_stream);
+                cudaStreamSynchronize(c->stream);
+                waited = true;
+            }
+            release_object_memory(c, *po);
+            c->objects.erase(op.partial_key[q]);
+        }
         op.merged.resize(k);
         op.partial_key.resize(k, 0);
     }

@@ -1,0 +1,136 @@
+"""Rounds on one context: objects are deleted and their ids, directory rows and arena blocks used again."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_05814_b200 as hpl
+from oracle.store import StoreError, OK, DT_F32, DT_BF16
+from tests.harness import Pair, gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2002_05814_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _rounds_timeline(seed):
+    """Several rounds on ONE context: each a small random DAG of collectives (composed, broadcast, min / max, partly
+    arriving sources, failures), checked against the oracle, then deleted -- ids, directory rows and arena blocks are
+    used again by the next round, and the arena must be back to its base level after every round."""
+    rng = np.random.default_rng(seed)
+    chunk = int(rng.choice([4096, 16384, 65536]))
+    p = Pair(chunk, int(rng.integers(1, 5)), int(rng.integers(1, 3)), tau=int(rng.integers(1, 40)),
+             eager=bool(rng.random() < 0.3), fuse=bool(rng.random() < 0.6), fuse_fanout=bool(rng.random() < 0.7))
+    base = None
+    tclock = 0
+    for rnd in range(int(rng.integers(2, 6))):
+        elems = int(rng.integers(1, 4)) * (chunk // 4) + int(rng.choice([0, 0, 8, 1000]))
+        elems -= elems % 8
+        n_ops = int(rng.integers(1, 6))
+        oid, recv_id = 0, 5000
+        outputs, plain, receivers = [], [], []
+
+        def new_obj(bf):
+            nonlocal oid
+            i = oid
+            oid += 1
+            p.create(i, i, gen(("normal", 0.02), 950 + seed + rnd, i, elems, "bf16") if bf else gen(("uniform",), 950 + seed + rnd, i, elems))
+            plain.append(i)
+            return i
+
+        for q in range(n_ops):
+            bf = rng.random() < 0.3
+            srcs = [new_obj(bf) for _ in range(int(rng.integers(1, 6)))]
+            if not bf and outputs and rng.random() < 0.5:
+                srcs.append(int(rng.choice(outputs)))
+            tgt = 1000 + q
+            p.reduce(tgt, srcs, len(srcs) if rng.random() < 0.7 else int(rng.integers(1, len(srcs) + 1)),
+                     int(rng.choice([0, 0, 1, 2])) if not bf else 0, DT_BF16 if bf else DT_F32)
+            outputs.append(tgt)
+            if rng.random() < 0.4:
+                dst = []
+                for _ in range(int(rng.integers(1, 4))):
+                    p.create(recv_id, 900 + recv_id, nbytes=elems * 4, dtype=DT_F32)
+                    dst.append(recv_id)
+                    recv_id += 1
+                p.broadcast(tgt, dst)
+                receivers += dst
+                for d_ in dst:
+                    if rng.random() < 0.8:
+                        p.join(d_)
+        for i in rng.permutation(plain):
+            tclock = max(tclock + int(rng.integers(0, 5)), p.o.now)
+            p.advance(tclock)
+            if rng.random() < 0.9 and p.o.objects[int(i)].alive:
+                p.put(int(i), None if rng.random() < 0.8 else min(chunk, p.host[int(i)].nbytes))
+            if rng.random() < 0.1:
+                p.progress()
+            if rng.random() < 0.05:
+                p.fail(int(rng.choice(plain)))
+        for oid_ in outputs + receivers:
+            ro = OK
+            try:
+                want = p.o.get(oid_)
+            except StoreError as e:
+                ro = e.code
+            rl, ptr, nb = p.c.try_get(oid_)
+            assert rl == ro, (rnd, oid_, ro, rl)
+            if ro == OK:
+                assert p.view(ptr, nb).cpu().numpy().tobytes() == want.tobytes(), f"round {rnd} object {oid_} differs"
+            tclock = max(tclock, p.o.now)
+            p.advance(tclock)
+        # the round's objects go: consumers before what they consume
+        for tgt in reversed(outputs):
+            p.c.delete(tgt)
+            p.o.delete(tgt)
+        for i in plain:
+            p.c.delete(i)
+            p.o.delete(i)
+        # receivers went with their broadcasts; immutability / canaries are checked at the end for what is still known
+        for i in plain + receivers:
+            p.host.pop(i, None)
+            p.dev.pop(i, None)
+            p.guarded.pop(i, None)
+        used = p.c.stats()["arena_used"]
+        if base is None:
+            base = used
+        assert used == base, ("arena not returned", rnd, used, base)
+        tclock += 1000
+        p.advance(tclock)
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_rounds_with_deletes_match_the_oracle_and_return_the_arena(block):
+    for seed in range(block * 30, (block + 1) * 30):
+        try:
+            _rounds_timeline(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
+
+
+def test_positions_that_a_shrinking_tree_loses_give_their_buffers_back():
+    """Every tree node keeps its reduced object (fuse = 0); members fail until the tree has shrunk to two positions; after the
+    Deletes the arena is where it was."""
+    p = Pair(16 << 10, 2, fuse=False)
+    base = p.c.stats()["arena_used"]
+    for i in range(8):
+        p.create(i, i, gen(("uniform",), 990, i, 3 * 4096 + 5))
+        p.put(i)
+    p.reduce(100, list(range(8)), 8)
+    p.check_target_bits(100)
+    assert p.c.stats()["arena_used"] > base
+    for t, w in enumerate((7, 6, 5, 4, 3, 2)):
+        p.advance(10 + t)
+        p.fail(w)
+        p.check_target_bits(100)
+    p.check_schedule(100)
+    for i in [100] + list(range(8)):
+        p.c.delete(i)
+        p.o.delete(i)
+    assert p.c.stats()["arena_used"] == base
+    p.close()
