@@ -14,6 +14,7 @@
 #include <dlfcn.h>
 
 #include <mutex>
+#include <set>
 
 using namespace hpl;
 
@@ -237,11 +238,34 @@ int progress(hpl_ctx* c) {
     return flush_small(c, sb);
 }
 
-// Voids what was planned by the passes whose waves have seq >= from_tag (a wave of that pass gave up, and
-// later passes may have built on it); earlier passes ran to completion and are kept.
-void undo_journal(hpl_ctx* c, uint64_t from_tag) {
+// A wave gave up.  Void: what its own planning pass had planned (tags in `failed`), whatever later passes planned
+// for the same collectives (they may have continued in place from a buffer the wave left half updated), and whatever
+// was planned since for collectives that consume their outputs, directly or not.  Collectives that have nothing to do
+// with them keep their work: their waves ran to completion.  `everything`: the failed wave could not be told apart
+// (more waves in flight than error records), so all passes from `from_tag` on are void.
+void undo_journal(hpl_ctx* c, uint64_t from_tag, const std::set<uint64_t>& failed, bool everything) {
+    std::set<int64_t> void_targets, void_srcs;
+    for (auto& e : c->journal.r)
+        if (everything ? e.tag >= from_tag : failed.count(e.tag) != 0) void_targets.insert(e.target);
+    for (auto& e : c->journal.b)
+        if (everything ? e.tag >= from_tag : failed.count(e.tag) != 0) void_srcs.insert(e.src);
+    for (bool grew = true; grew;) {
+        grew = false;
+        for (auto& kv : c->reduces) {
+            ReduceOp& op = kv.second;
+            if (void_targets.count(op.target)) continue;
+            for (int64_t sid : op.sched->sources())
+                if (void_targets.count(sid)) {
+                    void_targets.insert(op.target);
+                    grew = true;
+                    break;
+                }
+        }
+    }
+    for (auto& kv : c->bcasts)
+        if (void_targets.count(kv.second.src)) void_srcs.insert(kv.second.src);
     for (auto& e : c->journal.r) {
-        if (e.tag < from_tag) continue;
+        if (e.tag < from_tag || !void_targets.count(e.target)) continue;
         auto it = c->reduce_of_target.find(e.target);
         if (it == c->reduce_of_target.end()) continue;
         ReduceOp& op = c->reduces.at(it->second);
@@ -250,13 +274,13 @@ void undo_journal(hpl_ctx* c, uint64_t from_tag) {
         if (e.pos < (int)op.merged.size()) op.merged[e.pos].set(e.a, e.b, 0);
     }
     for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
-        if (it->tag < from_tag) continue;
+        if (it->tag < from_tag || !void_srcs.count(it->src)) continue;
         auto f = c->bcast_of_src.find(it->src);
         if (f == c->bcast_of_src.end()) continue;
         BcastOp& op = c->bcasts.at(f->second);
         if (it->loc < (int)op.phys_have.size()) op.phys_have[it->loc] = it->old_have;
     }
-    c->journal.clear();
+    c->journal.clear();   // everything in flight has been waited for: what was not voided is confirmed
 }
 
 int sync_and_check(hpl_ctx* c) {
@@ -292,8 +316,9 @@ int sync_and_check(hpl_ctx* c) {
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->work_in_flight = false;
     collect_kernel_times(c);
-    bool failed = false;
+    bool failed = false, ambiguous = false;
     uint64_t from_tag = ~0ull;
+    std::set<uint64_t> failed_tags;
     for (uint32_t i = 0; i < used; ++i) {
         c->stats.device_waits += c->h_status[i].waits;
         if (!c->h_status[i].error) continue;
@@ -302,6 +327,8 @@ int sync_and_check(hpl_ctx* c) {
         // the record in the last slot may stand for several waves: the earliest of them decides
         const uint64_t tag = c->wave_tag[i];
         from_tag = std::min(from_tag, tag);
+        failed_tags.insert(tag);
+        if (i == kStatusSlots - 1 && c->launch_seq - c->first_unchecked > kStatusSlots) ambiguous = true;
     }
     c->first_unchecked = c->launch_seq;
     c->wave_tag.clear();
@@ -310,7 +337,7 @@ int sync_and_check(hpl_ctx* c) {
     CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(DeviceStatus) * used, c->stream));
     if (failed) {
         c->stats.device_timeouts++;
-        undo_journal(c, from_tag);
+        undo_journal(c, from_tag, failed_tags, ambiguous);
         return HPL_ERR_TIMEOUT;
     }
     c->journal.clear();

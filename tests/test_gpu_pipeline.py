@@ -303,3 +303,32 @@ def test_partial_results_are_evicted_least_recently_used_when_the_arena_is_full(
     assert p.c.stats()["evictions"] > ev
     p.check_target_bits(200)                                # outputs were never touched
     p.close()
+
+
+def test_a_wait_that_runs_out_voids_its_own_collective_and_its_consumers_only():
+    """plan_ahead: Reduce A waits for chunks of an object that never come; Reduce C consumes A's output; Reduce B, requested
+    after both, has nothing to do with them.  Every Get plans A again and A's wave gives up again -- B's result, computed
+    once, stands and is returned; C cannot complete; when the object finally arrives everything completes."""
+    elems, chunk = 6 * 4096, 16 << 10
+    p = Pair(chunk, 2, plan_ahead=True, poll_budget_ns=2_000_000)
+    for i in range(6):
+        p.create(i, i, gen(("uniform",), 82, i, elems))
+    p.reduce(100, [0, 1], 2)                       # A
+    p.reduce(300, [100, 2], 2)                     # C consumes A
+    p.reduce(200, [3, 4, 5], 3)                    # B, independent
+    p.put(0)
+    p.put(1, chunk)                                # published, one chunk of six valid: A's wave will wait for the rest
+    for i in (2, 3, 4, 5):
+        p.put(i)
+    p.check_target_bits(200)                       # B completes although A's wave runs out in the same pass
+    launches = p.c.stats()["kernel_launches"]
+    for _ in range(3):
+        assert p.c.try_get(100)[0] == hpl.HPL_ERR_TIMEOUT and p.c.try_get(300)[0] == hpl.HPL_ERR_TIMEOUT
+        p.check_target_bits(200)                   # ... and is not computed again
+    st = p.c.stats()
+    assert st["device_timeouts"] >= 3
+    p.put(1)
+    p.check_target_bits(100)
+    p.check_target_bits(300)
+    p.check_target_bits(200)
+    p.close()
