@@ -34,6 +34,9 @@ import workloads as wl  # noqa: E402
 
 MiB = 1 << 20
 FALLBACK_HBM_GBS = 6650.0
+# the headline value is effective GB/s = algorithmic bytes / time of the default workload; the curve against object size
+# and the fractions of the HBM peak are in the same line (`sweep`, `frac_of_hbm_peak`, `roofline`)
+METRIC = "reduce/broadcast effective GB/s and fraction of HBM peak vs object size, 1 B200"
 
 KERNEL_SOURCES = ("paper_2002_05814_b200/csrc/kernels.cu", "paper_2002_05814_b200/csrc/device_types.h")
 
@@ -897,7 +900,7 @@ def main():
         if rank != 0:
             return
         value, sample, ms = oracle_sample(w, budget_s=min(60.0, max(5.0, 4.0 * (args.steps + args.warmup))))
-        line = {"impl": "reference", "metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value,
+        line = {"impl": "reference", "metric": METRIC, "value": value,
                 "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": config, "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
@@ -951,7 +954,7 @@ def main():
     traf = {k: ncu_traffic(w.name, k) for k in ("reduce", "fanout")} if args.shrink == 1 else {}
     r_red = roof("reduce_kernel_ns", "reduce_launches", ab["reduce"] * k_steps / max(1, st["reduce_launches"]), traf.get("reduce")) if ab["reduce"] else None
     r_fan = roof("fanout_kernel_ns", "fanout_launches", ab["broadcast"] * k_steps / max(1, st["fanout_launches"]), traf.get("fanout")) if ab["broadcast"] else None
-    line = {"metric": "reduce/broadcast effective GB/s (algorithmic bytes / time)", "value": value, "unit": "GB/s",
+    line = {"metric": METRIC, "value": value, "unit": "GB/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if w.dtype == "f32" else "f32 (bf16 inputs widened)", "data": "synthetic",
