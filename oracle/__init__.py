@@ -30,7 +30,7 @@ orphans of one failure ask again, and the way a prefix crosses dtypes in compose
 are build-defined readings.  Each is held to a hand-worked example under ``tests/golden/``
 (``reduce_shrink_example``, ``broadcast_two_slots_example``, ``broadcast_orphans_example``,
 ``composition_cross_dtype``; ``tests/test_golden_rules.py``) besides the invariants and
-brute-force value checks in ``tests/test_oracle_*.py``.  One rule stays **parity unpinned**:
-the order in which SEVERAL waiting receivers are served -- no timeline was found in which two
-receivers wait at once (a second orphan can always fetch from the first).
+brute-force value checks in ``tests/test_oracle_*.py``.  The order in which SEVERAL waiting receivers would be served is not pinned because it cannot be
+observed: at most one receiver ever waits (a second one could fetch from the first), which
+``tests/test_oracle_broadcast.py`` checks over random timelines.
 """

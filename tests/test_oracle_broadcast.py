@@ -207,3 +207,38 @@ def test_a_rebuilt_receiver_holds_nothing_until_it_asks_again():
     st.join(1)
     assert st.get(1).tobytes() == data.tobytes()           # a new location, fetched again from the start
     assert [l.obj for l in st.bcasts[0]["sched"].locs] == [0, 1, 1]
+
+
+def test_at_most_one_receiver_ever_waits():
+    """Why the serving order among SEVERAL waiting receivers cannot be pinned: it cannot be observed.  A receiver waits only
+    when no live location outside its own subtree has a free slot; a second receiver in that state could fetch from the
+    first (a fresh receiver has all its slots), so two never wait at once -- checked here over random timelines in which
+    the source, too, may fail, receivers fail in groups and are rebuilt."""
+    rng = np.random.default_rng(47)
+    most = 0
+    for trial in range(600):
+        C, d, tau, R = int(rng.integers(1, 10)), int(rng.integers(1, 4)), int(rng.integers(1, 20)), int(rng.integers(2, 14))
+        b = BroadcastSchedule(0, C, d, tau)
+        b.source_progress(0, int(rng.integers(0, C + 1)))
+        t = 0
+        alive = {j: True for j in range(0, R + 1)}
+        for _ in range(int(rng.integers(R, 5 * R))):
+            t += int(rng.integers(0, 3 * tau))
+            r = rng.random()
+            if r < 0.5:
+                j = int(rng.integers(1, R + 1))
+                if alive[j]:
+                    b.join(t, j)
+            elif r < 0.75:
+                group = [int(x) for x in rng.choice(np.arange(0, R + 1), size=int(rng.integers(1, 4)), replace=False)]
+                b.fail(t, group)
+                for j in group:
+                    alive[j] = False
+            elif r < 0.85:
+                j = int(rng.integers(1, R + 1))
+                alive[j] = True                      # rebuilt: it may ask again (a new location)
+            else:
+                b.source_progress(t, C)
+            most = max(most, len(b.waiting))
+            assert len(b.waiting) <= 1, (trial, [w.obj for w in b.waiting])
+    assert most == 1                                 # ... and one does wait in some of them
