@@ -314,7 +314,10 @@ const char* hpl_strerror(int code);
  *     left, hpl_progress is called again (receivers further down a broadcast tree are served by the next plan) until
  *     it plans nothing.  hpl_get does not drive this loop: it returns HPL_ERR_TIMEOUT until the object is done.
  *     While levels are pending, hpl_fail, hpl_rejoin, hpl_fail_rank and hpl_delete return HPL_ERR_INVALID: trees
- *     change and memory is recycled between plans, not inside one.
+ *     change and memory is recycled between plans, not inside one.  Bytes move only when the caller drives the levels:
+ *     hpl_fail cannot first copy what a disappearing broadcast copy could still serve (as it does on one GPU), so a
+ *     receiver that the schedule had given chunks which were never moved cannot complete from that copy afterwards
+ *     -- drive the pending plan before taking a worker out.
  * plan_ahead, eager and hpl_put_host are not available in this mode (HPL_ERR_INVALID).  A rank that is lost is taken
  * out with hpl_fail_rank on every survivor: its workers fail (Section 3.5), and what lived on it is re-made
  * elsewhere; a Reduce whose output lived there is lost (HPL_ERR_FAILED_WORKER). */

@@ -313,3 +313,97 @@ def test_random_timelines_on_emulated_ranks_match_the_oracle(block):
             _rank_timeline(seed)
         except AssertionError as e:
             raise AssertionError(f"seed {seed}: {e}") from e
+
+
+def _rank_timeline_composed(seed):
+    """As above with more of the path: a bf16 or fp32 Reduce whose output feeds a second Reduce whose output is broadcast, and
+    a plain object broadcast through its own tree.  A worker or a rank is taken out only after the pending levels have been
+    driven (in this mode bytes move when the caller drives; what a copy could still serve must have moved before it goes)."""
+    from oracle.store import StoreError, OK
+    rng = np.random.default_rng(seed)
+    world = int(rng.integers(2, 5))
+    k, kb, R = int(rng.integers(2, 8)), int(rng.integers(1, 4)), int(rng.integers(1, 5))
+    d = int(rng.integers(1, 4))
+    chunk = int(rng.choice([4096, 16384]))
+    elems = int(rng.integers(1, 6)) * (chunk // 4) + int(rng.choice([0, 0, 8, 1000]))
+    elems -= elems % 8
+    bf = bool(rng.random() < 0.35)
+    p = Ranks(world, chunk, d, bool(rng.random() < 0.5), arena_bytes=16 << 20, pipeline_chunks=int(rng.choice([0, 0, 1, 2, 3])))
+    T = 1000 - 1000 % world                                     # both outputs live on rank 0, which is never lost here
+    B = T + world
+    nbytes = elems * 4
+    for i in range(k):
+        p.create(i, int(rng.integers(0, 2 * world)),
+                 gen(("normal", 0.02), 650 + seed, i, elems, "bf16") if bf else gen(("uniform",), 650 + seed, i, elems))
+    for i in range(k, k + kb):
+        p.create(i, int(rng.integers(0, 2 * world)), gen(("uniform",), 650 + seed, i, elems))
+    X = k + kb
+    p.create(X, int(rng.integers(0, 2 * world)), gen(("uniform",), 650 + seed, X, elems))
+    for j in range(R):
+        p.create(500 + j, int(rng.integers(0, 2 * world)), nbytes=nbytes)
+        p.create(600 + j, int(rng.integers(0, 2 * world)), nbytes=nbytes)
+    n_all = X + 1
+    p.reduce(T, list(range(k)), int(rng.integers(1, k + 1)), DT_BF16 if bf else DT_F32)
+    p.reduce(B, [T] + list(range(k, k + kb)), int(rng.integers(1, kb + 2)))
+    p.broadcast(B, [500 + j for j in range(R)])
+    p.broadcast(X, [600 + j for j in range(R)])
+    size = {i: p.host[i].nbytes for i in range(n_all)}
+    prefix = {i: 0 for i in range(n_all)}
+    joiners = [500 + j for j in range(R)] + [600 + j for j in range(R)]
+    rng.shuffle(joiners)
+    lost_rank = False
+    t = 0
+    for _ in range(int(rng.integers(2 * n_all, 5 * n_all + 6))):
+        t = max(t + int(rng.integers(0, 40)), p.o.now)
+        p.advance(t)
+        r = rng.random()
+        if r < 0.5:
+            i = int(rng.integers(0, n_all))
+            if p.o.objects[i].alive:
+                nb_ = size[i] if rng.random() < 0.5 else min(size[i], prefix[i] + chunk)
+                p.put(i, nb_)
+                prefix[i] = nb_
+        elif r < 0.57:
+            w = int(rng.integers(0, 2 * world))
+            p.drive()
+            p.each("fail", w)
+            p.o.fail(w)
+        elif r < 0.62 and not lost_rank and world > 2:
+            p.drive()
+            p.fail_rank(int(rng.integers(1, world)))
+            lost_rank = True
+        elif r < 0.78 and joiners:
+            j = joiners.pop(0)
+            if p.o.objects[j].alive:
+                p.join(j)
+        else:
+            p.drive()
+        for rk in p.live:
+            assert p.c[rk].schedule_dump(T) == p.o.dump(T) and p.c[rk].schedule_dump(B) == p.o.dump(B), "schedules differ"
+    for i in range(n_all):
+        if p.o.objects[i].alive:
+            t = max(t + 5, p.o.now)
+            p.advance(t)
+            p.put(i)
+    p.drive()
+    for oid in [T, B] + [500 + j for j in range(R)] + [600 + j for j in range(R)]:
+        ro, want = OK, None
+        try:
+            want = p.o.get(oid)
+        except StoreError as e:
+            ro = e.code
+        codes = {p.c[rk].try_get(oid)[0] for rk in p.live}
+        assert codes == {ro}, (oid, ro, codes)
+        if ro == OK:
+            got = p.target_bits(oid).tobytes() if oid in (T, B) else p.dev[oid].cpu().numpy().tobytes()
+            assert got == want.tobytes(), f"object {oid} differs"
+    p.close()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_random_composed_timelines_on_emulated_ranks_match_the_oracle(block):
+    for seed in range(block * 30, (block + 1) * 30):
+        try:
+            _rank_timeline_composed(seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from e
