@@ -9,6 +9,7 @@
 #include <cstring>
 #include <map>
 #include <memory>
+#include <set>
 #include <unordered_map>
 #include <vector>
 
@@ -260,6 +261,7 @@ struct hpl_ctx {
     std::map<uint64_t, ReduceOp> reduces;  // by creation order
     std::map<uint64_t, BcastOp> bcasts;
     std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
+    std::set<uint64_t> composed_bcasts;   // keys of the broadcasts whose source is a Reduce output, in creation order
     std::unordered_map<int64_t, std::vector<uint64_t>> reduces_of_source;   // source id -> the Reduces that name it (keys of `reduces`)
     Journal journal;
     bool work_in_flight = false;

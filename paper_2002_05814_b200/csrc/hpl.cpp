@@ -348,9 +348,9 @@ int after_event(hpl_ctx* c) { return c->cfg.eager ? progress(c) : HPL_OK; }
 
 // After every event: a broadcast whose source is a Reduce output learns how far that output has got.
 void refresh_composed(hpl_ctx* c) {
-    for (auto& kv : c->bcasts) {
-        Object* src = find(c, kv.second.src);
-        if (src && src->kind == OBJ_TARGET) kv.second.sched->source_progress((int64_t)c->now, logical_delivered(c, src->id));
+    for (uint64_t key : c->composed_bcasts) {   // only those: a Put must not cost time in proportion to all broadcasts
+        BcastOp& op = c->bcasts.at(key);
+        op.sched->source_progress((int64_t)c->now, logical_delivered(c, op.src));
     }
 }
 
@@ -763,6 +763,7 @@ int hpl_broadcast(hpl_ctx* c, int64_t src_id, const int64_t* dst_ids, int32_t n)
     }
     c->bcast_of_src[src_id] = b.seq;
     const uint64_t key = b.seq;
+    if (src->kind == OBJ_TARGET) c->composed_bcasts.insert(key);   // an object's kind never changes while it is a source
     c->bcasts.emplace(key, std::move(b));
     return after_event(c);
 }
@@ -1109,6 +1110,7 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
                 c->objects.erase(d);
             }
         }
+        c->composed_bcasts.erase(b->second);
         c->bcasts.erase(b->second);
         c->bcast_of_src.erase(b);
     }

@@ -90,6 +90,10 @@ class Pair:
     def progress(self):
         self.c.progress()
 
+    def delete(self, oid):
+        self.c.delete(oid)
+        self.o.delete(oid)
+
     def view(self, ptr, nbytes) -> torch.Tensor:
         """Bytes at a device pointer that lies in the arena or in one of the buffers given to the library."""
         base = self.arena.data_ptr()

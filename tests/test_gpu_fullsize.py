@@ -228,3 +228,50 @@ def test_cfg5_fault_tolerant_reduce(size):
     assert sorted(obj_at) == [i for i in range(32) if i != 7]
     _check_reduce_windows(w, obj_at, seeds, out, np.random.default_rng(3))
     c.shutdown()
+
+
+def test_objects_beyond_four_gib():
+    """Byte offsets past 2^32 and element indices past 2^30: a Reduce over three 5 GiB objects with a ragged last chunk,
+    its output broadcast to two receivers; windows around the 4 GiB mark and the tail against the oracle."""
+    import dataclasses
+    base = wl.workload("cfg3")
+    elems = (5 << 30) // 4 + 1000
+    w = dataclasses.replace(base, elems=elems, degree=2)
+    S = w.object_bytes
+    arena, c = _ctx(w, (64 << 20) + S)
+    sh = Shadow(w)
+    seeds = {i: w.seed + i for i in range(3)}
+    dev = [wl.values_torch(w.dist, seeds[i], i, 0, elems, "f32") for i in range(3)]
+    recv = [torch.zeros(elems, dtype=torch.float32, device="cuda") for _ in range(2)]
+    for i in range(3):
+        c.create(i, i, S)
+        sh.o.create(i, i, S, DT_F32)
+        c.put(i, dev[i].data_ptr(), S)
+        sh.o.put(i, sh.placeholder(S, DT_F32), S)
+    c.reduce(100, [0, 1, 2], 3)
+    sh.o.reduce(100, [0, 1, 2], 3)
+    for j in range(2):
+        c.create(200 + j, 10 + j, S)
+        sh.o.create(200 + j, 10 + j, S, DT_F32)
+    c.broadcast(100, [200, 201])
+    sh.o.broadcast(100, [200, 201])
+    for j in range(2):
+        c.join(200 + j, recv[j].data_ptr())
+        sh.o.join(200 + j)
+    ptr, n = c.get(100)
+    for j in range(2):
+        c.get(200 + j)
+    assert n == S and c.schedule_dump(100) == sh.o.dump(100)
+    off = ptr - arena.data_ptr()
+    out = arena[off:off + n].view(torch.float32)
+    obj_at = sh.o.reduces[100]["sched"].obj_at
+    chunk_elems = w.chunk_bytes // 4
+    mark = (1 << 32) // 4                                            # the element at byte offset 2^32
+    for lo, hi in [(mark - 3000, mark + 3000), (elems - 5000, elems), (0, 5000),
+                   ((elems - 1) // chunk_elems * chunk_elems - 64, elems)]:
+        objs = {o: wl.values_np(w.dist, seeds[o], o, lo, hi - lo) for o in obj_at}
+        want = ov.tree_reduce(obj_at, w.degree, objs)
+        assert np.array_equal(out[lo:hi].cpu().numpy().view(np.uint32), want.view(np.uint32)), (lo, hi)
+    for j in range(2):
+        assert torch.equal(recv[j].view(torch.int32), out.view(torch.int32))
+    c.shutdown()

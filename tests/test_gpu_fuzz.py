@@ -48,6 +48,7 @@ def _timeline(seed, chunks=(4096, 16384)):
     flags = dict(fuse=bool(rng.random() < 0.6), eager=bool(rng.random() < 0.4), plan_ahead=plan_ahead,
                  poll_budget_ns=3_000_000 if plan_ahead else 0)
     p = Pair(chunk, d, int(rng.integers(1, 3)), tau=int(rng.integers(1, 50)), arena_bytes=32 << 20, **flags)
+    arena_used_at_start = p.c.stats()["arena_used"]
     n = na + nb
     nbytes = elems * 4
     n_workers = max(1, int(rng.integers(1, n + 1)))
@@ -129,6 +130,9 @@ def _timeline(seed, chunks=(4096, 16384)):
     p.check_schedule(B)
     if plan_ahead:
         p.c.sync()
+    for oid in [B, A] + list(range(n)):               # consumers before what they consume; receivers go with their broadcast
+        p.delete(oid)
+    assert p.c.stats()["arena_used"] == arena_used_at_start, "arena blocks are left after every object was deleted"
     p.close()
 
 
