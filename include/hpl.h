@@ -43,7 +43,9 @@ extern "C" {
 #define HPL_ERR_INSUFFICIENT  -5  /* a Reduce is left with no live source */
 #define HPL_ERR_FAILED_WORKER -6  /* the object's only copy was owned by a failed worker */
 #define HPL_ERR_CUDA          -7  /* a CUDA call failed, or the context has no device (schedule-only) */
-#define HPL_ERR_NOMEM         -8  /* the arena is exhausted */
+#define HPL_ERR_NOMEM         -8  /* the arena is exhausted.  From a call that plans work (hpl_progress, hpl_get, any event when
+                                    eager): the collective that needed the room has nothing of that pass noted as done, what
+                                    was planned before it runs, and the call may be repeated after room was made (hpl_delete) */
 
 #define HPL_F32  0   /* 32-bit IEEE float */
 #define HPL_BF16 1   /* bfloat16; reduced in fp32, result fp32 */
@@ -62,7 +64,8 @@ typedef struct hpl_config {
     int32_t  bcast_degree;    /* concurrent sends per location, >= 1 (1 = the rule of Section 3.4.1) */
     uint64_t virt_chunk_ns;   /* virtual time for one chunk to cross one broadcast edge; 0 = chunk_bytes at 64 GiB/s */
     uint64_t poll_budget_ns;  /* bound on any device-side wait; 0 = 2 s */
-    int32_t  eager;           /* 1: every event also plans and launches what has become runnable (as hpl_progress) */
+    int32_t  eager;           /* 1: every event also plans and launches what has become runnable (as hpl_progress); an
+                                 error of that planning is returned by the event's call, the event itself has been applied */
     int32_t  plan_ahead;      /* 1: chunks of a published object that are not ready yet are planned too; the
                                  kernels poll the directory's progress counters for them (bounded) */
     int32_t  fuse;            /* 1: a subtree whose inputs are all ready is reduced in registers in one pass

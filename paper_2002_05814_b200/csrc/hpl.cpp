@@ -65,6 +65,30 @@ int flush_small(hpl_ctx* c, SmallBatch& sb) {
     return HPL_OK;
 }
 
+// Planning a collective failed (the arena is exhausted, a node is too wide for a task) after parts of the same pass
+// had been noted as planned: nothing of that pass was launched, so its notes are taken back -- to the values before,
+// the buffers were not touched -- and the caller may make room and ask again.
+void rollback_pass(hpl_ctx* c, uint64_t tag) {
+    for (auto it = c->journal.r.rbegin(); it != c->journal.r.rend(); ++it) {
+        if (it->tag != tag) continue;
+        auto f = c->reduce_of_target.find(it->target);
+        if (f == c->reduce_of_target.end()) continue;
+        ReduceOp& op = c->reduces.at(f->second);
+        if (it->pos < (int)op.merged.size()) op.merged[it->pos].set(it->a, it->b, it->old_v);
+    }
+    for (auto it = c->journal.b.rbegin(); it != c->journal.b.rend(); ++it) {
+        if (it->tag != tag) continue;
+        auto f = c->bcast_of_src.find(it->src);
+        if (f == c->bcast_of_src.end()) continue;
+        BcastOp& op = c->bcasts.at(f->second);
+        if (it->loc < (int)op.phys_have.size()) op.phys_have[it->loc] = it->old_have;
+    }
+    auto& jr = c->journal.r;
+    jr.erase(std::remove_if(jr.begin(), jr.end(), [tag](const Journal::R& e) { return e.tag == tag; }), jr.end());
+    auto& jb = c->journal.b;
+    jb.erase(std::remove_if(jb.begin(), jb.end(), [tag](const Journal::B& e) { return e.tag == tag; }), jb.end());
+}
+
 // Worker-per-GPU mode: the plan of one pass, identical on every rank, is kept as dependency levels; nothing is
 // launched here.  A task sits in the level after everything it reads: the levels of its own tree below it, the
 // collectives whose output it consumes.  hpl_run_level releases one level at a time, each rank launching the tasks
@@ -85,7 +109,10 @@ int plan_levels(hpl_ctx* c) {
             ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
             int rc = plan_reduce(c, op, tasks);
-            if (rc != HPL_OK) return rc;
+            if (rc != HPL_OK) {
+                rollback_pass(c, c->batch_tag);
+                return rc;
+            }
             int base = 0, top = 0;
             for (int p = 0; p < op.sched->k(); ++p) {
                 auto e = end_level.find(op.sched->object_at(p));
@@ -117,7 +144,10 @@ int plan_levels(hpl_ctx* c) {
             BcastOp& op = bi->second;
             std::vector<PlannedFanout> tasks;
             int rc = plan_bcast(c, op, tasks);
-            if (rc != HPL_OK) return rc;
+            if (rc != HPL_OK) {
+                rollback_pass(c, c->batch_tag);
+                return rc;
+            }
             auto e = end_level.find(op.src);
             const int lvl = (e == end_level.end() ? 0 : e->second);
             const uint32_t g = c->cfg.pipeline_chunks > 0 ? (uint32_t)c->cfg.pipeline_chunks : ~0u;
@@ -193,7 +223,11 @@ int progress(hpl_ctx* c) {
             ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
             int rc = plan_reduce(c, op, tasks);
-            if (rc != HPL_OK) return rc;
+            if (rc != HPL_OK) {   // what was planned before it runs all the same
+                rollback_pass(c, c->batch_tag);
+                flush_small(c, sb);
+                return rc;
+            }
             bool small = op.elems * 4 <= kSmallObjectBytes;
             for (auto& t : tasks) small = small && !t.poll;
             if (small && !tasks.empty()) {
@@ -219,7 +253,11 @@ int progress(hpl_ctx* c) {
             BcastOp& op = bi->second;
             std::vector<PlannedFanout> tasks;
             int rc = plan_bcast(c, op, tasks);
-            if (rc != HPL_OK) return rc;
+            if (rc != HPL_OK) {
+                rollback_pass(c, c->batch_tag);
+                flush_small(c, sb);
+                return rc;
+            }
             Object* src = find(c, op.src);
             bool small = src && src->bytes <= kSmallObjectBytes;
             for (auto& t : tasks) small = small && !t.poll;

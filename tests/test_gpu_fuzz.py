@@ -201,37 +201,73 @@ def _tight_arena_timeline(seed):
             if final:
                 p.check_schedule(tgt)
 
+    def tolerant(call, *a):
+        """The library's half of an event whose planning may run out of arena: the event itself is applied all the same
+        (the oracle's half follows), only the work it would have started is not."""
+        try:
+            call(*a)
+        except hpl.HplError as e:
+            if e.code != hpl.HPL_ERR_NOMEM:
+                raise
+            nomem[0] += 1
+
+    nomem = [0]
     try:
         for tgt, ids in ops:
             p.reduce(tgt, ids, len(ids) - 1)                # one spare each
-        pend = [i for _, ids in ops for i in ids]
-        t = 0
-        for idx in rng.permutation(len(pend)):
-            i = pend[idx]
-            t += int(rng.integers(0, 10))
-            p.advance(t)
-            if rng.random() < 0.85:
-                p.put(i, S if rng.random() < 0.7 else min(S, chunk))
-            r = rng.random()
-            if r < 0.3:
-                p.progress()
-            elif r < 0.38 and p.o.objects[i].alive:
-                p.fail(i)
-            elif r < 0.5:
-                check(ops[int(rng.integers(0, n_ops))][0], False)
-        for _, ids in ops:
-            for i in ids:
-                if p.o.objects[i].alive:
-                    t += 1
-                    p.advance(t)
-                    p.put(i)
-        for tgt, _ in ops:
-            check(tgt, True)
-    except hpl.HplError as e:
+    except hpl.HplError as e:                               # not even the outputs fit
         if e.code != hpl.HPL_ERR_NOMEM:
             raise
         p.c.shutdown()
         return None
+    pend = [i for _, ids in ops for i in ids]
+    t = 0
+    for idx in rng.permutation(len(pend)):
+        i = pend[idx]
+        t += int(rng.integers(0, 10))
+        p.advance(t)
+        if rng.random() < 0.85:
+            nb_ = S if rng.random() < 0.7 else min(S, chunk)
+            tolerant(p.c.put, i, p.dev[i].data_ptr(), nb_)
+            p.o.put(i, p.host[i], nb_)
+        r = rng.random()
+        if r < 0.3:
+            tolerant(p.progress)
+        elif r < 0.38 and p.o.objects[i].alive:
+            tolerant(p.c.fail, i)
+            p.o.fail(i)
+        elif r < 0.5:
+            tolerant(check, ops[int(rng.integers(0, n_ops))][0], False)
+    for _, ids in ops:
+        for i in ids:
+            if p.o.objects[i].alive:
+                t += 1
+                p.advance(t)
+                tolerant(p.c.put, i, p.dev[i].data_ptr(), S)
+                p.o.put(i, p.host[i], S)
+    done = []
+    for tgt, ids in ops:
+        try:
+            check(tgt, True)
+        except hpl.HplError as e:
+            if e.code != hpl.HPL_ERR_NOMEM:
+                raise
+            # a pass that ran out of arena left nothing half done: make room (the outputs checked so far go, with their
+            # partial results) and ask again
+            nomem[0] += 1
+            for d_tgt, d_ids in done:
+                p.delete(d_tgt)
+                for i in d_ids:
+                    p.delete(i)
+            done = []
+            try:
+                check(tgt, True)
+            except hpl.HplError as e2:
+                if e2.code != hpl.HPL_ERR_NOMEM:
+                    raise
+                p.c.shutdown()
+                return None
+        done.append((tgt, ids))
     ev = p.c.stats()["evictions"]
     p.close()
     return ev

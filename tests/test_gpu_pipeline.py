@@ -305,6 +305,41 @@ def test_partial_results_are_evicted_least_recently_used_when_the_arena_is_full(
     p.close()
 
 
+def test_a_pass_that_runs_out_of_arena_leaves_nothing_noted_as_done():
+    """The arena holds two outputs and nothing else.  A Get of the Reduce finds its first chunk computable in one fused
+    pass and, for the chunks behind it, needs a buffer for an inner node -- which the arena cannot give: the Get says so,
+    and nothing of that pass counts as done.  Once the other output is deleted the same Get computes every chunk."""
+    elems, chunk = 64 * 1024, 64 << 10                      # four chunks; an object is larger than the arena's slack
+    S = elems * 4
+    fixed = 4096 * 32 + 256 * 32 + (64 << 10)              # directory, error records, slack
+    p = Pair(chunk, 2, fuse=True, arena_bytes=fixed + 2 * (S + 512))
+    for i in range(6):
+        p.create(i, i, gen(("uniform",), 83, i, elems))
+    p.put(4)
+    p.put(5)
+    p.reduce(900, [4, 5], 2)                                # its output fills the second half of the arena
+    p.check_target_bits(900)
+    p.reduce(100, [0, 1, 2, 3], 4)
+    p.advance(1)
+    p.put(0)                                                # first arrival: position 3, the leaf under position 1
+    p.advance(2)
+    p.put(1)                                                # position 1: that node has everything it needs
+    p.advance(3)
+    p.put(2, chunk)                                         # the root's own object, first chunk only
+    p.advance(4)
+    p.put(3, chunk)                                         # position 2, first chunk only
+    assert p.o.reduces[100]["sched"].obj_at == [2, 1, 3, 0]
+    assert p.c.try_get(100)[0] == hpl.HPL_ERR_NOMEM
+    assert p.c.try_get(100)[0] == hpl.HPL_ERR_NOMEM         # and again: the state is as before the attempt
+    p.delete(900)
+    p.advance(5)
+    p.put(2)
+    p.put(3)
+    p.check_target_bits(100)
+    p.check_schedule(100)
+    p.close()
+
+
 def test_a_wait_that_runs_out_voids_its_own_collective_and_its_consumers_only():
     """plan_ahead: Reduce A waits for chunks of an object that never come; Reduce C consumes A's output; Reduce B, requested
     after both, has nothing to do with them.  Every Get plans A again and A's wave gives up again -- B's result, computed
