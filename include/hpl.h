@@ -24,6 +24,14 @@
  *     device except hpl_get, hpl_get_host, hpl_sync and hpl_shutdown; every wait of a kernel on
  *     a progress counter is bounded by poll_budget_ns, after which the kernel gives up, records
  *     HPL_ERR_TIMEOUT and returns (the context stays usable).
+ *
+ * Capacities
+ *   - The device directory has 4096 rows: one per published object (a put source, a joined receiver, a Reduce output,
+ *     a partial result of a tree node).  A call that needs a row when none is free returns HPL_ERR_NOMEM and changes
+ *     nothing; hpl_delete gives rows back.
+ *   - A tree node has at most 638 children (the degree that counts is min(reduce_degree, k - 1); wider stars are
+ *     refused with HPL_ERR_INVALID at hpl_reduce).  Objects, chunks and receivers per broadcast have no fixed limit:
+ *     byte offsets and element counts are 64-bit, long receiver lists are served by several waves.
  */
 #ifndef HPL_H_
 #define HPL_H_

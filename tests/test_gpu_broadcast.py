@@ -60,6 +60,29 @@ def test_all_join_before_any_launch_is_one_read_many_writes():
     p.close()
 
 
+def test_more_receivers_than_one_wave_addresses():
+    """1500 receivers of one object (a wave's table holds 1024 receiver addresses; the directory 4096 rows): the list is
+    split over waves, every receiver gets the bytes, the source is read once per wave."""
+    elems, R = 3 * 4096 + 5, 1500
+    p = Pair(16 << 10, 2, 4, tau=3)
+    p.create(0, 99, gen(("uniform",), 32, 0, elems))
+    for j in range(1, R + 1):
+        p.create(j, j % 50, nbytes=elems * 4, dtype=DT_F32)
+    p.put(0)
+    p.broadcast(0, list(range(1, R + 1)))
+    for j in range(1, R + 1):
+        p.join(j)
+    p.check_schedule(0)
+    for j in (1, 2, 1023, 1024, 1025, 1026, R - 1, R):
+        p.check_receiver_bytes(j)
+    src = p.dev[0].view(torch.uint8)
+    for j in range(1, R + 1):
+        assert torch.equal(p.dev[j], src), j
+    st = p.c.stats()
+    assert st["kernel_launches"] == 2 and st["bytes_written_planned"] == R * elems * 4
+    p.close()
+
+
 def test_partial_source_feeds_receivers_chunk_by_chunk():
     nbytes, chunk = 10 * 4096 + 40, 4096
     p = Pair(chunk, 2, 2)

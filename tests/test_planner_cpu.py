@@ -185,3 +185,35 @@ def test_small_collectives_planned_in_one_pass_share_their_launches():
             c.reduce(10_000 + r, ids, 4)
         c.progress()
         assert c.stats()["reduce_launches"] == 3
+
+
+def test_directory_rows_run_out_gracefully_and_come_back_with_delete():
+    """The device directory has 4096 rows, one per published object.  The Put that finds none free says so and changes
+    nothing; after a Delete the same Put goes through; a wider star than a task holds is refused at the request."""
+    c = hpl.Context(4096, 2, 2)
+    n = 4096 + 3
+    for i in range(n):
+        c.create(i, i, 4096)
+    for i in range(4096):
+        c.put(i, 4096 * (i + 1), 4096)
+    with pytest.raises(hpl.HplError) as e:
+        c.put(4096, 4096 * 5000, 4096)
+    assert e.value.code == hpl.HPL_ERR_NOMEM
+    with pytest.raises(hpl.HplError) as e:
+        c.reduce(9000, [0, 1], 2)                      # the output needs a row as well
+    assert e.value.code == hpl.HPL_ERR_NOMEM
+    c.delete(7)
+    c.put(4096, 4096 * 5000, 4096)
+    c.delete(8)
+    c.reduce(9000, [0, 1], 2)
+    c.progress()
+    assert c.stats()["reduce_tasks"] == 1
+    c.shutdown()
+    c = hpl.Context(4096, 1000, 2)
+    for i in range(700):
+        c.create(i, i, 4096)
+    with pytest.raises(hpl.HplError) as e:
+        c.reduce(9000, list(range(700)), 700)          # 699 children of one node
+    assert e.value.code == hpl.HPL_ERR_INVALID
+    c.reduce(9001, list(range(600)), 600)              # 599 children fit
+    c.shutdown()
