@@ -215,7 +215,8 @@ int hpl_reduce(hpl_ctx* ctx, int64_t target_id, const int64_t* src_ids, int32_t 
 int hpl_broadcast(hpl_ctx* ctx, int64_t src_id, const int64_t* dst_ids, int32_t n);
 
 /* Receiver `dst_id` asks for the object now (its Get): the directory gives it one sender and lists it as a
- * partial copy.  `dst_buf`: device buffer of the object's size (16-byte aligned), caller-owned. */
+ * partial copy.  `dst_buf`: device buffer of the object's size (16-byte aligned), caller-owned.  HPL_ERR_NOT_FOUND when
+ * `dst_id` names no receiver of a broadcast (unknown, or an object that no hpl_broadcast listed). */
 int hpl_join(hpl_ctx* ctx, int64_t dst_id, void* dst_buf);
 
 /* Get (Table 1), read-only form (Section 3.3, immutable get): waits until the object is complete, returns a
