@@ -699,12 +699,16 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     }
     uint64_t bytes = 0;
     int live = 0;
-    for (int64_t s : srcs) {
-        Object* o = find(c, s);
+    struct Src { int64_t t_arrival; int index; int64_t id; bool alive, arrived; uint32_t C; };
+    std::vector<Src> info;   // what the steps below need of each source, looked up once (the map may rehash below)
+    info.reserve(n);
+    for (int i = 0; i < n; ++i) {
+        Object* o = find(c, srcs[i]);
         if (!o) return HPL_ERR_NOT_FOUND;
         if (o->dtype != dtype || (bytes && o->bytes != bytes) || o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;
         bytes = o->bytes;
         if (o->alive) ++live;
+        info.push_back({o->t_arrival, i, o->id, o->alive, o->arrived, o->C});
     }
     if (live < 1) return HPL_ERR_INSUFFICIENT;
     const uint64_t elems = bytes / elem_size(dtype);
@@ -749,19 +753,18 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     r.red_op = op;
     r.in_dtype = dtype;
     r.elems = elems;
-    r.C = find(c, srcs[0])->C;          // chunks of this Reduce follow its inputs (chunk_bytes of the input dtype)
+    r.C = info[0].C;                    // chunks of this Reduce follow its inputs (chunk_bytes of the input dtype)
     r.chunk_elems = (uint32_t)(std::min<uint64_t>(c->cfg.chunk_bytes, bytes) / elem_size(dtype));
     if (r.chunk_elems == 0) r.chunk_elems = 1;
     r.seq = c->seq++;
     ReduceOp* rp = &r;
     auto dl = [c, rp](int64_t o) { return logical_delivered_in(c, o, *rp); };
-    for (int64_t s : srcs)
-        if (!find(c, s)->alive) r.sched->fail(s, 0, dl);  // sources lost before the call never take part
+    for (const Src& x : info)
+        if (!x.alive) r.sched->fail(x.id, 0, dl);  // sources lost before the call never take part
     std::vector<std::pair<std::pair<int64_t, int>, int64_t>> arrived;
-    for (int i = 0; i < n; ++i) {
-        Object* o = find(c, srcs[i]);
-        if (o->alive && o->arrived) arrived.push_back({{o->t_arrival, i}, o->id});
-    }
+    arrived.reserve(n);
+    for (const Src& x : info)
+        if (x.alive && x.arrived) arrived.push_back({{x.t_arrival, x.index}, x.id});
     std::sort(arrived.begin(), arrived.end());
     for (auto& a : arrived) r.sched->arrive(a.second);
     r.merged.assign(r.sched->k(), IntervalMap());

@@ -47,12 +47,23 @@ int choose_reduce_degree(int n, double size_bytes, double latency_s, double band
 
 ReduceTreeSchedule::ReduceTreeSchedule(const std::vector<int64_t>& srcs, int k, int d)
     : srcs_(srcs), k0_(k), k_(k), d_(d), at_(k, -1) {
-    for (int64_t s : srcs_) alive_[s] = true;
+    const int n = (int)srcs_.size();
+    sorted_.reserve(n);
+    for (int i = 0; i < n; ++i) sorted_.emplace_back(srcs_[i], i);
+    std::sort(sorted_.begin(), sorted_.end());
+    alive_.assign(n, 1);
+    arrived_.assign(n, 0);
+    pos_.assign(n, -1);
+}
+
+int ReduceTreeSchedule::index_of(int64_t obj) const {
+    auto it = std::lower_bound(sorted_.begin(), sorted_.end(), std::make_pair(obj, -1));
+    return (it != sorted_.end() && it->first == obj) ? it->second : -1;
 }
 
 int ReduceTreeSchedule::position_of(int64_t obj) const {
-    auto it = pos_.find(obj);
-    return it == pos_.end() ? -1 : it->second;
+    const int i = index_of(obj);
+    return i < 0 ? -1 : pos_[i];
 }
 
 bool ReduceTreeSchedule::full() const {
@@ -64,8 +75,7 @@ bool ReduceTreeSchedule::full() const {
 
 int ReduceTreeSchedule::live() const {
     int n = 0;
-    for (int64_t s : srcs_)
-        if (alive_.at(s)) ++n;
+    for (uint8_t a : alive_) n += a;
     return n;
 }
 
@@ -97,14 +107,14 @@ int ReduceTreeSchedule::first_open() const {
 
 void ReduceTreeSchedule::assign(int64_t obj, int pos) {
     at_[pos] = obj;
-    pos_[obj] = pos;
+    pos_[index_of(obj)] = pos;
     placements_.emplace_back(obj, pos);
 }
 
 void ReduceTreeSchedule::arrive(int64_t obj) {
-    auto it = alive_.find(obj);
-    if (it == alive_.end() || !it->second || arrived_.count(obj)) return;
-    arrived_[obj] = true;
+    const int i = index_of(obj);
+    if (i < 0 || !alive_[i] || arrived_[i]) return;
+    arrived_[i] = 1;
     const int p = first_open();
     if (p < 0)
         spares_.push_back(obj);
@@ -113,25 +123,24 @@ void ReduceTreeSchedule::arrive(int64_t obj) {
 }
 
 void ReduceTreeSchedule::rejoin(int64_t obj) {
-    auto it = alive_.find(obj);
-    if (it == alive_.end() || it->second) return;
-    it->second = true;
-    arrived_.erase(obj);
+    const int i = index_of(obj);
+    if (i < 0 || alive_[i]) return;
+    alive_[i] = 1;
+    arrived_[i] = 0;
 }
 
 ReduceInvalidation ReduceTreeSchedule::fail(int64_t obj, int64_t delivered,
                                             const std::function<int64_t(int64_t)>& delivered_of) {
     ReduceInvalidation inv;
     filled_prefix_ = 0;   // a position may open anywhere
-    auto it = alive_.find(obj);
-    if (it == alive_.end() || !it->second) return inv;
-    it->second = false;
+    const int i = index_of(obj);
+    if (i < 0 || !alive_[i]) return inv;
+    alive_[i] = 0;
     auto sp = std::find(spares_.begin(), spares_.end(), obj);
     if (sp != spares_.end()) spares_.erase(sp);
-    auto pit = pos_.find(obj);
-    if (pit != pos_.end()) {
-        const int p = pit->second;
-        pos_.erase(pit);
+    if (pos_[i] >= 0) {
+        const int p = pos_[i];
+        pos_[i] = -1;
         at_[p] = -1;
         ++epoch_;
         inv.positions.push_back(p);
@@ -169,7 +178,7 @@ void ReduceTreeSchedule::shrink(int p, int64_t old_obj, int64_t hi_failed,
     inv.touched.push_back(q);
     int64_t dest = -1, hi_moved = 0, moved_from = -1, new_obj = -1;
     if (q != p && moved >= 0) {
-        pos_.erase(moved);
+        pos_[index_of(moved)] = -1;
         dest = p >= 0 ? p : first_open();
         hi_moved = delivered_of ? delivered_of(moved) : 0;
         moved_from = q;

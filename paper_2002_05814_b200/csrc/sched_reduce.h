@@ -11,7 +11,6 @@
 #pragma once
 #include <cstdint>
 #include <functional>
-#include <unordered_map>
 #include <vector>
 
 namespace hpl {
@@ -39,7 +38,7 @@ public:
     int d() const { return d_; }
     int64_t object_at(int pos) const { return at_[pos]; }
     int position_of(int64_t obj) const;
-    bool has_source(int64_t obj) const { return alive_.count(obj) != 0; }
+    bool has_source(int64_t obj) const { return index_of(obj) >= 0; }
     bool full() const;
     int live() const;
     const std::vector<int64_t>& sources() const { return srcs_; }
@@ -66,9 +65,11 @@ private:
     std::vector<int64_t> srcs_;
     int k0_, k_, d_;
     int64_t epoch_ = 0;
-    std::unordered_map<int64_t, bool> alive_;
-    std::unordered_map<int64_t, bool> arrived_;
-    std::unordered_map<int64_t, int> pos_;
+    // per source, by its index in srcs_ (found through the sorted list: no allocation per source, per event)
+    int index_of(int64_t obj) const;
+    std::vector<std::pair<int64_t, int>> sorted_;   // (object id, index in srcs_)
+    std::vector<uint8_t> alive_, arrived_;
+    std::vector<int> pos_;                          // position in the tree, -1 = none
     std::vector<int64_t> at_;
     std::vector<int64_t> spares_;
     std::vector<std::pair<int64_t, int>> placements_;
