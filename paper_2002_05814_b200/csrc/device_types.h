@@ -57,6 +57,18 @@ inline unsigned long long pack_step(const ReduceStep& st) {
     return (st.ptr & ((1ull << kRecShift) - 1)) | (meta << kRecShift);
 }
 
+// Tile size of a fan-out wave.  A tile is one CTA's unit of work: read once, then one bulk copy per receiver, a chain of
+// latencies.  When an object has far fewer full tiles than there are resident CTAs (`slots`) the tiles are made smaller
+// so that more CTAs share the chain -- 256 KiB to 16 receivers is 8 full tiles, or 64 tiles of 4 KiB on 64 CTAs, a
+// third faster.  From a quarter of the slots upwards the full tile stays (measured: nothing to gain there).
+inline uint32_t spread_tile_bytes(unsigned long long full_tiles, unsigned long long slots, uint32_t full, uint32_t gran, uint32_t floor) {
+    if (full_tiles == 0 || full_tiles * 4 >= slots) return full;
+    unsigned long long size = ((unsigned long long)full * full_tiles + slots - 1) / slots;
+    size = (size + gran - 1) / gran * gran;
+    if (size < floor) size = floor;
+    return size > full ? full : (uint32_t)size;
+}
+
 struct ReduceTask {
     unsigned long long out_ptr;   // fp32 result (partial or target)
     unsigned long long elems;     // elements in the whole object
@@ -94,6 +106,7 @@ struct FanoutTask {
     uint32_t src_row;                // its directory row (polled when the task polls)
     uint32_t c_begin, c_end;
     uint32_t tiles_per_chunk;
+    uint32_t tile_bytes;             // bytes per tile: kFanoutTileBytes, or fewer for small objects (a multiple of 512)
     uint32_t tile_begin;
     uint32_t dst_begin, n_dst;
     uint32_t poll;

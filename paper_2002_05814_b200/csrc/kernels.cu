@@ -471,8 +471,8 @@ __global__ void __launch_bounds__(kFanoutThreads) fanout_wave_kernel(const __gri
         const unsigned int lt = g - task.tile_begin;
         const unsigned int c = task.c_begin + lt / task.tiles_per_chunk;
         const unsigned int j = lt % task.tiles_per_chunk;
-        const unsigned long long b0 = (unsigned long long)c * task.chunk_bytes + (unsigned long long)j * kFanoutTileBytes;
-        unsigned long long b1 = b0 + kFanoutTileBytes;
+        const unsigned long long b0 = (unsigned long long)c * task.chunk_bytes + (unsigned long long)j * task.tile_bytes;
+        unsigned long long b1 = b0 + task.tile_bytes;
         const unsigned long long chunk_end = (unsigned long long)(c + 1) * task.chunk_bytes;
         if (b1 > chunk_end) b1 = chunk_end;
         if (b1 > task.bytes) b1 = task.bytes;

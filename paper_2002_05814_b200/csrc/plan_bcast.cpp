@@ -151,6 +151,7 @@ int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanou
             d.c_begin = tt.a;
             d.c_end = tt.b;
             d.tiles_per_chunk = tpc;
+            d.tile_bytes = kFanoutTileBytes;
             d.tile_begin = w.total_tiles;
             d.dst_begin = n_dst;
             d.n_dst = (uint32_t)tt.dst.size();
@@ -178,6 +179,17 @@ int launch_fanout_group(hpl_ctx* c, std::vector<std::pair<BcastOp*, PlannedFanou
             continue;
         }
         if (c->occ_fanout == 0) c->occ_fanout = fanout_ctas_per_sm();
+        const uint32_t tb = spread_tile_bytes(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout, kFanoutTileBytes, 512, 4096);
+        if (tb != (uint32_t)kFanoutTileBytes) {
+            w.total_tiles = 0;
+            for (uint32_t q = 0; q < w.n_tasks; ++q) {
+                FanoutTask& d = w.tasks[q];
+                d.tile_bytes = tb;
+                d.tiles_per_chunk = (uint32_t)((std::min<uint64_t>(d.chunk_bytes, d.bytes) + tb - 1) / tb);
+                d.tile_begin = w.total_tiles;
+                w.total_tiles += (d.c_end - d.c_begin) * d.tiles_per_chunk;
+            }
+        }
         int grid = (int)std::min<uint64_t>(w.total_tiles, (uint64_t)c->n_sm * c->occ_fanout);
         if (grid < 1) grid = 1;
         if (flush_directory(c) != HPL_OK) return HPL_ERR_CUDA;
