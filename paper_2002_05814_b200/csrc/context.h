@@ -143,6 +143,40 @@ struct Arena {
 
 enum ObjKind { OBJ_PLAIN = 0, OBJ_TARGET = 1, OBJ_RECEIVER = 2, OBJ_PARTIAL = 3 };
 
+// The Reduces that name an object as a source (keys of `reduces`), in creation order.  Almost always one: that one
+// lives in the object itself, so that a Reduce request allocates nothing per source.
+struct ConsumerList {
+    uint64_t first = 0;
+    bool has_first = false;
+    std::vector<uint64_t> rest;
+    bool empty() const { return !has_first; }
+    void push_back(uint64_t key) {
+        if (!has_first) {
+            first = key;
+            has_first = true;
+        } else {
+            rest.push_back(key);
+        }
+    }
+    void erase(uint64_t key) {
+        if (has_first && first == key) {
+            has_first = !rest.empty();
+            if (has_first) {
+                first = rest.front();
+                rest.erase(rest.begin());
+            }
+        } else {
+            rest.erase(std::remove(rest.begin(), rest.end(), key), rest.end());
+        }
+    }
+    template <class F>
+    void for_each(F f) const {
+        if (!has_first) return;
+        f(first);
+        for (uint64_t key : rest) f(key);
+    }
+};
+
 struct Object {
     int64_t id = 0;
     int32_t worker = -1;
@@ -166,6 +200,7 @@ struct Object {
     int pos = -1;              // partial result: its tree position (op_key = the Reduce's target)
     uint64_t last_use = 0;     // partial result: when a planning pass last wrote or read it (eviction order)
     uint64_t last_pass = 0;    //                 and which pass that was
+    ConsumerList consumers;    // the Reduces it is a source of
 };
 
 struct Journal {  // what was planned since the last successful wait (undone if a device wait expires)
@@ -262,7 +297,6 @@ struct hpl_ctx {
     std::map<uint64_t, BcastOp> bcasts;
     std::unordered_map<int64_t, uint64_t> reduce_of_target, bcast_of_src;
     std::set<uint64_t> composed_bcasts;   // keys of the broadcasts whose source is a Reduce output, in creation order
-    std::unordered_map<int64_t, std::vector<uint64_t>> reduces_of_source;   // source id -> the Reduces that name it (keys of `reduces`)
     Journal journal;
     bool work_in_flight = false;
     bool polling_in_flight = false;   // some wave in flight polls progress counters (only those can record an error)

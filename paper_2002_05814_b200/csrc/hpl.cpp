@@ -408,12 +408,11 @@ void invalidate_consumers(hpl_ctx* c, int64_t target) {
 }
 
 void notify_arrival(hpl_ctx* c, Object& o) {
-    auto it = c->reduces_of_source.find(o.id);
-    if (it == c->reduces_of_source.end()) return;
-    for (uint64_t key : it->second) {   // in creation order
+    const int64_t id = o.id;
+    o.consumers.for_each([c, id](uint64_t key) {   // in creation order
         auto r = c->reduces.find(key);
-        if (r != c->reduces.end()) r->second.sched->arrive(o.id);
-    }
+        if (r != c->reduces.end()) r->second.sched->arrive(id);
+    });
 }
 
 int do_put_common(hpl_ctx* c, Object& o, uint64_t bytes, bool first) {
@@ -699,8 +698,8 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     }
     uint64_t bytes = 0;
     int live = 0;
-    struct Src { int64_t t_arrival; int index; int64_t id; bool alive, arrived; uint32_t C; };
-    std::vector<Src> info;   // what the steps below need of each source, looked up once (the map may rehash below)
+    struct Src { int64_t t_arrival; int index; int64_t id; bool alive, arrived; uint32_t C; Object* o; };
+    std::vector<Src> info;   // what the steps below need of each source, looked up once (entries of the object table do not move)
     info.reserve(n);
     for (int i = 0; i < n; ++i) {
         Object* o = find(c, srcs[i]);
@@ -708,7 +707,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
         if (o->dtype != dtype || (bytes && o->bytes != bytes) || o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;
         bytes = o->bytes;
         if (o->alive) ++live;
-        info.push_back({o->t_arrival, i, o->id, o->alive, o->arrived, o->C});
+        info.push_back({o->t_arrival, i, o->id, o->alive, o->arrived, o->C, o});
     }
     if (live < 1) return HPL_ERR_INSUFFICIENT;
     const uint64_t elems = bytes / elem_size(dtype);
@@ -770,7 +769,7 @@ int hpl_reduce(hpl_ctx* c, int64_t target, const int64_t* src_ids, int32_t n, in
     r.merged.assign(r.sched->k(), IntervalMap());
     r.partial_key.assign(r.sched->k(), 0);
     const uint64_t key = r.seq;
-    for (int64_t sid : srcs) c->reduces_of_source[sid].push_back(key);
+    for (const Src& x : info) x.o->consumers.push_back(key);
     c->reduce_of_target[target] = key;
     c->reduces.emplace(key, std::move(r));
     refresh_composed(c);
@@ -916,8 +915,11 @@ int hpl_rejoin(hpl_ctx* c, int32_t worker) {
         o.lib_owned = false;
         o.from_host = false;
         o.async_counter = false;
-        for (auto& rk : c->reduces)
-            if (rk.second.sched->has_source(o.id)) rk.second.sched->rejoin(o.id);
+        const int64_t id = o.id;
+        o.consumers.for_each([c, id](uint64_t key) {
+            auto r = c->reduces.find(key);
+            if (r != c->reduces.end()) r->second.sched->rejoin(id);
+        });
     }
     return after_event(c);
 }
@@ -1110,10 +1112,7 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
     if (!o || id < 0) return HPL_ERR_NOT_FOUND;
     if (!c->levels.empty()) return HPL_ERR_INVALID;       // worker-per-GPU mode: a planned level may still name it
     if (o->kind == OBJ_RECEIVER) return HPL_ERR_INVALID;  // deleted with its broadcast
-    {
-        auto it = c->reduces_of_source.find(id);
-        if (it != c->reduces_of_source.end() && !it->second.empty()) return HPL_ERR_INVALID;  // still referenced by a Reduce
-    }
+    if (!o->consumers.empty()) return HPL_ERR_INVALID;  // still referenced by a Reduce
     if (c->device && (c->work_in_flight || c->copy_pending || c->ctl_unconfirmed)) {
         // rows and arena memory are recycled only when nothing enqueued can still read them (nothing of the
         // library's is in flight after a Get or a wait, so a round's Deletes cost no device wait)
@@ -1133,10 +1132,8 @@ int hpl_delete(hpl_ctx* c, int64_t id) {
                 }
             }
         for (int64_t sid : op.sched->sources()) {
-            auto it = c->reduces_of_source.find(sid);
-            if (it == c->reduces_of_source.end()) continue;
-            it->second.erase(std::remove(it->second.begin(), it->second.end(), key), it->second.end());
-            if (it->second.empty()) c->reduces_of_source.erase(it);
+            Object* so = find(c, sid);
+            if (so) so->consumers.erase(key);
         }
         c->reduces.erase(key);
         c->reduce_of_target.erase(id);

@@ -240,8 +240,12 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         Planning(hpl_ctx* ctx, int64_t t) : c(ctx) { c->planning_target = t; }
         ~Planning() { c->planning_target = -1; }
     } planning(c, op.target);
-    std::vector<uint32_t> ready(k, 0), landed(k, 0);
-    std::vector<uint32_t> bp = {0u, op.C};
+    // scratch that keeps its memory between calls (planning is not re-entrant: one pass at a time per thread)
+    static thread_local std::vector<uint32_t> ready, landed, bp;
+    static thread_local ReducePlanCtx p;
+    ready.assign(k, 0);
+    landed.assign(k, 0);
+    bp.assign({0u, op.C});
     for (int p = 0; p < k; ++p) {
         op.merged[p].breakpoints(bp);
         const int64_t oid = s.object_at(p);
@@ -263,7 +267,7 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
     bp.erase(std::unique(bp.begin(), bp.end()), bp.end());
 
     for (size_t i = 0; i + 1 < bp.size(); ++i) {
-        ReducePlanCtx p;
+        p.err = HPL_OK;
         p.c = c;
         p.op = &op;
         p.a = bp[i];
