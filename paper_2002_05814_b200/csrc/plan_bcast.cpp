@@ -106,9 +106,7 @@ int plan_bcast(hpl_ctx* c, BcastOp& op, std::vector<PlannedFanout>& tasks) {
                 }
             }
             if (!merged) {
-                PlannedFanout t{loc, a, b, poll};
-                t.level = level;
-                t.dst = g.second;
+                PlannedFanout t{loc, a, b, poll, level, g.second};
                 tasks.push_back(std::move(t));
             }
         }

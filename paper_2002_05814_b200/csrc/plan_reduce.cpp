@@ -307,6 +307,7 @@ int plan_reduce(hpl_ctx* c, ReduceOp& op, std::vector<PlannedReduceTask>& tasks)
         } else {
             visit_for_progress(p, 0);
         }
+        p.out = nullptr;   // (the scratch outlives this call; `local` does not)
         if (p.err != HPL_OK) return p.err;
         for (auto& t : local) {
             c->journal.r.push_back({op.target, t.pos, t.a, t.b, p.m0[t.pos], c->batch_tag});
