@@ -83,6 +83,25 @@ def test_more_receivers_than_one_wave_addresses():
     p.close()
 
 
+def test_a_small_object_is_spread_over_more_ctas_than_it_has_full_tiles():
+    """256 KiB is 8 tiles of 32 KiB -- far fewer than there are CTAs: the wave uses 4 KiB tiles (64 of them); a 16 MiB
+    object keeps the full tile.  Ragged sizes stay exact either way."""
+    for nbytes, want_tiles in ((256 << 10, 64), ((256 << 10) + 36, 65), (16 << 20, 512)):
+        p = Pair(1 << 20, 2, 2)
+        p.create(0, 99, gen(("uniform",), 33, 0, nbytes // 4))
+        for j in range(1, 5):
+            p.create(j, j, nbytes=nbytes, dtype=DT_F32)
+        p.put(0)
+        p.broadcast(0, [1, 2, 3, 4])
+        for j in range(1, 5):
+            p.join(j)
+        for j in range(1, 5):
+            p.check_receiver_bytes(j)
+        st = p.c.stats()
+        assert st["kernel_launches"] == 1 and st["tiles"] == want_tiles, (nbytes, st["tiles"])
+        p.close()
+
+
 def test_partial_source_feeds_receivers_chunk_by_chunk():
     nbytes, chunk = 10 * 4096 + 40, 4096
     p = Pair(chunk, 2, 2)

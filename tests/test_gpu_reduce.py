@@ -416,3 +416,34 @@ def test_gaussian_inputs_with_real_tails_stay_within_the_fp64_bound():
         got = p.check_target_bits(100).cpu().numpy()
         assert _norm_err(got, ov.naive_sum_f64(list(range(k)), p.host)) <= 1e-5 * 4
         p.close()
+
+
+def test_the_readme_example_runs_as_written():
+    """The minimal use shown in the README, with smaller objects: the calls and their keyword names stay valid."""
+    arena = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    ctx = hpl.Context(chunk_bytes=1 << 20, reduce_degree=2, bcast_degree=2,
+                      arena=arena.data_ptr(), arena_bytes=arena.numel(),
+                      stream=torch.cuda.current_stream().cuda_stream)
+    grads = [torch.randn(1 << 18, device="cuda") for _ in range(16)]
+    for i, g in enumerate(grads):
+        ctx.create(i, worker=i, total_bytes=g.numel() * 4)
+    ctx.reduce(100, list(range(16)), k_first_ready=8)
+    order = [3, 0, 9, 12, 5, 1, 14, 7]
+    for t, i in enumerate(order):
+        ctx.advance(1000 * (t + 1))
+        ctx.put(i, grads[i].data_ptr(), grads[i].numel() * 4)
+    ptr, nbytes = ctx.get(100)
+    assert nbytes == (1 << 18) * 4
+    off = ptr - arena.data_ptr()
+    got = arena[off:off + nbytes].view(torch.float32)
+    want = torch.stack([grads[i] for i in order]).double().sum(0)
+    assert torch.allclose(got.double(), want, rtol=0, atol=1e-5 * 3 * float(want.abs().max()))
+    ctx.fail(9)                                      # its position stays open for the next arrival
+    assert ctx.try_get(100)[0] == hpl.HPL_ERR_TIMEOUT
+    ctx.advance(20000)
+    ctx.put(2, grads[2].data_ptr(), grads[2].numel() * 4)
+    ptr, nbytes = ctx.get(100)
+    got = arena[ptr - arena.data_ptr():ptr - arena.data_ptr() + nbytes].view(torch.float32)
+    want = torch.stack([grads[i] for i in order if i != 9] + [grads[2]]).double().sum(0)
+    assert torch.allclose(got.double(), want, rtol=0, atol=1e-5 * 3 * float(want.abs().max()))
+    ctx.shutdown()
