@@ -215,7 +215,7 @@ class Runner:
         """Event lists of round ``r``: (first part, second part, deletes, h2d bytes, d2h bytes).  The first part
         holds the broadcast of the round (if any), the second the reduce; each is applied by ONE hpl_submit.
         ``marks``: three CUDA event handles the library records on its stream at the start of the step, between
-        the two parts and at the end (device timing without a foreign call of its own)."""
+        the two parts (when the step has two) and at the end (device timing without a foreign call of its own)."""
         H, w = self.hpl, self.w
         S = w.object_bytes
         t = (r + 1) * 2_000_000_000
@@ -226,7 +226,6 @@ class Runner:
             e2, dl = H.EventList(8 + m * (2 * n + 2)), H.EventList(4 + m * (n + 1))
             if marks:
                 e2.add(H.HPL_EV_MARK, 0, ptr=marks[0])
-                e2.add(H.HPL_EV_MARK, 0, ptr=marks[1])
             for q in range(m):
                 ids = list(range(q * n, (q + 1) * n))
                 for i in ids:
@@ -283,7 +282,7 @@ class Runner:
                 e1.add(H.HPL_EV_GET, 0, dsts[j])          # every receiver's Get
             t += 200_000_000                             # the Gets let virtual time run until the copies had landed
             dl.add(H.HPL_EV_DELETE, 0, src_id)
-        if marks:
+        if marks and w.kind == "round":                  # (a step with one part is timed from its first mark to its last)
             first.add(H.HPL_EV_MARK, 0, ptr=marks[1])
         if w.kind in ("reduce", "round", "ft_reduce"):
             if not early:
@@ -383,7 +382,7 @@ def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
         runner.mid_event = lambda: ev[cur["i"]][1].record()
         runner.end_event = lambda: ev[cur["i"]][2].record()
     else:
-        # device-resident step: the library records the three events itself, inside hpl_submit (HPL_EV_MARK)
+        # device-resident step: the library records the events itself, inside hpl_submit (HPL_EV_MARK)
         for tri in ev:
             for e in tri:
                 e.record()              # creates the underlying CUDA event
@@ -407,9 +406,14 @@ def time_steps(runner: Runner, steps: int, warmup: int, dist=None):
     wall_ms = (time.perf_counter() - t0) * 1e3
     st1 = runner.ctx.stats()
     runner.mid_event = runner.end_event = lambda: None
-    bc = [e[0].elapsed_time(e[1]) for e in ev]
-    rd = [e[1].elapsed_time(e[2]) for e in ev]
     tot = [e[0].elapsed_time(e[2]) for e in ev]
+    if runner.w.kind == "round" or runner.host_buffers:
+        bc = [e[0].elapsed_time(e[1]) for e in ev]
+        rd = [e[1].elapsed_time(e[2]) for e in ev]
+    elif runner.w.kind == "broadcast":
+        bc, rd = tot, [0.0] * len(tot)
+    else:
+        bc, rd = [0.0] * len(tot), tot
     delta = {k: st1[k] - st0[k] for k in st1}
     return {"bcast_ms": bc, "reduce_ms": rd, "total_ms": tot, "wall_ms": wall_ms, "stats": delta,
             "h2d": h2d, "d2h": d2h}
