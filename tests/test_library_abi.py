@@ -99,3 +99,35 @@ def test_batch_calls_are_the_single_calls_in_array_order():
         assert ei.value.code == hpl.HPL_ERR_EXISTS
         with pytest.raises(hpl.HplError):
             a.create(60, 0, 256)
+
+
+def test_the_header_is_plain_c_and_the_library_links_from_c(tmp_path):
+    """include/hpl.h compiles as pedantic C99 and a C program linked against the library gets, for the same calls,
+    the schedule the Python binding gets."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    libdir = os.path.dirname(hpl.lib_path())
+    exe = str(tmp_path / "abi_from_c")
+    lib = os.path.basename(hpl.lib_path())[3:-3]                       # libhpl.so -> hpl
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(root, "include"),
+                    os.path.join(root, "tests", "abi_from_c.c"), "-L", libdir, "-l" + lib, "-Wl,-rpath," + libdir, "-o", exe],
+                   check=True, capture_output=True)
+    out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout.splitlines()
+    with hpl.Context(chunk_bytes=64) as c:
+        for i in (1, 2, 3):
+            c.create(i, i - 1, 256)
+        c.reduce(9, [1, 2, 3], 2)
+        c.advance(10)
+        c.put(2, 4096, 256)
+        c.advance(20)
+        c.put(3, 8192, 128)
+        assert [int(x) for x in out[0].split()] == c.schedule_dump(9)
+    assert out[1] == lib_strerror(hpl.HPL_ERR_TIMEOUT)
+
+
+def lib_strerror(code):
+    return hpl.load_library().hpl_strerror(code).decode()
