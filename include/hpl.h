@@ -23,7 +23,9 @@
  *   - All device work is enqueued on the stream given to hpl_init().  No call blocks on the
  *     device except hpl_get, hpl_get_host, hpl_sync and hpl_shutdown; every wait of a kernel on
  *     a progress counter is bounded by poll_budget_ns, after which the kernel gives up, records
- *     HPL_ERR_TIMEOUT and returns (the context stays usable).
+ *     HPL_ERR_TIMEOUT and returns (the context stays usable).  One more wait exists: when the arena is full, a call
+ *     that plans work waits for what is enqueued before it drops partial results (least recently used first; sources,
+ *     Reduce outputs and store copies of host objects are never dropped) and, if need be, plans again.
  *
  * Capacities
  *   - The device directory has 4096 rows: one per published object (a put source, a joined receiver, a Reduce output,

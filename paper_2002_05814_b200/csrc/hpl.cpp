@@ -223,6 +223,19 @@ int progress(hpl_ctx* c) {
             ReduceOp& op = ri->second;
             std::vector<PlannedReduceTask> tasks;
             int rc = plan_reduce(c, op, tasks);
+            if (rc == HPL_ERR_NOMEM && c->device && (c->work_in_flight || !sb.empty())) {
+                // The arena is full of partial results that this pass itself (or work still in flight) uses.  What was
+                // planned so far runs to its end; after that those buffers may go, least recently used first, and this
+                // Reduce is planned again, as a pass of its own.
+                rollback_pass(c, c->batch_tag);
+                int rc2 = flush_small(c, sb);
+                if (rc2 == HPL_OK) rc2 = sync_and_check(c);
+                if (rc2 != HPL_OK) return rc2;
+                ++c->plan_pass;
+                c->batch_tag = ++c->tag_counter;
+                tasks.clear();
+                rc = plan_reduce(c, op, tasks);
+            }
             if (rc != HPL_OK) {   // what was planned before it runs all the same
                 rollback_pass(c, c->batch_tag);
                 flush_small(c, sb);
