@@ -148,3 +148,25 @@ def test_calls_of_the_other_modes_and_helpers():
     for f in (lib.hpl_progress, lib.hpl_sync, lib.hpl_shutdown):
         assert f(None) == I
     c.shutdown()
+
+
+def test_an_object_named_by_several_reduces_is_held_until_the_last_one_is_deleted():
+    c = _ctx()
+    I = hpl.HPL_ERR_INVALID
+    c.reduce(100, [0, 1], 2)
+    c.reduce(101, [1, 2], 2)
+    c.reduce(102, [1, 3, 4], 2)
+    c.put(1, 1 << 20, S)                                # one arrival, noted by all three trees, in the order of their requests
+    for tgt in (100, 101, 102):
+        assert 1 in c.schedule_dump(tgt)[7:9]           # the first placement: (object 1, its position)
+    assert _code(c.delete, 1) == I
+    c.delete(101)
+    assert _code(c.delete, 1) == I
+    c.delete(100)
+    assert _code(c.delete, 1) == I                      # 102 still names it
+    c.put(3, 1 << 21, S)
+    c.delete(102)
+    c.delete(1)
+    c.delete(3)
+    assert c.try_get(1)[0] == hpl.HPL_ERR_NOT_FOUND
+    c.shutdown()
